@@ -1,0 +1,145 @@
+"""CPU oracle (test infrastructure): ctypes access to ``strata_oracle.c``.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg import this
+package.  It never imports the CUDA binding, and the CUDA binding never
+imports it.  Arrays are numpy; bf16 travels as uint16 bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Dict, Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "strata_oracle.c")
+_LIB = os.path.join(_HERE, "libstrata_oracle.so")
+_lib: Optional[ctypes.CDLL] = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (IEEE arithmetic: no fast-math, no contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-march=native", "-fno-fast-math", "-ffp-contract=off", "-fopenmp",
+               "-std=c11", "-Wall", "-Wextra", "-shared", "-fPIC", _SRC, "-o", _LIB + ".tmp", "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(_LIB + ".tmp", _LIB)
+    return _LIB
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        i32, i64, vp = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p
+        L.oracle_layout.restype = i64
+        L.oracle_layout.argtypes = [i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.oracle_dispatch_bf16.restype = None
+        L.oracle_dispatch_bf16.argtypes = [i64, i32, i32, vp, vp, vp, i32]
+        L.oracle_dispatch_fp8.restype = None
+        L.oracle_dispatch_fp8.argtypes = [i64, i32, i32, vp, vp, vp, vp, i32]
+        L.oracle_combine.restype = None
+        L.oracle_combine.argtypes = [i64, i32, i32, vp, vp, vp, vp, i32]
+        L.oracle_e4m3_encode.restype = ctypes.c_uint8
+        L.oracle_e4m3_encode.argtypes = [ctypes.c_float]
+        L.oracle_max_threads.restype = i32
+        L.oracle_max_threads.argtypes = []
+        _lib = L
+    return _lib
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype) -> np.ndarray:
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def max_threads() -> int:
+    return int(lib().oracle_max_threads())
+
+
+class BadExpertId(ValueError):
+    def __init__(self, item: int):
+        super().__init__(f"expert id out of range at flat item {item}")
+        self.item = item
+
+
+def layout(ids: np.ndarray, E: int) -> Dict[str, np.ndarray]:
+    """Routing layout of ids int32 [R,T,K]; raises BadExpertId for an id outside [0,E)."""
+    ids = _c(ids, np.int32)
+    R, T, K = ids.shape
+    N = R * T * K
+    out = {
+        "expert_count": np.zeros(E, np.int32),
+        "expert_offset": np.zeros(E + 1, np.int32),
+        "rank_count": np.zeros(R, np.int32),
+        "rank_offset": np.zeros(R + 1, np.int32),
+        "src_expert_count": np.zeros((R, E), np.int32),
+        "dst_row": np.full((R, T, K), -1, np.int32),
+        "src_of_row": np.full(N, -1, np.int32),
+    }
+    rc = lib().oracle_layout(R, T, K, E, _p(ids), _p(out["expert_count"]), _p(out["expert_offset"]),
+                             _p(out["rank_count"]), _p(out["rank_offset"]), _p(out["src_expert_count"]),
+                             _p(out["dst_row"]), _p(out["src_of_row"]))
+    if rc < 0:
+        if rc < -(1 << 40):
+            raise ValueError("invalid shape (need R,K,E > 0 and E % R == 0)")
+        raise BadExpertId(int(-rc - 1))
+    return out
+
+
+def dispatch_bf16(dst_row: np.ndarray, x: np.ndarray, nthreads: int = 1,
+                  recv: Optional[np.ndarray] = None) -> np.ndarray:
+    """recv uint16 [N,H] with recv[dst_row[i]] = x[i // K]."""
+    dst_row = _c(dst_row, np.int32)
+    K = dst_row.shape[-1]
+    H = x.shape[-1]
+    x2 = _c(x, np.uint16).reshape(-1, H)
+    n_tok = x2.shape[0]
+    assert dst_row.size == n_tok * K
+    if recv is None:
+        recv = np.empty((n_tok * K, H), np.uint16)
+    assert recv.dtype == np.uint16 and recv.flags.c_contiguous
+    lib().oracle_dispatch_bf16(n_tok, K, H, _p(dst_row), _p(x2), _p(recv), nthreads)
+    return recv
+
+
+def dispatch_fp8(dst_row: np.ndarray, x: np.ndarray, nthreads: int = 1):
+    """(recv_q uint8 [N,H], recv_scale float32 [N,H/128])."""
+    dst_row = _c(dst_row, np.int32)
+    K = dst_row.shape[-1]
+    H = x.shape[-1]
+    assert H % 128 == 0
+    x2 = _c(x, np.uint16).reshape(-1, H)
+    n_tok = x2.shape[0]
+    assert dst_row.size == n_tok * K
+    q = np.empty((n_tok * K, H), np.uint8)
+    s = np.empty((n_tok * K, H // 128), np.float32)
+    lib().oracle_dispatch_fp8(n_tok, K, H, _p(dst_row), _p(x2), _p(q), _p(s), nthreads)
+    return q, s
+
+
+def combine(dst_row: np.ndarray, y: np.ndarray, w: np.ndarray, nthreads: int = 1) -> np.ndarray:
+    """out uint16 [n_tok,H] = bf16(sum_k w[n,k] * y[dst_row[n,k]]) (fp32 FMA chain, slot order)."""
+    dst_row = _c(dst_row, np.int32)
+    K = dst_row.shape[-1]
+    y = _c(y, np.uint16)
+    H = y.shape[-1]
+    w2 = _c(w, np.float32).reshape(-1, K)
+    n_tok = w2.shape[0]
+    assert dst_row.size == n_tok * K
+    out = np.empty((n_tok, H), np.uint16)
+    lib().oracle_combine(n_tok, K, H, _p(dst_row), _p(y), _p(w2), _p(out), nthreads)
+    return out
+
+
+def e4m3_encode(v: np.ndarray) -> np.ndarray:
+    """uint8 codes of a float32 array (scalar loop in C; for tests)."""
+    v = _c(v, np.float32)
+    f = lib().oracle_e4m3_encode
+    return np.fromiter((f(float(t)) for t in v.ravel()), dtype=np.uint8, count=v.size).reshape(v.shape)

@@ -1,0 +1,286 @@
+/*
+ * CPU oracle for MoE routing layout, token dispatch and gate-weighted combine.
+ *
+ * THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  It is the plain definition of
+ * what the GPU path must compute, written to be checked against the paper by
+ * eye: one loop per definition, no blocking, no fusion, no reordering.  It
+ * shares no code, header, table or constant with the CUDA library and neither
+ * includes the other.  Only tests, the smoke check and the CPU-baseline leg of
+ * the benchmark may call it.
+ *
+ * What it follows:
+ *  - Routing metadata (paper App. C, "token placement"): destination expert,
+ *    per-expert counts, prefix-sum offsets and token-local offsets, which
+ *    dispatch and combine both reuse.
+ *  - Dispatch (paper Sec. 6.2 / 7.1): each routed token's hidden vector is
+ *    moved to the receive segment of the rank that owns its expert, directly
+ *    into the user buffer (no staging copy).
+ *  - Combine (paper Sec. 6.1, reduction-bearing operators): the top-k expert
+ *    outputs of a token are accumulated into the token's local destination.
+ * The paper prints no pseudo-code, layout, dtype or worked example for this
+ * path; the concrete conventions below (segment order expert -> source rank ->
+ * token -> slot, packed segments, contiguous expert->rank blocks, fp32 FMA in
+ * slot order, e4m3 with one scale per 128 columns) are this build's stated
+ * readings of it.
+ *
+ * Pins (tests/test_oracle_*.py): sort-based brute force, a hand-worked
+ * example, closed forms (E=1; round-robin ids), bijection/ordering invariants,
+ * row-equality after dispatch, nearest-code brute force and a library cast for
+ * the e4m3 encoder, identity/one-hot/K=1/doubling/fp64 checks for combine.
+ * No function here is "parity unpinned".
+ *
+ * Index convention: rank r in [0,R), token t in [0,T), slot k in [0,K),
+ * flat item i = (r*T + t)*K + k, token n = r*T + t, N = R*T*K.
+ * bf16 values travel as uint16_t bit patterns.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ------------------------------------------------------------------ */
+/* O1: routing layout = stable counting sort of items by expert id.    */
+/* Returns 0, or -(i+1) where i is the first item whose id is outside  */
+/* [0,E) (nothing is written for a rejected input beyond the counts    */
+/* seen so far), or -2^31 for an invalid shape.                        */
+/* Optional outputs (src_expert_count, src_of_row) may be NULL.        */
+/* ------------------------------------------------------------------ */
+int64_t oracle_layout(int32_t R, int32_t T, int32_t K, int32_t E,
+                      const int32_t *ids,           /* [R,T,K] */
+                      int32_t *expert_count,        /* [E]     */
+                      int32_t *expert_offset,       /* [E+1]   */
+                      int32_t *rank_count,          /* [R]     */
+                      int32_t *rank_offset,         /* [R+1]   */
+                      int32_t *src_expert_count,    /* [R,E] or NULL */
+                      int32_t *dst_row,             /* [R,T,K] */
+                      int32_t *src_of_row)          /* [N] or NULL */
+{
+    if (R <= 0 || T < 0 || K <= 0 || E <= 0 || E % R != 0) return INT64_MIN / 2;
+    const int64_t N = (int64_t)R * T * K;
+    const int64_t per_rank = (int64_t)T * K;
+    const int32_t E_loc = E / R;
+
+    /* per-expert counts (and per-(source rank, expert) counts) */
+    for (int32_t e = 0; e < E; ++e) expert_count[e] = 0;
+    if (src_expert_count)
+        for (int64_t j = 0; j < (int64_t)R * E; ++j) src_expert_count[j] = 0;
+    for (int64_t i = 0; i < N; ++i) {
+        const int32_t e = ids[i];
+        if (e < 0 || e >= E) return -(i + 1);
+        expert_count[e] += 1;
+        if (src_expert_count) src_expert_count[(i / per_rank) * E + e] += 1;
+    }
+
+    /* prefix-sum offsets: segment of expert e is rows [offset[e], offset[e+1]) */
+    expert_offset[0] = 0;
+    for (int32_t e = 0; e < E; ++e) expert_offset[e + 1] = expert_offset[e] + expert_count[e];
+
+    /* rows received per destination rank; rank d owns experts [d*E_loc,(d+1)*E_loc) */
+    for (int32_t d = 0; d < R; ++d) {
+        int32_t s = 0;
+        for (int32_t e = d * E_loc; e < (d + 1) * E_loc; ++e) s += expert_count[e];
+        rank_count[d] = s;
+        rank_offset[d] = expert_offset[d * E_loc];
+    }
+    rank_offset[R] = (int32_t)N;
+
+    /* token-local offsets: the j-th item (in increasing i) that chose expert e
+       lands in row offset[e] + j.  Increasing i is lexicographic (r,t,k). */
+    int32_t *seen = (int32_t *)calloc((size_t)E, sizeof(int32_t));
+    if (!seen) return INT64_MIN / 2;
+    for (int64_t i = 0; i < N; ++i) {
+        const int32_t e = ids[i];
+        const int32_t row = expert_offset[e] + seen[e];
+        seen[e] += 1;
+        dst_row[i] = row;
+        if (src_of_row) src_of_row[row] = (int32_t)i;
+    }
+    free(seen);
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
+/* O2: bf16 dispatch = bit copy of the source row into its K rows.     */
+/* ------------------------------------------------------------------ */
+void oracle_dispatch_bf16(int64_t n_tok, int32_t K, int32_t H,
+                          const int32_t *dst_row,   /* [n_tok*K] */
+                          const uint16_t *x,        /* [n_tok,H] */
+                          uint16_t *recv,           /* [N,H]     */
+                          int32_t nthreads)
+{
+    (void)nthreads;
+#pragma omp parallel for num_threads(nthreads > 0 ? nthreads : 1) schedule(static)
+    for (int64_t n = 0; n < n_tok; ++n)
+        for (int32_t k = 0; k < K; ++k) {
+            const int64_t row = dst_row[n * K + k];
+            memcpy(recv + (size_t)row * H, x + (size_t)n * H, (size_t)H * 2);
+        }
+}
+
+/* ------------------------------------------------------------------ */
+/* OCP 8-bit float e4m3 ("fn": bias 7, 3 mantissa bits, no infinity,   */
+/* NaN = S.1111.111, largest finite 448 = S.1111.110), encoder from    */
+/* binary32 with round-to-nearest, ties to even, saturating to +-448.  */
+/* Pure integer arithmetic on the binary32 bit pattern.                */
+/* ------------------------------------------------------------------ */
+uint8_t oracle_e4m3_encode(float v)
+{
+    uint32_t u;
+    memcpy(&u, &v, 4);
+    const uint8_t sign = (uint8_t)((u >> 24) & 0x80);
+    const uint32_t a = u & 0x7FFFFFFFu;              /* |v| bits */
+    if (a > 0x7F800000u) return (uint8_t)(sign | 0x7F);   /* NaN in -> NaN out */
+    if (a == 0x7F800000u) return (uint8_t)(sign | 0x7E);  /* inf saturates */
+    const int32_t e32 = (int32_t)(a >> 23);          /* biased binary32 exponent */
+    const uint32_t m32 = a & 0x7FFFFFu;
+
+    /* Express |v| = sig * 2^(q) with sig a 24-bit integer (hidden bit set for
+       normals), then count in units of the target's step. */
+    uint32_t sig;
+    int32_t  q;                                      /* |v| = sig * 2^q */
+    if (e32 == 0) { sig = m32;            q = -126 - 23; }
+    else          { sig = m32 | 0x800000; q = e32 - 127 - 23; }
+    if (sig == 0) return sign;
+
+    /* unbiased exponent of |v| (position of the leading bit) */
+    int32_t lead = 23;
+    while (!(sig >> lead)) --lead;
+    const int32_t ex = lead + q;                     /* floor(log2 |v|) */
+
+    /* step (ulp) of the target at this magnitude: 2^(ex-3) for normals
+       (ex >= -6), 2^-9 in the subnormal range */
+    const int32_t step_exp = (ex >= -6) ? ex - 3 : -9;
+    /* steps = |v| / 2^step_exp, rounded to nearest even */
+    const int32_t sh = step_exp - q;                 /* shift right by sh bits */
+    uint64_t steps;
+    if (sh <= 0) {
+        steps = (uint64_t)sig << (-sh);
+    } else if (sh > 40) {
+        steps = 0;                                   /* far below half the smallest step */
+    } else {
+        const uint64_t s64 = sig;
+        const uint64_t fl = s64 >> sh;
+        const uint64_t rem = s64 & ((1ull << sh) - 1);
+        const uint64_t half = 1ull << (sh - 1);
+        steps = fl;
+        if (rem > half || (rem == half && (fl & 1))) steps += 1;
+    }
+
+    /* assemble: value = steps * 2^step_exp */
+    uint32_t code;
+    if (ex < -6) {
+        /* subnormal range: steps in [0,8]; 8 is exactly the smallest normal */
+        code = (uint32_t)steps;                      /* 8 -> exponent field 1, mantissa 0 */
+    } else {
+        /* normal: steps in [8,16]; 16 carries into the next binade */
+        int32_t be = ex + 7;                         /* biased target exponent */
+        uint32_t mant;
+        if (steps == 16) { be += 1; mant = 0; }
+        else             { mant = (uint32_t)steps - 8; }
+        if (be > 15) return (uint8_t)(sign | 0x7E);
+        code = ((uint32_t)be << 3) | mant;
+    }
+    if (code > 0x7E) code = 0x7E;                    /* 0x7F is NaN: saturate to 448 */
+    return (uint8_t)(sign | code);
+}
+
+/* ------------------------------------------------------------------ */
+/* O3: FP8 dispatch.  Per token and per block of 128 columns:          */
+/*   amax  = max |x|            (exact in binary32)                    */
+/*   scale = amax / 448         (one binary32 division, RNE)           */
+/*   q[c]  = e4m3(x[c] / d),  d = scale, or 1 for an all-zero block    */
+/* The stored scale is amax/448 (0 for an all-zero block).  Codes and  */
+/* scales are written to each of the token's K destination rows.       */
+/* ------------------------------------------------------------------ */
+static inline float bf16_to_f32(uint16_t b)
+{
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+void oracle_dispatch_fp8(int64_t n_tok, int32_t K, int32_t H,
+                         const int32_t *dst_row,    /* [n_tok*K]   */
+                         const uint16_t *x,         /* [n_tok,H]   */
+                         uint8_t *recv_q,           /* [N,H]       */
+                         float *recv_scale,         /* [N,H/128]   */
+                         int32_t nthreads)
+{
+    (void)nthreads;
+    const int32_t nb = H / 128;
+#pragma omp parallel for num_threads(nthreads > 0 ? nthreads : 1) schedule(static)
+    for (int64_t n = 0; n < n_tok; ++n) {
+        uint8_t *q = (uint8_t *)malloc((size_t)H);
+        float *sc = (float *)malloc((size_t)nb * sizeof(float));
+        const uint16_t *xr = x + (size_t)n * H;
+        for (int32_t b = 0; b < nb; ++b) {
+            float amax = 0.0f;
+            for (int32_t c = 0; c < 128; ++c) {
+                const float a = fabsf(bf16_to_f32(xr[b * 128 + c]));
+                if (a > amax) amax = a;
+            }
+            const float scale = amax / 448.0f;
+            const float d = (amax == 0.0f) ? 1.0f : scale;
+            for (int32_t c = 0; c < 128; ++c) {
+                const float quo = bf16_to_f32(xr[b * 128 + c]) / d;
+                q[b * 128 + c] = oracle_e4m3_encode(quo);
+            }
+            sc[b] = scale;
+        }
+        for (int32_t k = 0; k < K; ++k) {
+            const int64_t row = dst_row[n * K + k];
+            memcpy(recv_q + (size_t)row * H, q, (size_t)H);
+            memcpy(recv_scale + (size_t)row * nb, sc, (size_t)nb * sizeof(float));
+        }
+        free(q);
+        free(sc);
+    }
+}
+
+/* ------------------------------------------------------------------ */
+/* O4: combine.  out[n,c] = bf16( sum_k w[n,k] * y[dst_row[n,k], c] )  */
+/* accumulated in binary32 with one fused multiply-add per slot, in    */
+/* slot order 0..K-1 starting from +0, then rounded to bf16 (RNE).     */
+/* ------------------------------------------------------------------ */
+static inline uint16_t f32_to_bf16_rne(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((u >> 16) | 0x0040); /* quiet NaN */
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+void oracle_combine(int64_t n_tok, int32_t K, int32_t H,
+                    const int32_t *dst_row,         /* [n_tok*K] */
+                    const uint16_t *y,              /* [N,H]     */
+                    const float *w,                 /* [n_tok,K] */
+                    uint16_t *out,                  /* [n_tok,H] */
+                    int32_t nthreads)
+{
+    (void)nthreads;
+#pragma omp parallel for num_threads(nthreads > 0 ? nthreads : 1) schedule(static)
+    for (int64_t n = 0; n < n_tok; ++n)
+        for (int32_t c = 0; c < H; ++c) {
+            float acc = 0.0f;
+            for (int32_t k = 0; k < K; ++k) {
+                const int64_t row = dst_row[n * K + k];
+                acc = fmaf(w[n * K + k], bf16_to_f32(y[(size_t)row * H + c]), acc);
+            }
+            out[(size_t)n * H + c] = f32_to_bf16_rne(acc);
+        }
+}
+
+int32_t oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

@@ -1,0 +1,149 @@
+"""Pins for the oracle's routing layout (paper App. C, token placement).
+
+None of these retype the oracle's counting sort: they use a comparison sort of
+(expert, rank, token, slot) tuples, a hand-worked example, closed forms and
+structural invariants.
+"""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def brute_force_layout(ids: np.ndarray, E: int):
+    """Independent formulation: sort item tuples lexicographically; row = position."""
+    R, T, K = ids.shape
+    tuples = [(int(ids[r, t, k]), r, t, k) for r in range(R) for t in range(T) for k in range(K)]
+    order = sorted(tuples)
+    dst = np.empty((R, T, K), np.int32)
+    for pos, (e, r, t, k) in enumerate(order):
+        dst[r, t, k] = pos
+    cnt = np.zeros(E, np.int32)
+    src_cnt = np.zeros((R, E), np.int32)
+    for e, r, _, _ in tuples:
+        cnt[e] += 1
+        src_cnt[r, e] += 1
+    return dst, cnt, src_cnt
+
+
+def check_invariants(ids, E, lay):
+    R, T, K = ids.shape
+    N = R * T * K
+    e_loc = E // R
+    assert lay["expert_count"].sum() == N                     # counts sum to R*T*K
+    assert lay["expert_offset"][0] == 0 and lay["expert_offset"][E] == N
+    assert np.all(np.diff(lay["expert_offset"]) == lay["expert_count"])
+    assert np.array_equal(np.sort(lay["dst_row"].ravel()), np.arange(N))   # bijection
+    assert np.array_equal(lay["rank_offset"][:R], lay["expert_offset"][0:E:e_loc])
+    assert lay["rank_offset"][R] == N
+    assert np.array_equal(np.diff(lay["rank_offset"]), lay["rank_count"])
+    assert np.array_equal(lay["src_expert_count"].sum(axis=0), lay["expert_count"])
+    assert np.all(lay["src_expert_count"].sum(axis=1) == T * K)
+    src = lay["src_of_row"]
+    assert np.array_equal(lay["dst_row"].ravel()[src], np.arange(N))       # inverse map
+    flat = ids.ravel()
+    # row lies inside its expert's segment
+    d = lay["dst_row"].ravel()
+    assert np.all(d >= lay["expert_offset"][flat]) and np.all(d < lay["expert_offset"][flat + 1])
+    # inside a segment the source item index (= (r,t,k) lexicographic) strictly increases
+    for e in range(E):
+        seg = src[lay["expert_offset"][e]:lay["expert_offset"][e + 1]]
+        assert np.all(flat[seg] == e)
+        assert np.all(np.diff(seg) > 0)
+
+
+def test_worked_example():
+    rows = {}
+    with open(os.path.join(GOLDEN, "layout_worked_example.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].split()
+            if line:
+                rows[line[0]] = np.array(line[1:], dtype=np.int64)
+    R, T, K, E = rows["shape"]
+    lay = oracle.layout(rows["ids"].astype(np.int32).reshape(R, T, K), int(E))
+    for key in ("expert_count", "expert_offset", "rank_count", "rank_offset",
+                "src_expert_count", "dst_row", "src_of_row"):
+        assert np.array_equal(lay[key].ravel(), rows[key]), key
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_matches_sort_brute_force(seed):
+    rng = np.random.default_rng(seed)
+    R = int(rng.choice([1, 2, 3, 4]))
+    e_loc = int(rng.integers(1, 5))
+    E = R * e_loc
+    T = int(rng.integers(0, 40))
+    K = int(rng.integers(1, 5))
+    # duplicates inside a token are legal; some experts stay empty
+    ids = rng.integers(0, max(1, E - (seed % 2)), size=(R, T, K)).astype(np.int32)
+    lay = oracle.layout(ids, E)
+    dst, cnt, src_cnt = brute_force_layout(ids, E)
+    assert np.array_equal(lay["dst_row"], dst)
+    assert np.array_equal(lay["expert_count"], cnt)
+    assert np.array_equal(lay["src_expert_count"], src_cnt)
+    check_invariants(ids, E, lay)
+
+
+def test_all_to_one_expert_and_k1_and_r1():
+    ids = np.full((3, 7, 2), 4, np.int32)
+    lay = oracle.layout(ids, 6)
+    assert np.array_equal(lay["dst_row"].ravel(), np.arange(42))
+    assert lay["expert_count"].tolist() == [0, 0, 0, 0, 42, 0]
+    assert lay["rank_count"].tolist() == [0, 0, 42]
+    ids = np.arange(10, dtype=np.int32).reshape(1, 10, 1) % 3
+    lay = oracle.layout(ids, 3)
+    dst, _, _ = brute_force_layout(ids, 3)
+    assert np.array_equal(lay["dst_row"], dst)
+
+
+def test_closed_form_single_expert():
+    ids = np.zeros((2, 5, 3), np.int32)
+    lay = oracle.layout(ids, 2)          # E=2, only expert 0 used
+    assert np.array_equal(lay["dst_row"].ravel(), np.arange(30))
+    lay = oracle.layout(np.zeros((1, 5, 3), np.int32), 1)   # E = 1
+    assert np.array_equal(lay["dst_row"].ravel(), np.arange(15))
+
+
+def test_closed_form_round_robin():
+    # ids[i] = i mod E with K = E: expert e receives item e of every token, in token order
+    R, T, E = 4, 6, 8
+    K = E
+    n_tok = R * T
+    ids = (np.arange(R * T * K) % E).astype(np.int32).reshape(R, T, K)
+    lay = oracle.layout(ids, E)
+    i = np.arange(R * T * K)
+    assert np.array_equal(lay["dst_row"].ravel(), (i % E) * n_tok + i // E)
+    assert np.all(lay["expert_count"] == n_tok)
+
+
+def test_empty_batch():
+    lay = oracle.layout(np.zeros((2, 0, 2), np.int32), 4)
+    assert lay["expert_offset"].tolist() == [0, 0, 0, 0, 0]
+    assert lay["rank_count"].tolist() == [0, 0]
+
+
+def test_bad_expert_id_is_rejected():
+    ids = np.zeros((2, 3, 2), np.int32)
+    ids[1, 0, 1] = 4
+    with pytest.raises(oracle.BadExpertId) as ei:
+        oracle.layout(ids, 4)
+    assert ei.value.item == 7
+    ids[1, 0, 1] = -1
+    with pytest.raises(oracle.BadExpertId):
+        oracle.layout(ids, 4)
+    with pytest.raises(ValueError):
+        oracle.layout(np.zeros((3, 2, 1), np.int32), 4)    # E % R != 0
+
+
+def test_invariants_on_tiny_config():
+    from paper_2607_26444_b200 import workloads as wl
+    cfg = wl.CONFIGS["tiny"]
+    ids = wl.gen_topk_ids(cfg)
+    lay = oracle.layout(ids, cfg.E)
+    check_invariants(ids, cfg.E, lay)
+    dst, cnt, _ = brute_force_layout(ids, cfg.E)
+    assert np.array_equal(lay["dst_row"], dst)
