@@ -1,0 +1,184 @@
+/*
+ * strata_moe.h -- C ABI of the B200 (sm_100a) MoE routing-layout / token-dispatch /
+ * gate-weighted-combine library.
+ *
+ * Conventions for every function
+ *  - Returns a strata_status.  Nothing throws, traps, asserts or aborts.
+ *  - "device pointer" = address in the memory of the context's GPU; "host
+ *    pointer" = ordinary process memory.  All data buffers belong to the
+ *    caller; the library owns only the opaque host-side strata_ctx and never
+ *    allocates or frees device memory.
+ *  - The three moe calls enqueue kernels on the given CUDA stream
+ *    (a cudaStream_t passed as void*; NULL = the legacy default stream) and
+ *    return without synchronising.  Errors that can be seen on the host
+ *    (NULL pointer, shape, alignment, unregistered receive buffer, capacity)
+ *    are returned before anything is launched.  Errors that only the device
+ *    can see (an expert id outside [0,E), a destination row outside the
+ *    receive buffer, a bounded wait that ran out) set a device status word
+ *    (first error wins), the offending item is skipped, nothing is accessed
+ *    out of bounds, and the error is reported by strata_device_status().
+ *  - Index convention: rank r in [0,R), token t in [0,T), slot k in [0,K);
+ *    flat item i = (r*T + t)*K + k; token n = r*T + t; N = R*T*K.
+ *    Expert e belongs to rank e / (E/R).  All R ranks are partitions of one
+ *    GPU's memory.
+ *  - bf16 tensors are row-major arrays of 16-bit patterns.
+ */
+#ifndef STRATA_MOE_H
+#define STRATA_MOE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    STRATA_OK = 0,
+    STRATA_ERR_INVALID_ARG = 1,    /* NULL or otherwise unusable argument            */
+    STRATA_ERR_SHAPE = 2,          /* shape outside what the kernels support          */
+    STRATA_ERR_ALIGNMENT = 3,      /* a data pointer is not 16-byte aligned           */
+    STRATA_ERR_NOT_REGISTERED = 4, /* receive buffer not inside a registered region   */
+    STRATA_ERR_CAPACITY = 5,       /* receive buffer / region / workspace too small   */
+    STRATA_ERR_BAD_EXPERT_ID = 6,  /* device: an id outside [0,E) was skipped         */
+    STRATA_ERR_WORKSPACE = 7,      /* no workspace set on the context                 */
+    STRATA_ERR_CUDA = 8,           /* a CUDA runtime call failed                      */
+    STRATA_ERR_TIMEOUT = 9,        /* device: a bounded wait ran out                  */
+    STRATA_ERR_BAD_ROW = 10        /* device: a destination row outside the buffer    */
+} strata_status;
+
+typedef enum {
+    STRATA_BF16 = 0,               /* dispatch copies bf16 rows bit for bit           */
+    STRATA_FP8_E4M3_B128 = 1       /* dispatch quantises to e4m3, one fp32 scale per
+                                      token per block of 128 columns                  */
+} strata_dtype;
+
+/* Problem shape.  Requirements: R,T,H,E,K > 0; E % R == 0; E <= 1024; K <= 32;
+ * H % 8 == 0 (rows are whole 16-byte vectors); H % 128 == 0 for FP8;
+ * R*T*K < 2^31. */
+typedef struct {
+    int32_t R, T, H, E, K;
+    int32_t dispatch_dtype;        /* a strata_dtype */
+} strata_moe_shape;
+
+typedef struct strata_ctx strata_ctx;   /* opaque, host side */
+
+/* Routing metadata (paper App. C, "token placement": destination expert,
+ * per-expert counts, prefix-sum offsets, token-local offsets), produced by
+ * strata_moe_layout and consumed by dispatch and combine.  All members are
+ * device pointers to int32 arrays owned by the caller. */
+typedef struct {
+    int32_t *expert_count;      /* [E]    items routed to expert e                       */
+    int32_t *expert_offset;     /* [E+1]  exclusive scan; segment e = rows [off[e],off[e+1]) */
+    int32_t *rank_count;        /* [R]    rows received by rank d                        */
+    int32_t *rank_offset;       /* [R+1]  rank d's partition = rows [off[d],off[d+1])    */
+    int32_t *src_expert_count;  /* [R,E]  items of source rank r routed to e; may be NULL */
+    int32_t *dst_row;           /* [R,T,K] receive row of item i (-1 for a skipped item) */
+    int32_t *src_of_row;        /* [N]    inverse of dst_row; may be NULL                */
+} strata_moe_layout_t;
+
+const char *strata_status_string(strata_status s);
+
+/* ---- context ------------------------------------------------------------ */
+
+/* Creates a context for one shape on CUDA device `device` (made current for the
+ * duration of each call).  Host errors: INVALID_ARG, SHAPE, CUDA.
+ * device = -1 creates a host-only context: the pool and all argument validation
+ * work as usual (pointers are recorded, never dereferenced), and every call that
+ * would launch or touch device memory returns STRATA_ERR_CUDA instead.  It
+ * computes nothing; it exists so that host logic can be exercised without a GPU. */
+strata_status strata_ctx_create(strata_ctx **out, const strata_moe_shape *shape, int device);
+strata_status strata_ctx_destroy(strata_ctx *ctx);
+
+/* Scratch memory the layout kernels need for this shape (per-tile histograms,
+ * a ticket and the device status word).  The caller allocates at least `bytes`
+ * bytes of device memory, 256-byte aligned, and hands it over with
+ * strata_ctx_set_workspace, which zeroes it (synchronously).  It must stay
+ * valid and unshared while calls on this context are in flight. */
+strata_status strata_moe_workspace_bytes(const strata_moe_shape *shape, size_t *bytes);
+strata_status strata_ctx_set_workspace(strata_ctx *ctx, void *dptr, size_t bytes);
+
+/* Number of kernels this context has launched so far (for accounting). */
+strata_status strata_ctx_launch_count(strata_ctx *ctx, uint64_t *count);
+
+/* ---- pool: registration at allocation time ------------------------------
+ * Analogue of the paper's registration-on-allocation (Sec. 5.1): a buffer is
+ * registered once, when it is allocated (phase 1); every later operator call
+ * only performs a cheap local readiness check (phase 2).  Here the caller
+ * allocates (e.g. a torch tensor), the library records [base, base+bytes) and
+ * can sub-allocate from it, so the receive buffer handed to dispatch is the
+ * very tensor the expert GEMM reads: no staging copy exists (Sec. 2.2 / 7.1
+ * describe the staging copies this removes).  Rank partitions are disjoint
+ * sub-ranges of one address space (Sec. 5.2). */
+strata_status strata_pool_register(strata_ctx *ctx, void *dbase, size_t bytes, uint64_t *region_id);
+/* OK iff [dptr, dptr+bytes) lies inside one registered region; pure host lookup. */
+strata_status strata_pool_is_ready(strata_ctx *ctx, const void *dptr, size_t bytes);
+strata_status strata_pool_unregister(strata_ctx *ctx, uint64_t region_id);
+/* Bump sub-allocation inside a region (align: power of two, >= 1).  CAPACITY if it does not fit. */
+strata_status strata_pool_carve(strata_ctx *ctx, uint64_t region_id, size_t bytes, size_t align, void **dptr);
+strata_status strata_pool_reset(strata_ctx *ctx, uint64_t region_id);
+
+/* ---- the hot path --------------------------------------------------------- */
+
+/* Routing layout (paper App. C, level 1).  topk_ids: device int32 [R,T,K].
+ * Computes a stable counting sort of the items by expert id: dst_row[i] =
+ * expert_offset[e_i] + #{j < i : e_j = e_i}, i.e. segments ordered by expert,
+ * then source rank, then token, then slot, packed without padding.
+ * Duplicate ids inside a token are legal.  An id outside [0,E) is skipped
+ * (dst_row = -1, not counted) and raises BAD_EXPERT_ID on the device status.
+ * Needs a workspace.  Two kernel launches. */
+strata_status strata_moe_layout(strata_ctx *ctx, const int32_t *topk_ids,
+                                const strata_moe_layout_t *layout, void *stream);
+
+/* Dispatch (paper Sec. 6.2 / 7.1).  x: device bf16 [R,T,H].
+ * BF16:  recv is device bf16 [capacity_rows, H]; recv[dst_row[i], :] = x[n(i), :] bit for bit;
+ *        recv_scale must be NULL.
+ * FP8:   recv is device uint8 [capacity_rows, H], recv_scale device float [capacity_rows, H/128];
+ *        per token and block of 128 columns: amax = max|x|, scale = amax/448 (IEEE binary32
+ *        division), q = e4m3_rne_satfinite(x / (amax == 0 ? 1 : scale)); codes and the stored
+ *        scale (amax/448) go to each of the token's K rows.
+ * recv (and recv_scale) must lie inside a registered region (NOT_REGISTERED otherwise), be
+ * 16-byte aligned, and capacity_rows >= N (CAPACITY otherwise).  Rows whose dst_row is outside
+ * [0, capacity_rows) are skipped and raise BAD_ROW.  One kernel launch. */
+strata_status strata_moe_dispatch(strata_ctx *ctx, const strata_moe_layout_t *layout, const void *x,
+                                  void *recv, float *recv_scale, size_t capacity_rows, void *stream);
+
+/* Combine (paper Sec. 6.1, reduction-bearing operators).  y: device bf16 [y_rows, H] (expert
+ * outputs, row j answers receive row j; may be the receive buffer itself), topk_w: device
+ * float [R,T,K], out: device bf16 [R,T,H].
+ * out[n,c] = bf16_rne( fma(w[n,K-1], y[dst_row[n,K-1],c], ... fma(w[n,0], y[dst_row[n,0],c], +0)) ):
+ * binary32 fused multiply-add chain in slot order, one rounding to bf16.  Slots whose dst_row is
+ * outside [0, y_rows) contribute nothing and raise BAD_ROW.  One kernel launch. */
+strata_status strata_moe_combine(strata_ctx *ctx, const strata_moe_layout_t *layout, const void *y,
+                                 size_t y_rows, const float *topk_w, void *out, void *stream);
+
+/* Host helper: rank d's partition of the receive buffer, from a HOST copy of rank_offset[R+1]:
+ * *rank_base = recv + rank_offset[d] * row_bytes, *rows = rank_offset[d+1] - rank_offset[d]. */
+strata_status strata_moe_recv_view(strata_ctx *ctx, const int32_t *h_rank_offset, int rank,
+                                   void *recv, void **rank_base, int64_t *rows);
+
+/* Synchronises the stream, reads the device status word into *out and clears it. */
+strata_status strata_device_status(strata_ctx *ctx, void *stream, strata_status *out);
+
+/* Whole path from HOST buffers with identity experts (BF16 contexts only): copies ids, x and
+ * gate weights to the device buffers given in `dev`, runs layout -> dispatch -> combine with
+ * y = recv, copies out back and synchronises the stream.  h_* are host pointers (pinned memory
+ * makes the copies asynchronous); every member of `dev` is a device pointer owned by the caller,
+ * dev->recv inside a registered region with room for N rows.  Used for end-to-end timing and
+ * smoke checks; the paper has no counterpart (its operators take device buffers). */
+typedef struct {
+    int32_t *ids;       /* [R,T,K] */
+    void *x;            /* bf16 [R,T,H] */
+    float *w;           /* [R,T,K] */
+    void *recv;         /* bf16 [N,H] */
+    void *out;          /* bf16 [R,T,H] */
+    strata_moe_layout_t layout;
+} strata_moe_device_buffers;
+strata_status strata_moe_roundtrip_host(strata_ctx *ctx, const strata_moe_device_buffers *dev,
+                                        const int32_t *h_ids, const void *h_x, const float *h_w,
+                                        void *h_out, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STRATA_MOE_H */

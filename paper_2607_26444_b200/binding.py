@@ -1,0 +1,312 @@
+"""ctypes binding of the C-ABI library: argument marshalling only.
+
+Every function named ``strata_*`` forwards to the C entry point of the same
+name (see ``include/strata_moe.h``).  ``MoEContext`` is a small convenience
+wrapper that uses torch for device memory and streams; it performs no
+arithmetic of its own.  There is no CPU fallback: if the CUDA library has not
+been built, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libstrata_moe.so")
+
+STRATA_OK = 0
+STRATA_ERR_INVALID_ARG = 1
+STRATA_ERR_SHAPE = 2
+STRATA_ERR_ALIGNMENT = 3
+STRATA_ERR_NOT_REGISTERED = 4
+STRATA_ERR_CAPACITY = 5
+STRATA_ERR_BAD_EXPERT_ID = 6
+STRATA_ERR_WORKSPACE = 7
+STRATA_ERR_CUDA = 8
+STRATA_ERR_TIMEOUT = 9
+STRATA_ERR_BAD_ROW = 10
+
+STRATA_BF16 = 0
+STRATA_FP8_E4M3_B128 = 1
+
+EXPORTS = [
+    "strata_status_string", "strata_ctx_create", "strata_ctx_destroy", "strata_moe_workspace_bytes",
+    "strata_ctx_set_workspace", "strata_ctx_launch_count", "strata_pool_register", "strata_pool_is_ready",
+    "strata_pool_unregister", "strata_pool_carve", "strata_pool_reset", "strata_moe_layout",
+    "strata_moe_dispatch", "strata_moe_combine", "strata_moe_recv_view", "strata_device_status",
+    "strata_moe_roundtrip_host",
+]
+
+
+class strata_moe_shape(ctypes.Structure):
+    _fields_ = [("R", ctypes.c_int32), ("T", ctypes.c_int32), ("H", ctypes.c_int32),
+                ("E", ctypes.c_int32), ("K", ctypes.c_int32), ("dispatch_dtype", ctypes.c_int32)]
+
+
+class strata_moe_layout_t(ctypes.Structure):
+    _fields_ = [("expert_count", ctypes.c_void_p), ("expert_offset", ctypes.c_void_p),
+                ("rank_count", ctypes.c_void_p), ("rank_offset", ctypes.c_void_p),
+                ("src_expert_count", ctypes.c_void_p), ("dst_row", ctypes.c_void_p),
+                ("src_of_row", ctypes.c_void_p)]
+
+
+class strata_moe_device_buffers(ctypes.Structure):
+    _fields_ = [("ids", ctypes.c_void_p), ("x", ctypes.c_void_p), ("w", ctypes.c_void_p),
+                ("recv", ctypes.c_void_p), ("out", ctypes.c_void_p), ("layout", strata_moe_layout_t)]
+
+
+class StrataError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = int(code)
+        super().__init__(f"{where}: status {self.code} ({strata_status_string(self.code)})")
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library; raises if it has not been built (no fallback)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with "
+                           f"`python -m paper_2607_26444_b200.build` (there is no CPU fallback)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, sz, i32, u64 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint64
+    P = ctypes.POINTER
+    L.strata_status_string.restype = ctypes.c_char_p
+    L.strata_status_string.argtypes = [i32]
+    sigs = {
+        "strata_ctx_create": [P(vp), P(strata_moe_shape), i32],
+        "strata_ctx_destroy": [vp],
+        "strata_moe_workspace_bytes": [P(strata_moe_shape), P(sz)],
+        "strata_ctx_set_workspace": [vp, vp, sz],
+        "strata_ctx_launch_count": [vp, P(u64)],
+        "strata_pool_register": [vp, vp, sz, P(u64)],
+        "strata_pool_is_ready": [vp, vp, sz],
+        "strata_pool_unregister": [vp, u64],
+        "strata_pool_carve": [vp, u64, sz, sz, P(vp)],
+        "strata_pool_reset": [vp, u64],
+        "strata_moe_layout": [vp, vp, P(strata_moe_layout_t), vp],
+        "strata_moe_dispatch": [vp, P(strata_moe_layout_t), vp, vp, vp, sz, vp],
+        "strata_moe_combine": [vp, P(strata_moe_layout_t), vp, sz, vp, vp, vp],
+        "strata_moe_recv_view": [vp, vp, i32, vp, P(vp), P(ctypes.c_int64)],
+        "strata_device_status": [vp, vp, P(i32)],
+        "strata_moe_roundtrip_host": [vp, P(strata_moe_device_buffers), vp, vp, vp, vp, vp],
+    }
+    for name, args in sigs.items():
+        fn = getattr(L, name)
+        fn.restype = i32
+        fn.argtypes = args
+    _lib = L
+    return L
+
+
+# ---- one Python function per C entry point (same names, raw pointers) -------
+
+def strata_status_string(code: int) -> str:
+    return lib().strata_status_string(int(code)).decode()
+
+
+def strata_ctx_create(shape: strata_moe_shape, device: int) -> Tuple[int, Optional[int]]:
+    h = ctypes.c_void_p()
+    rc = lib().strata_ctx_create(ctypes.byref(h), ctypes.byref(shape), device)
+    return rc, h.value
+
+
+def strata_ctx_destroy(ctx) -> int:
+    return lib().strata_ctx_destroy(ctx)
+
+
+def strata_moe_workspace_bytes(shape: strata_moe_shape) -> Tuple[int, int]:
+    n = ctypes.c_size_t()
+    rc = lib().strata_moe_workspace_bytes(ctypes.byref(shape), ctypes.byref(n))
+    return rc, n.value
+
+
+def strata_ctx_set_workspace(ctx, dptr: int, nbytes: int) -> int:
+    return lib().strata_ctx_set_workspace(ctx, dptr, nbytes)
+
+
+def strata_ctx_launch_count(ctx) -> Tuple[int, int]:
+    n = ctypes.c_uint64()
+    rc = lib().strata_ctx_launch_count(ctx, ctypes.byref(n))
+    return rc, n.value
+
+
+def strata_pool_register(ctx, dbase: int, nbytes: int) -> Tuple[int, int]:
+    rid = ctypes.c_uint64()
+    rc = lib().strata_pool_register(ctx, dbase, nbytes, ctypes.byref(rid))
+    return rc, rid.value
+
+
+def strata_pool_is_ready(ctx, dptr: int, nbytes: int) -> int:
+    return lib().strata_pool_is_ready(ctx, dptr, nbytes)
+
+
+def strata_pool_unregister(ctx, region_id: int) -> int:
+    return lib().strata_pool_unregister(ctx, region_id)
+
+
+def strata_pool_carve(ctx, region_id: int, nbytes: int, align: int) -> Tuple[int, Optional[int]]:
+    p = ctypes.c_void_p()
+    rc = lib().strata_pool_carve(ctx, region_id, nbytes, align, ctypes.byref(p))
+    return rc, p.value
+
+
+def strata_pool_reset(ctx, region_id: int) -> int:
+    return lib().strata_pool_reset(ctx, region_id)
+
+
+def strata_moe_layout(ctx, topk_ids: int, layout: strata_moe_layout_t, stream: int) -> int:
+    return lib().strata_moe_layout(ctx, topk_ids, ctypes.byref(layout), stream)
+
+
+def strata_moe_dispatch(ctx, layout: strata_moe_layout_t, x: int, recv: int, recv_scale: Optional[int],
+                        capacity_rows: int, stream: int) -> int:
+    return lib().strata_moe_dispatch(ctx, ctypes.byref(layout), x, recv, recv_scale, capacity_rows, stream)
+
+
+def strata_moe_combine(ctx, layout: strata_moe_layout_t, y: int, y_rows: int, topk_w: int, out: int,
+                       stream: int) -> int:
+    return lib().strata_moe_combine(ctx, ctypes.byref(layout), y, y_rows, topk_w, out, stream)
+
+
+def strata_moe_recv_view(ctx, h_rank_offset, rank: int, recv: int) -> Tuple[int, Optional[int], int]:
+    """h_rank_offset: a host numpy int32 array [R+1]."""
+    base, rows = ctypes.c_void_p(), ctypes.c_int64()
+    rc = lib().strata_moe_recv_view(ctx, h_rank_offset.ctypes.data, rank, recv, ctypes.byref(base),
+                                    ctypes.byref(rows))
+    return rc, base.value, rows.value
+
+
+def strata_device_status(ctx, stream: int) -> Tuple[int, int]:
+    out = ctypes.c_int()
+    rc = lib().strata_device_status(ctx, stream, ctypes.byref(out))
+    return rc, out.value
+
+
+def strata_moe_roundtrip_host(ctx, dev: strata_moe_device_buffers, h_ids: int, h_x: int, h_w: int, h_out: int,
+                              stream: int) -> int:
+    return lib().strata_moe_roundtrip_host(ctx, ctypes.byref(dev), h_ids, h_x, h_w, h_out, stream)
+
+
+# ---- convenience wrapper over torch tensors (memory + streams only) ---------
+
+def _check(rc: int, where: str) -> None:
+    if rc != STRATA_OK:
+        raise StrataError(rc, where)
+
+
+class Layout:
+    """Device tensors holding the routing metadata, plus the C struct pointing at them."""
+
+    def __init__(self, R: int, T: int, K: int, E: int, device, with_optional: bool = True):
+        import torch
+        i32 = dict(dtype=torch.int32, device=device)
+        self.expert_count = torch.empty(E, **i32)
+        self.expert_offset = torch.empty(E + 1, **i32)
+        self.rank_count = torch.empty(R, **i32)
+        self.rank_offset = torch.empty(R + 1, **i32)
+        self.src_expert_count = torch.empty((R, E), **i32) if with_optional else None
+        self.dst_row = torch.empty((R, T, K), **i32)
+        self.src_of_row = torch.empty(R * T * K, **i32) if with_optional else None
+        self.c = strata_moe_layout_t(
+            self.expert_count.data_ptr(), self.expert_offset.data_ptr(), self.rank_count.data_ptr(),
+            self.rank_offset.data_ptr(),
+            self.src_expert_count.data_ptr() if with_optional else None,
+            self.dst_row.data_ptr(),
+            self.src_of_row.data_ptr() if with_optional else None)
+
+
+class MoEContext:
+    """One shape on one GPU.  Owns a strata_ctx and its workspace tensor."""
+
+    def __init__(self, R: int, T: int, H: int, E: int, K: int, dispatch_dtype: int = STRATA_BF16,
+                 device: int = 0):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("MoEContext needs a CUDA device (there is no CPU fallback)")
+        self.shape = strata_moe_shape(R, T, H, E, K, dispatch_dtype)
+        self.R, self.T, self.H, self.E, self.K = R, T, H, E, K
+        self.fp8 = dispatch_dtype == STRATA_FP8_E4M3_B128
+        self.n_tok, self.n_items = R * T, R * T * K
+        self.device = torch.device("cuda", device)
+        rc, h = strata_ctx_create(self.shape, device)
+        _check(rc, "strata_ctx_create")
+        self.h = h
+        rc, nbytes = strata_moe_workspace_bytes(self.shape)
+        _check(rc, "strata_moe_workspace_bytes")
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        _check(strata_ctx_set_workspace(self.h, self.workspace.data_ptr(), nbytes), "strata_ctx_set_workspace")
+        self._regions = {}
+
+    def close(self) -> None:
+        if getattr(self, "h", None):
+            strata_ctx_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @staticmethod
+    def _stream() -> int:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+
+    # pool -----------------------------------------------------------------
+    def register(self, tensor) -> int:
+        rc, rid = strata_pool_register(self.h, tensor.data_ptr(), tensor.numel() * tensor.element_size())
+        _check(rc, "strata_pool_register")
+        self._regions[rid] = tensor          # keep the allocation alive while registered
+        return rid
+
+    def unregister(self, rid: int) -> None:
+        _check(strata_pool_unregister(self.h, rid), "strata_pool_unregister")
+        self._regions.pop(rid, None)
+
+    def carve(self, rid: int, shape, dtype, align: int = 256):
+        """A tensor view of a sub-range carved from a registered region (zero copy)."""
+        import torch
+        base = self._regions[rid]
+        n = 1
+        for d in shape:
+            n *= int(d)
+        nbytes = n * torch.empty((), dtype=dtype).element_size()
+        rc, p = strata_pool_carve(self.h, rid, nbytes, align)
+        _check(rc, "strata_pool_carve")
+        off = p - base.data_ptr()
+        return base.view(torch.uint8).reshape(-1)[off:off + nbytes].view(dtype).reshape(*shape)
+
+    def new_layout(self, with_optional: bool = True) -> Layout:
+        return Layout(self.R, self.T, self.K, self.E, self.device, with_optional)
+
+    # hot path ---------------------------------------------------------------
+    def layout(self, ids, layout: Optional[Layout] = None) -> Layout:
+        layout = layout or self.new_layout()
+        _check(strata_moe_layout(self.h, ids.data_ptr(), layout.c, self._stream()), "strata_moe_layout")
+        return layout
+
+    def dispatch(self, layout: Layout, x, recv, recv_scale=None) -> None:
+        _check(strata_moe_dispatch(self.h, layout.c, x.data_ptr(), recv.data_ptr(),
+                                   recv_scale.data_ptr() if recv_scale is not None else None,
+                                   recv.shape[0], self._stream()), "strata_moe_dispatch")
+
+    def combine(self, layout: Layout, y, w, out) -> None:
+        _check(strata_moe_combine(self.h, layout.c, y.data_ptr(), y.shape[0], w.data_ptr(), out.data_ptr(),
+                                  self._stream()), "strata_moe_combine")
+
+    def device_status(self) -> int:
+        rc, st = strata_device_status(self.h, self._stream())
+        _check(rc, "strata_device_status")
+        return st
+
+    def launch_count(self) -> int:
+        rc, n = strata_ctx_launch_count(self.h)
+        _check(rc, "strata_ctx_launch_count")
+        return n

@@ -1,0 +1,407 @@
+// C ABI: context, registration pool, argument validation and kernel launches.
+// Host-side only; every device-side step lives in layout.cu / dispatch.cu / combine.cu.
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+namespace strata {
+cudaError_t configure_layout_kernels();
+cudaError_t configure_dispatch_kernels();
+}  // namespace strata
+
+struct strata_region {
+    uint64_t id;
+    uintptr_t base;
+    size_t bytes;
+    size_t used;      // bump pointer of strata_pool_carve
+};
+
+struct strata_ctx {
+    strata_moe_shape shape;
+    int device;
+    int n_sm;
+    int* ws;              // device workspace (header + tile counts)
+    size_t ws_bytes;
+    uint64_t next_region;
+    uint64_t launches;
+    std::vector<strata_region> regions;
+    std::mutex mu;
+};
+
+namespace {
+
+using namespace strata;
+
+strata_status check_shape(const strata_moe_shape* s)
+{
+    if (!s) return STRATA_ERR_INVALID_ARG;
+    if (s->R <= 0 || s->T <= 0 || s->H <= 0 || s->E <= 0 || s->K <= 0) return STRATA_ERR_SHAPE;
+    if (s->E % s->R != 0 || s->E > kMaxExperts || s->K > kMaxTopK) return STRATA_ERR_SHAPE;
+    if (s->H % 8 != 0) return STRATA_ERR_SHAPE;
+    if (s->dispatch_dtype != STRATA_BF16 && s->dispatch_dtype != STRATA_FP8_E4M3_B128) return STRATA_ERR_SHAPE;
+    if (s->dispatch_dtype == STRATA_FP8_E4M3_B128 && s->H % 128 != 0) return STRATA_ERR_SHAPE;
+    const long long n = (long long)s->R * s->T * s->K;
+    if (n >= (1ll << 31)) return STRATA_ERR_SHAPE;
+    return STRATA_OK;
+}
+
+size_t workspace_bytes(const strata_moe_shape& s)
+{
+    const LayoutGeom g = layout_geom(s);
+    size_t b = (size_t)kWsHeaderBytes + (size_t)g.n_tiles * s.E * sizeof(int);
+    return (b + 255) & ~(size_t)255;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        if (prev == dev) prev = -1;
+    }
+    ~DeviceGuard()
+    {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+bool region_contains(const strata_ctx* c, const void* p, size_t bytes)
+{
+    const uintptr_t a = reinterpret_cast<uintptr_t>(p);
+    for (const strata_region& r : c->regions)
+        if (a >= r.base && bytes <= r.bytes && a - r.base <= r.bytes - bytes) return true;
+    return false;
+}
+
+strata_status check_layout_ptrs(const strata_moe_layout_t* L, bool need_all)
+{
+    if (!L || !L->dst_row) return STRATA_ERR_INVALID_ARG;
+    if (need_all && (!L->expert_count || !L->expert_offset || !L->rank_count || !L->rank_offset))
+        return STRATA_ERR_INVALID_ARG;
+    return STRATA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* strata_status_string(strata_status s)
+{
+    switch (s) {
+        case STRATA_OK: return "ok";
+        case STRATA_ERR_INVALID_ARG: return "invalid argument";
+        case STRATA_ERR_SHAPE: return "unsupported shape";
+        case STRATA_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+        case STRATA_ERR_NOT_REGISTERED: return "buffer not inside a registered region";
+        case STRATA_ERR_CAPACITY: return "capacity too small";
+        case STRATA_ERR_BAD_EXPERT_ID: return "expert id out of range (item skipped)";
+        case STRATA_ERR_WORKSPACE: return "no workspace set";
+        case STRATA_ERR_CUDA: return "CUDA runtime error";
+        case STRATA_ERR_TIMEOUT: return "bounded device wait ran out";
+        case STRATA_ERR_BAD_ROW: return "destination row out of range (row skipped)";
+    }
+    return "unknown status";
+}
+
+strata_status strata_ctx_create(strata_ctx** out, const strata_moe_shape* shape, int device)
+{
+    if (!out) return STRATA_ERR_INVALID_ARG;
+    *out = nullptr;
+    strata_status st = check_shape(shape);
+    if (st != STRATA_OK) return st;
+    int n_sm = 0;
+    if (device != -1) {
+        int n_dev = 0;
+        if (cudaGetDeviceCount(&n_dev) != cudaSuccess) {
+            cudaGetLastError();
+            return STRATA_ERR_CUDA;
+        }
+        if (device < 0 || device >= n_dev) return STRATA_ERR_INVALID_ARG;
+        DeviceGuard g(device);
+        if (!g.ok) return STRATA_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+            return STRATA_ERR_CUDA;
+        if (configure_layout_kernels() != cudaSuccess || configure_dispatch_kernels() != cudaSuccess) {
+            cudaGetLastError();
+            return STRATA_ERR_CUDA;
+        }
+    }
+    strata_ctx* c = new (std::nothrow) strata_ctx();
+    if (!c) return STRATA_ERR_INVALID_ARG;
+    c->shape = *shape;
+    c->device = device;
+    c->n_sm = n_sm;
+    c->ws = nullptr;
+    c->ws_bytes = 0;
+    c->next_region = 1;
+    c->launches = 0;
+    *out = c;
+    return STRATA_OK;
+}
+
+strata_status strata_ctx_destroy(strata_ctx* ctx)
+{
+    if (!ctx) return STRATA_ERR_INVALID_ARG;
+    delete ctx;
+    return STRATA_OK;
+}
+
+strata_status strata_moe_workspace_bytes(const strata_moe_shape* shape, size_t* bytes)
+{
+    if (!bytes) return STRATA_ERR_INVALID_ARG;
+    strata_status st = check_shape(shape);
+    if (st != STRATA_OK) return st;
+    *bytes = workspace_bytes(*shape);
+    return STRATA_OK;
+}
+
+strata_status strata_ctx_set_workspace(strata_ctx* ctx, void* dptr, size_t bytes)
+{
+    if (!ctx || !dptr) return STRATA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(dptr) & 255u) != 0) return STRATA_ERR_ALIGNMENT;
+    if (bytes < workspace_bytes(ctx->shape)) return STRATA_ERR_CAPACITY;
+    if (ctx->device < 0) {               // host-only context: record, never touch
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        ctx->ws = static_cast<int*>(dptr);
+        ctx->ws_bytes = bytes;
+        return STRATA_OK;
+    }
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return STRATA_ERR_CUDA;
+    if (cudaMemset(dptr, 0, workspace_bytes(ctx->shape)) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+        cudaGetLastError();
+        return STRATA_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lk(ctx->mu);
+    ctx->ws = static_cast<int*>(dptr);
+    ctx->ws_bytes = bytes;
+    return STRATA_OK;
+}
+
+strata_status strata_ctx_launch_count(strata_ctx* ctx, uint64_t* count)
+{
+    if (!ctx || !count) return STRATA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(ctx->mu);
+    *count = ctx->launches;
+    return STRATA_OK;
+}
+
+// ---- pool -------------------------------------------------------------------------
+
+strata_status strata_pool_register(strata_ctx* ctx, void* dbase, size_t bytes, uint64_t* region_id)
+{
+    if (!ctx || !dbase || !region_id || bytes == 0) return STRATA_ERR_INVALID_ARG;
+    if (!aligned16(dbase)) return STRATA_ERR_ALIGNMENT;
+    const uintptr_t a = reinterpret_cast<uintptr_t>(dbase);
+    if (a + bytes < a) return STRATA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(ctx->mu);
+    for (const strata_region& r : ctx->regions)
+        if (a < r.base + r.bytes && r.base < a + bytes) return STRATA_ERR_INVALID_ARG;   // overlap
+    strata_region r{ctx->next_region++, a, bytes, 0};
+    ctx->regions.push_back(r);
+    *region_id = r.id;
+    return STRATA_OK;
+}
+
+strata_status strata_pool_is_ready(strata_ctx* ctx, const void* dptr, size_t bytes)
+{
+    if (!ctx || !dptr) return STRATA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(ctx->mu);
+    return region_contains(ctx, dptr, bytes) ? STRATA_OK : STRATA_ERR_NOT_REGISTERED;
+}
+
+strata_status strata_pool_unregister(strata_ctx* ctx, uint64_t region_id)
+{
+    if (!ctx) return STRATA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(ctx->mu);
+    for (size_t i = 0; i < ctx->regions.size(); ++i)
+        if (ctx->regions[i].id == region_id) {
+            ctx->regions.erase(ctx->regions.begin() + (long)i);
+            return STRATA_OK;
+        }
+    return STRATA_ERR_NOT_REGISTERED;
+}
+
+strata_status strata_pool_carve(strata_ctx* ctx, uint64_t region_id, size_t bytes, size_t align, void** dptr)
+{
+    if (!ctx || !dptr || align == 0 || (align & (align - 1)) != 0) return STRATA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(ctx->mu);
+    for (strata_region& r : ctx->regions)
+        if (r.id == region_id) {
+            const uintptr_t cur = r.base + r.used;
+            const uintptr_t al = (cur + (align - 1)) & ~(uintptr_t)(align - 1);
+            const size_t start = al - r.base;
+            if (start > r.bytes || bytes > r.bytes - start) return STRATA_ERR_CAPACITY;
+            r.used = start + bytes;
+            *dptr = reinterpret_cast<void*>(al);
+            return STRATA_OK;
+        }
+    return STRATA_ERR_NOT_REGISTERED;
+}
+
+strata_status strata_pool_reset(strata_ctx* ctx, uint64_t region_id)
+{
+    if (!ctx) return STRATA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(ctx->mu);
+    for (strata_region& r : ctx->regions)
+        if (r.id == region_id) {
+            r.used = 0;
+            return STRATA_OK;
+        }
+    return STRATA_ERR_NOT_REGISTERED;
+}
+
+// ---- hot path -----------------------------------------------------------------------
+
+strata_status strata_moe_layout(strata_ctx* ctx, const int32_t* topk_ids, const strata_moe_layout_t* layout,
+                                void* stream)
+{
+    if (!ctx || !topk_ids) return STRATA_ERR_INVALID_ARG;
+    strata_status st = check_layout_ptrs(layout, true);
+    if (st != STRATA_OK) return st;
+    if (!ctx->ws) return STRATA_ERR_WORKSPACE;
+    if (ctx->device < 0) return STRATA_ERR_CUDA;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return STRATA_ERR_CUDA;
+    int n = 0;
+    cudaError_t err = launch_layout(ctx->shape, topk_ids, *layout, ctx->ws, ctx->ws + kWsHeaderBytes / sizeof(int),
+                                    static_cast<cudaStream_t>(stream), &n);
+    {
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        ctx->launches += (uint64_t)n;
+    }
+    return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
+}
+
+strata_status strata_moe_dispatch(strata_ctx* ctx, const strata_moe_layout_t* layout, const void* x, void* recv,
+                                  float* recv_scale, size_t capacity_rows, void* stream)
+{
+    if (!ctx || !x || !recv) return STRATA_ERR_INVALID_ARG;
+    strata_status st = check_layout_ptrs(layout, false);
+    if (st != STRATA_OK) return st;
+    const strata_moe_shape& s = ctx->shape;
+    const bool fp8 = s.dispatch_dtype == STRATA_FP8_E4M3_B128;
+    if (fp8 != (recv_scale != nullptr)) return STRATA_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(recv) || (fp8 && !aligned16(recv_scale))) return STRATA_ERR_ALIGNMENT;
+    if (!ctx->ws) return STRATA_ERR_WORKSPACE;
+    const size_t n_rows = (size_t)s.R * s.T * s.K;
+    if (capacity_rows < n_rows) return STRATA_ERR_CAPACITY;
+    const size_t row_bytes = fp8 ? (size_t)s.H : (size_t)s.H * 2;
+    {
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        if (!region_contains(ctx, recv, capacity_rows * row_bytes)) return STRATA_ERR_NOT_REGISTERED;
+        if (fp8 && !region_contains(ctx, recv_scale, capacity_rows * (size_t)(s.H / 128) * sizeof(float)))
+            return STRATA_ERR_NOT_REGISTERED;
+    }
+    if (ctx->device < 0) return STRATA_ERR_CUDA;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return STRATA_ERR_CUDA;
+    cudaError_t err =
+        fp8 ? launch_dispatch_fp8(s, layout->dst_row, x, recv, recv_scale, capacity_rows, ctx->ws, ctx->n_sm,
+                                  static_cast<cudaStream_t>(stream))
+            : launch_dispatch_bf16(s, layout->dst_row, x, recv, capacity_rows, ctx->ws, ctx->n_sm,
+                                   static_cast<cudaStream_t>(stream));
+    {
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        ctx->launches += 1;
+    }
+    return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
+}
+
+strata_status strata_moe_combine(strata_ctx* ctx, const strata_moe_layout_t* layout, const void* y, size_t y_rows,
+                                 const float* topk_w, void* out, void* stream)
+{
+    if (!ctx || !y || !topk_w || !out) return STRATA_ERR_INVALID_ARG;
+    strata_status st = check_layout_ptrs(layout, false);
+    if (st != STRATA_OK) return st;
+    if (!aligned16(y) || !aligned16(out)) return STRATA_ERR_ALIGNMENT;
+    if (!ctx->ws) return STRATA_ERR_WORKSPACE;
+    if (ctx->device < 0) return STRATA_ERR_CUDA;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return STRATA_ERR_CUDA;
+    cudaError_t err = launch_combine(ctx->shape, layout->dst_row, y, y_rows, topk_w, out, ctx->ws, ctx->n_sm,
+                                     static_cast<cudaStream_t>(stream));
+    {
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        ctx->launches += 1;
+    }
+    return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
+}
+
+strata_status strata_moe_recv_view(strata_ctx* ctx, const int32_t* h_rank_offset, int rank, void* recv,
+                                   void** rank_base, int64_t* rows)
+{
+    if (!ctx || !h_rank_offset || !recv || !rank_base || !rows) return STRATA_ERR_INVALID_ARG;
+    const strata_moe_shape& s = ctx->shape;
+    if (rank < 0 || rank >= s.R) return STRATA_ERR_INVALID_ARG;
+    const int64_t lo = h_rank_offset[rank], hi = h_rank_offset[rank + 1];
+    if (lo < 0 || hi < lo) return STRATA_ERR_INVALID_ARG;
+    const size_t row_bytes = s.dispatch_dtype == STRATA_FP8_E4M3_B128 ? (size_t)s.H : (size_t)s.H * 2;
+    *rank_base = static_cast<unsigned char*>(recv) + (size_t)lo * row_bytes;
+    *rows = hi - lo;
+    return STRATA_OK;
+}
+
+strata_status strata_device_status(strata_ctx* ctx, void* stream, strata_status* out)
+{
+    if (!ctx || !out) return STRATA_ERR_INVALID_ARG;
+    if (!ctx->ws) return STRATA_ERR_WORKSPACE;
+    if (ctx->device < 0) return STRATA_ERR_CUDA;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return STRATA_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int word = 0;
+    if (cudaMemcpyAsync(&word, ctx->ws, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return STRATA_ERR_CUDA;
+    }
+    if (word != 0) {
+        if (cudaMemsetAsync(ctx->ws, 0, sizeof(int), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) {
+            cudaGetLastError();
+            return STRATA_ERR_CUDA;
+        }
+    }
+    *out = static_cast<strata_status>(word);
+    return STRATA_OK;
+}
+
+strata_status strata_moe_roundtrip_host(strata_ctx* ctx, const strata_moe_device_buffers* dev, const int32_t* h_ids,
+                                        const void* h_x, const float* h_w, void* h_out, void* stream)
+{
+    if (!ctx || !dev || !h_ids || !h_x || !h_w || !h_out) return STRATA_ERR_INVALID_ARG;
+    if (!dev->ids || !dev->x || !dev->w || !dev->recv || !dev->out) return STRATA_ERR_INVALID_ARG;
+    const strata_moe_shape& s = ctx->shape;
+    if (s.dispatch_dtype != STRATA_BF16) return STRATA_ERR_SHAPE;
+    if (ctx->device < 0) return STRATA_ERR_CUDA;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return STRATA_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t n_tok = (size_t)s.R * s.T, n = n_tok * s.K;
+    if (cudaMemcpyAsync(dev->ids, h_ids, n * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(dev->x, h_x, n_tok * s.H * 2, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(dev->w, h_w, n * sizeof(float), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return STRATA_ERR_CUDA;
+    }
+    strata_status rc = strata_moe_layout(ctx, dev->ids, &dev->layout, stream);
+    if (rc != STRATA_OK) return rc;
+    rc = strata_moe_dispatch(ctx, &dev->layout, dev->x, dev->recv, nullptr, n, stream);
+    if (rc != STRATA_OK) return rc;
+    rc = strata_moe_combine(ctx, &dev->layout, dev->recv, n, dev->w, dev->out, stream);
+    if (rc != STRATA_OK) return rc;
+    if (cudaMemcpyAsync(h_out, dev->out, n_tok * s.H * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return STRATA_ERR_CUDA;
+    }
+    return STRATA_OK;
+}
+
+}  // extern "C"

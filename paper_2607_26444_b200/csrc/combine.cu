@@ -1,0 +1,172 @@
+// Gate-weighted combine (paper Sec. 6.1, reduction-bearing operators: remote operands are
+// accumulated into the local destination).  Per token n and column c:
+//   out[n,c] = bf16_rne( fma(w[n,K-1], y[row(n,K-1),c], ... fma(w[n,0], y[row(n,0),c], +0) ) )
+// with binary32 fused multiply-adds in slot order 0..K-1.
+//
+// Work split: persistent CTAs take tokens round-robin; every token costs K row reads and one
+// row write, so the split is even whatever the expert popularity is.  A thread owns one
+// 16-byte column vector at a time: it issues the K independent 16-byte streaming loads first
+// (K requests in flight per thread), then runs the FMA chain in registers and writes 16 bytes.
+// The accumulation lives in registers; no atomics and no shared-memory staging are needed
+// because one thread sees all K operands of its columns.
+#include "common.cuh"
+
+namespace strata {
+
+namespace {
+
+constexpr int kCombineThreads = 128;
+
+struct CombineParams {
+    const int32_t* dst_row;
+    const unsigned char* y;
+    const float* w;
+    unsigned char* out;
+    long long n_tok;
+    long long y_rows;
+    int H;
+    int K;
+    int* status;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+__device__ __forceinline__ void fma8(float (&a)[8], float wv, const uint4& d)
+{
+    a[0] = __fmaf_rn(wv, __uint_as_float(d.x << 16), a[0]);
+    a[1] = __fmaf_rn(wv, __uint_as_float(d.x & 0xffff0000u), a[1]);
+    a[2] = __fmaf_rn(wv, __uint_as_float(d.y << 16), a[2]);
+    a[3] = __fmaf_rn(wv, __uint_as_float(d.y & 0xffff0000u), a[3]);
+    a[4] = __fmaf_rn(wv, __uint_as_float(d.z << 16), a[4]);
+    a[5] = __fmaf_rn(wv, __uint_as_float(d.z & 0xffff0000u), a[5]);
+    a[6] = __fmaf_rn(wv, __uint_as_float(d.w << 16), a[6]);
+    a[7] = __fmaf_rn(wv, __uint_as_float(d.w & 0xffff0000u), a[7]);
+}
+
+// K known at compile time: row pointers and weights of the token live in registers.
+template <int K>
+__global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams p)
+{
+    const int tid = threadIdx.x;
+    const int vpr = p.H / 8;                       // 16-byte vectors per row
+    const size_t row_bytes = (size_t)p.H * 2u;
+
+    for (long long n = blockIdx.x; n < p.n_tok; n += gridDim.x) {
+        const unsigned char* src[K];
+        float wk[K];
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            const int row = p.dst_row[n * K + k];
+            const bool row_ok = row >= 0 && row < p.y_rows;
+            if (!row_ok && tid == 0) report_status(p.status, STRATA_ERR_BAD_ROW);
+            src[k] = row_ok ? p.y + (size_t)row * row_bytes : nullptr;
+            wk[k] = p.w[n * K + k];
+        }
+        unsigned char* dst = p.out + (size_t)n * row_bytes;
+        for (int v = tid; v < vpr; v += kCombineThreads) {
+            uint4 d[K];
+#pragma unroll
+            for (int k = 0; k < K; ++k)
+                d[k] = src[k] ? ld_stream16(src[k] + (size_t)v * 16) : make_uint4(0, 0, 0, 0);
+            float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int k = 0; k < K; ++k)
+                if (src[k]) fma8(a, wk[k], d[k]);
+            uint4 o;
+            o.x = pack_bf16x2(a[0], a[1]);
+            o.y = pack_bf16x2(a[2], a[3]);
+            o.z = pack_bf16x2(a[4], a[5]);
+            o.w = pack_bf16x2(a[6], a[7]);
+            st_stream16(dst + (size_t)v * 16, o);
+        }
+    }
+}
+
+// Any K <= kMaxTopK: slots are taken in groups of up to 8, still in slot order.
+template <>
+__global__ void __launch_bounds__(kCombineThreads) combine_kernel<0>(CombineParams p)
+{
+    const int tid = threadIdx.x, K = p.K;
+    const int vpr = p.H / 8;
+    const size_t row_bytes = (size_t)p.H * 2u;
+    __shared__ long long s_off[kMaxTopK];          // byte offset of the row, -1 if skipped
+    __shared__ float s_w[kMaxTopK];
+
+    for (long long n = blockIdx.x; n < p.n_tok; n += gridDim.x) {
+        __syncthreads();
+        if (tid < K) {
+            const int row = p.dst_row[n * K + tid];
+            const bool row_ok = row >= 0 && row < p.y_rows;
+            if (!row_ok) report_status(p.status, STRATA_ERR_BAD_ROW);
+            s_off[tid] = row_ok ? (long long)row * (long long)row_bytes : -1;
+            s_w[tid] = p.w[n * K + tid];
+        }
+        __syncthreads();
+        unsigned char* dst = p.out + (size_t)n * row_bytes;
+        for (int v = tid; v < vpr; v += kCombineThreads) {
+            float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            for (int k0 = 0; k0 < K; k0 += 8) {
+                uint4 d[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const long long off = (k0 + k < K) ? s_off[k0 + k] : -1;
+                    d[k] = off >= 0 ? ld_stream16(p.y + off + (size_t)v * 16) : make_uint4(0, 0, 0, 0);
+                }
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (k0 + k < K && s_off[k0 + k] >= 0) fma8(a, s_w[k0 + k], d[k]);
+            }
+            uint4 o;
+            o.x = pack_bf16x2(a[0], a[1]);
+            o.y = pack_bf16x2(a[2], a[3]);
+            o.z = pack_bf16x2(a[4], a[5]);
+            o.w = pack_bf16x2(a[6], a[7]);
+            st_stream16(dst + (size_t)v * 16, o);
+        }
+    }
+}
+
+template <int KT>
+cudaError_t launch_k(const CombineParams& p, int n_sm, cudaStream_t st)
+{
+    int per_sm = 0;
+    cudaError_t err =
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, combine_kernel<KT>, kCombineThreads, 0);
+    if (err != cudaSuccess) return err;
+    if (per_sm < 1) per_sm = 1;
+    const long long grid = min((long long)n_sm * per_sm, p.n_tok);
+    combine_kernel<KT><<<(unsigned)grid, kCombineThreads, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_combine(const strata_moe_shape& s, const int32_t* dst_row, const void* y, size_t y_rows,
+                           const float* w, void* out, int* status, int n_sm, cudaStream_t st)
+{
+    CombineParams p{};
+    p.dst_row = dst_row;
+    p.y = static_cast<const unsigned char*>(y);
+    p.w = w;
+    p.out = static_cast<unsigned char*>(out);
+    p.n_tok = (long long)s.R * s.T;
+    p.y_rows = (long long)y_rows;
+    p.H = s.H;
+    p.K = s.K;
+    p.status = status;
+    switch (s.K) {
+        case 1: return launch_k<1>(p, n_sm, st);
+        case 2: return launch_k<2>(p, n_sm, st);
+        case 4: return launch_k<4>(p, n_sm, st);
+        case 6: return launch_k<6>(p, n_sm, st);
+        case 8: return launch_k<8>(p, n_sm, st);
+        default: return launch_k<0>(p, n_sm, st);
+    }
+}
+
+}  // namespace strata

@@ -1,0 +1,313 @@
+// Token dispatch (paper Sec. 6.2 / 7.1): every token's hidden vector goes to the K receive rows
+// the layout assigned, straight into the caller's (registered) receive buffer.
+//
+// Work split: a unit is one token (or one column chunk of a token when a row is larger than
+// a stage).  Units are dealt round-robin to a persistent grid, so every CTA moves the same
+// number of bytes whatever the expert popularity is: 1 row read + K row writes per unit.
+//
+// bf16: each CTA is a single warp that runs the SM's bulk-copy engine as a small DMA program
+//       (the on-SM counterpart of the paper's device-issued SDMA descriptors, Sec. 6.3):
+//       bulk load global->shared into a ring of stages, completion on an mbarrier, then K bulk
+//       stores shared->global.  No register or ALU touches the payload.
+// fp8:  128-thread CTAs; the row lands in shared memory the same way, the threads compute
+//       the per-128-column amax, scale = amax/448 and the e4m3 codes into an output stage,
+//       and K bulk stores ship the codes; the scales (H/128 floats per row) go out with plain
+//       coalesced stores.
+#include "common.cuh"
+
+namespace strata {
+
+namespace {
+
+constexpr uint32_t kMaxChunkBytes = 16384;   // one stage of the bf16 ring
+constexpr int kBf16Stages = 3;
+constexpr int kFp8Threads = 128;
+constexpr int kFp8MaxChunkCols = 4096;       // 8 KB in, 4 KB out per stage
+
+struct DispatchParams {
+    const int32_t* dst_row;
+    const unsigned char* x;
+    unsigned char* recv;
+    float* recv_scale;
+    long long n_units;          // n_tok * chunks_per_row
+    long long capacity_rows;
+    int K;
+    int H;
+    int chunks_per_row;
+    uint32_t chunk_cols;        // columns per chunk (last chunk of a row may be shorter)
+    int* status;
+};
+
+__global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    const uint32_t stage_bytes = p.chunk_cols * 2u;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kBf16Stages * stage_bytes);
+    const int lane = threadIdx.x;
+    const size_t row_bytes = (size_t)p.H * 2u;
+
+    const long long first = blockIdx.x, stride = gridDim.x;
+    if (first >= p.n_units) return;
+    const long long n_my = (p.n_units - first + stride - 1) / stride;
+
+    if (lane == 0) {
+        for (int s = 0; s < kBf16Stages; ++s) mbar_init(&bars[s], 1);
+        mbar_fence_init();
+    }
+    __syncwarp();
+    const uint64_t pol = policy_evict_first();
+
+    auto issue_load = [&](long long j) {   // lane 0 only
+        const long long u = first + j * stride;
+        const long long tok = u / p.chunks_per_row;
+        const int ch = (int)(u - tok * p.chunks_per_row);
+        const uint32_t col0 = (uint32_t)ch * p.chunk_cols;
+        const uint32_t bytes = min(p.chunk_cols, (uint32_t)p.H - col0) * 2u;
+        const int s = (int)(j % kBf16Stages);
+        mbar_expect_tx(&bars[s], bytes);
+        bulk_g2s(smem + (size_t)s * stage_bytes, p.x + (size_t)tok * row_bytes + (size_t)col0 * 2u, bytes, &bars[s],
+                 pol);
+    };
+
+    if (lane == 0)
+        for (long long j = 0; j < kBf16Stages - 1 && j < n_my; ++j) issue_load(j);
+
+    bool ok = true;
+    for (long long j = 0; j < n_my; ++j) {
+        const long long u = first + j * stride;
+        const long long tok = u / p.chunks_per_row;
+        const int ch = (int)(u - tok * p.chunks_per_row);
+        const uint32_t col0 = (uint32_t)ch * p.chunk_cols;
+        const uint32_t bytes = min(p.chunk_cols, (uint32_t)p.H - col0) * 2u;
+        const int s = (int)(j % kBf16Stages);
+        const uint32_t parity = (uint32_t)((j / kBf16Stages) & 1);
+
+        const int my_row = (lane < p.K) ? p.dst_row[tok * p.K + lane] : -1;
+        const bool row_ok = (lane >= p.K) || (my_row >= 0 && my_row < p.capacity_rows);
+        if (!row_ok) report_status(p.status, STRATA_ERR_BAD_ROW);
+
+        ok = mbar_wait_bounded(&bars[s], parity);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+
+        for (int k = 0; k < p.K; ++k) {
+            const int row = __shfl_sync(0xffffffffu, my_row, k);
+            if (lane == 0 && row >= 0 && row < p.capacity_rows)
+                bulk_s2g(p.recv + (size_t)row * row_bytes + (size_t)col0 * 2u, smem + (size_t)s * stage_bytes, bytes);
+        }
+        if (lane == 0) {
+            bulk_commit();
+            // The stage that unit j-1 used is refilled next; its stores must have left shared memory.
+            const long long jn = j + kBf16Stages - 1;
+            if (jn < n_my) {
+                bulk_wait_read<1>();
+                issue_load(jn);
+            }
+        }
+        __syncwarp();
+    }
+    if (lane == 0) {
+        if (!ok) report_status(p.status, STRATA_ERR_TIMEOUT);
+        bulk_wait_read<0>();
+    }
+}
+
+// ---- fp8 -------------------------------------------------------------------------
+
+__device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+// e4m3 (OCP "fn"), round to nearest even, saturating to +-448; `hi` lands in the upper byte.
+__device__ __forceinline__ uint32_t cvt_e4m3x2(float hi, float lo)
+{
+    uint16_t d;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+__global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParams p)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    const uint32_t in_bytes = p.chunk_cols * 2u, out_bytes = p.chunk_cols;
+    auto in_stage = [&](int s) { return smem + (size_t)s * in_bytes; };
+    auto out_stage = [&](int s) { return smem + 2 * (size_t)in_bytes + (size_t)s * out_bytes; };
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * in_bytes + 2 * out_bytes);
+    const int tid = threadIdx.x, lane = tid & 31;
+    const size_t in_row_bytes = (size_t)p.H * 2u, out_row_bytes = (size_t)p.H;
+    const int nb_row = p.H / 128;
+
+    const long long first = blockIdx.x, stride = gridDim.x;
+    if (first >= p.n_units) return;
+    const long long n_my = (p.n_units - first + stride - 1) / stride;
+
+    if (tid == 0) {
+        mbar_init(&bars[0], 1);
+        mbar_init(&bars[1], 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+    const uint64_t pol = policy_evict_first();
+
+    auto issue_load = [&](long long j) {   // thread 0 only
+        const long long u = first + j * stride;
+        const long long tok = u / p.chunks_per_row;
+        const int ch = (int)(u - tok * p.chunks_per_row);
+        const uint32_t col0 = (uint32_t)ch * p.chunk_cols;
+        const uint32_t cols = min(p.chunk_cols, (uint32_t)p.H - col0);
+        const int s = (int)(j & 1);
+        mbar_expect_tx(&bars[s], cols * 2u);
+        bulk_g2s(in_stage(s), p.x + (size_t)tok * in_row_bytes + (size_t)col0 * 2u, cols * 2u, &bars[s], pol);
+    };
+    if (tid == 0) {
+        issue_load(0);
+        if (n_my > 1) issue_load(1);
+    }
+
+    __shared__ int s_rows[kMaxTopK];
+    __shared__ float s_scale[kFp8MaxChunkCols / 128];
+    bool ok = true;
+    for (long long j = 0; j < n_my; ++j) {
+        const long long u = first + j * stride;
+        const long long tok = u / p.chunks_per_row;
+        const int ch = (int)(u - tok * p.chunks_per_row);
+        const uint32_t col0 = (uint32_t)ch * p.chunk_cols;
+        const uint32_t cols = min(p.chunk_cols, (uint32_t)p.H - col0);
+        const int s = (int)(j & 1);
+        const uint32_t parity = (uint32_t)((j >> 1) & 1);
+
+        if (tid < p.K) {
+            const int row = p.dst_row[tok * p.K + tid];
+            const bool row_ok = row >= 0 && row < p.capacity_rows;
+            if (!row_ok) report_status(p.status, STRATA_ERR_BAD_ROW);
+            s_rows[tid] = row_ok ? row : -1;
+        }
+        if (tid == 0) bulk_wait_read<1>();     // stores of unit j-2 have left out_stage(s)
+        ok = mbar_wait_bounded(&bars[s], parity);
+        ok = __syncthreads_and(ok);
+        if (!ok) break;
+
+        const uint4* in = reinterpret_cast<const uint4*>(in_stage(s));
+        uint2* outq = reinterpret_cast<uint2*>(out_stage(s));
+        const uint32_t nvec = cols / 8;        // multiple of 16
+        for (uint32_t v0 = (uint32_t)(tid - lane); v0 < nvec; v0 += kFp8Threads) {
+            const uint32_t v = v0 + lane;
+            const bool act = v < nvec;
+            uint4 d = act ? in[v] : make_uint4(0, 0, 0, 0);
+            float f[8] = {bf16lo(d.x), bf16hi(d.x), bf16lo(d.y), bf16hi(d.y),
+                          bf16lo(d.z), bf16hi(d.z), bf16lo(d.w), bf16hi(d.w)};
+            float amax = 0.0f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(f[i]));
+#pragma unroll
+            for (int m = 8; m >= 1; m >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, m));
+            const float scale = __fdiv_rn(amax, 448.0f);
+            const float dv = (amax == 0.0f) ? 1.0f : scale;
+            float q[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) q[i] = __fdiv_rn(f[i], dv);
+            uint2 o;
+            o.x = cvt_e4m3x2(q[1], q[0]) | (cvt_e4m3x2(q[3], q[2]) << 16);
+            o.y = cvt_e4m3x2(q[5], q[4]) | (cvt_e4m3x2(q[7], q[6]) << 16);
+            if (act) {
+                outq[v] = o;
+                if ((lane & 15) == 0) s_scale[v >> 4] = scale;
+            }
+        }
+        fence_async_smem();
+        __syncthreads();
+        {   // scales: K rows x (cols/128) floats, coalesced along the row
+            const int nb = (int)(cols >> 7);
+            for (int idx = tid; idx < p.K * nb; idx += kFp8Threads) {
+                const int k = idx / nb, b = idx - k * nb;
+                const int row = s_rows[k];
+                if (row >= 0) p.recv_scale[(size_t)row * nb_row + (col0 >> 7) + b] = s_scale[b];
+            }
+        }
+        if (tid == 0) {
+            for (int k = 0; k < p.K; ++k) {
+                const int row = s_rows[k];
+                if (row >= 0) bulk_s2g(p.recv + (size_t)row * out_row_bytes + col0, out_stage(s), cols);
+            }
+            bulk_commit();
+            if (j + 2 < n_my) issue_load(j + 2);    // in_stage(s) was fully consumed before the barrier above
+        }
+        __syncthreads();                            // s_rows is rewritten next iteration
+    }
+    if (tid == 0) {
+        if (!ok) report_status(p.status, STRATA_ERR_TIMEOUT);
+        bulk_wait_read<0>();
+    }
+}
+
+uint32_t pick_chunk_cols_bf16(int H)
+{
+    const uint32_t row_bytes = (uint32_t)H * 2u;
+    if (row_bytes <= kMaxChunkBytes) return (uint32_t)H;
+    const uint32_t n = (row_bytes + kMaxChunkBytes - 1) / kMaxChunkBytes;
+    uint32_t cols = ((uint32_t)H + n - 1) / n;
+    cols = (cols + 7u) & ~7u;        // chunks start on 16-byte boundaries
+    return cols;
+}
+
+}  // namespace
+
+cudaError_t configure_dispatch_kernels()
+{
+    cudaError_t err = cudaFuncSetAttribute(dispatch_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           kBf16Stages * (int)kMaxChunkBytes + 64);
+    if (err != cudaSuccess) return err;
+    return cudaFuncSetAttribute(dispatch_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                kFp8MaxChunkCols * 6 + 64);
+}
+
+cudaError_t launch_dispatch_bf16(const strata_moe_shape& s, const int32_t* dst_row, const void* x, void* recv,
+                                 size_t capacity_rows, int* status, int n_sm, cudaStream_t st)
+{
+    DispatchParams p{};
+    p.dst_row = dst_row;
+    p.x = static_cast<const unsigned char*>(x);
+    p.recv = static_cast<unsigned char*>(recv);
+    p.recv_scale = nullptr;
+    p.K = s.K;
+    p.H = s.H;
+    p.chunk_cols = pick_chunk_cols_bf16(s.H);
+    p.chunks_per_row = (int)(((uint32_t)s.H + p.chunk_cols - 1) / p.chunk_cols);
+    p.n_units = (long long)s.R * s.T * p.chunks_per_row;
+    p.capacity_rows = (long long)capacity_rows;
+    p.status = status;
+    const size_t smem = (size_t)kBf16Stages * p.chunk_cols * 2u + 64;
+    int per_sm = 0;
+    cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dispatch_bf16_kernel, 32, smem);
+    if (err != cudaSuccess) return err;
+    if (per_sm < 1) per_sm = 1;
+    const long long grid = min((long long)n_sm * per_sm, p.n_units);
+    dispatch_bf16_kernel<<<(unsigned)grid, 32, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_dispatch_fp8(const strata_moe_shape& s, const int32_t* dst_row, const void* x, void* recv_q,
+                                float* recv_scale, size_t capacity_rows, int* status, int n_sm, cudaStream_t st)
+{
+    DispatchParams p{};
+    p.dst_row = dst_row;
+    p.x = static_cast<const unsigned char*>(x);
+    p.recv = static_cast<unsigned char*>(recv_q);
+    p.recv_scale = recv_scale;
+    p.K = s.K;
+    p.H = s.H;
+    p.chunk_cols = (uint32_t)min(s.H, kFp8MaxChunkCols);
+    p.chunks_per_row = (int)(((uint32_t)s.H + p.chunk_cols - 1) / p.chunk_cols);
+    p.n_units = (long long)s.R * s.T * p.chunks_per_row;
+    p.capacity_rows = (long long)capacity_rows;
+    p.status = status;
+    const size_t smem = (size_t)p.chunk_cols * 6u + 64;
+    int per_sm = 0;
+    cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dispatch_fp8_kernel, kFp8Threads, smem);
+    if (err != cudaSuccess) return err;
+    if (per_sm < 1) per_sm = 1;
+    const long long grid = min((long long)n_sm * per_sm, p.n_units);
+    dispatch_fp8_kernel<<<(unsigned)grid, kFp8Threads, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace strata

@@ -1,0 +1,373 @@
+"""GPU-vs-oracle parity through the C ABI (run with -m gpu on a B200).
+
+Bars: layout, bf16 dispatch and e4m3 dispatch bit-exact; combine within 1 bf16
+ulp (both sides run the same fp32 FMA chain, so equality is expected and the
+ulp bound is the stated tolerance).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_26444_b200 import binding as B
+from paper_2607_26444_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+SENTINEL16 = 0x7FC7          # a NaN pattern no input contains
+GUARD = 3
+
+
+def ulp_distance(a: np.ndarray, b: np.ndarray) -> np.ndarray:
+    def line(u):
+        u = u.astype(np.int32)
+        return np.where(u & 0x8000, -(u & 0x7FFF), u & 0x7FFF)
+    return np.abs(line(a) - line(b))
+
+
+def to_dev(a: np.ndarray) -> torch.Tensor:
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).to(DEV)
+    return torch.from_numpy(a).to(DEV)
+
+
+def u16(t: torch.Tensor) -> np.ndarray:
+    return t.cpu().numpy().view(np.uint16)
+
+
+def make_ctx(cfg: wl.MoEConfig) -> B.MoEContext:
+    return B.MoEContext(cfg.R, cfg.T, cfg.H, cfg.E, cfg.K, cfg.dispatch_dtype)
+
+
+def assert_layout_equal(lay: B.Layout, ref: dict):
+    torch.cuda.synchronize()
+    for key in ("expert_count", "expert_offset", "rank_count", "rank_offset", "src_expert_count", "dst_row",
+                "src_of_row"):
+        got = getattr(lay, key).cpu().numpy()
+        assert np.array_equal(got, ref[key]), key
+
+
+def guarded(n_rows: int, width: int, dtype, fill):
+    """A tensor of n_rows+2*GUARD rows filled with a sentinel; returns (whole, middle view)."""
+    whole = torch.full((n_rows + 2 * GUARD, width), fill, dtype=dtype, device=DEV)
+    return whole, whole[GUARD:GUARD + n_rows]
+
+
+def run_full_case(cfg: wl.MoEConfig, inp=None, threads=8):
+    """Whole path on one config, every output compared with the oracle element by element."""
+    inp = inp or wl.generate(cfg)
+    ref_lay = oracle.layout(inp["ids"], cfg.E)
+    N, n_tok, H, K = cfg.n_items, cfg.n_tok, cfg.H, cfg.K
+    fp8 = cfg.dispatch_dtype == wl.FP8_E4M3_B128
+
+    ctx = make_ctx(cfg)
+    ids_d, x_d, w_d = to_dev(inp["ids"]), to_dev(inp["x"]), to_dev(inp["w"])
+    lay = ctx.layout(ids_d)
+    assert_layout_equal(lay, ref_lay)
+
+    if fp8:
+        whole, recv = guarded(N, H, torch.uint8, 0x7F)
+        whole_s, recv_s = guarded(N, H // 128, torch.float32, -7.0)
+        ctx.register(whole)
+        ctx.register(whole_s)
+        ctx.dispatch(lay, x_d, recv, recv_s)
+        ref_q, ref_s = oracle.dispatch_fp8(ref_lay["dst_row"], inp["x"], nthreads=threads)
+        got_q, got_s = recv.cpu().numpy(), recv_s.cpu().numpy()
+        assert np.array_equal(got_q, ref_q)
+        assert np.array_equal(got_s.view(np.uint32), ref_s.view(np.uint32))
+        hw, hs = whole.cpu().numpy(), whole_s.cpu().numpy()
+        assert np.all(hw[:GUARD] == 0x7F) and np.all(hw[GUARD + N:] == 0x7F)
+        assert np.all(hs[:GUARD] == -7.0) and np.all(hs[GUARD + N:] == -7.0)
+        y = wl.expert_standin(cfg, ref_q, ref_lay["expert_offset"], ref_s)
+    else:
+        whole, recv = guarded(N, H, torch.int16, SENTINEL16)
+        ctx.register(whole)
+        ctx.dispatch(lay, x_d, recv)
+        ref_recv = oracle.dispatch_bf16(ref_lay["dst_row"], inp["x"], nthreads=threads)
+        assert np.array_equal(u16(recv), ref_recv)
+        hw = u16(whole)
+        assert np.all(hw[:GUARD] == SENTINEL16) and np.all(hw[GUARD + N:] == SENTINEL16)
+        y = wl.expert_standin(cfg, ref_recv, ref_lay["expert_offset"])
+
+    y_d = recv if (cfg.expert == "identity" and not fp8) else to_dev(y)
+    out_whole, out = guarded(n_tok, H, torch.int16, SENTINEL16)
+    ctx.combine(lay, y_d, w_d, out)
+    ref_out = oracle.combine(ref_lay["dst_row"], y, inp["w"], nthreads=threads)
+    got_out = u16(out)
+    d = ulp_distance(got_out, ref_out)
+    assert d.max() <= 1, f"combine: max ulp distance {d.max()}"
+    assert np.array_equal(got_out, ref_out), "combine: expected bit equality (same FMA chain)"
+    ow = u16(out_whole)
+    assert np.all(ow[:GUARD] == SENTINEL16) and np.all(ow[GUARD + n_tok:] == SENTINEL16)
+    if cfg.expert == "identity" and not fp8:
+        assert np.array_equal(got_out, inp["x"].reshape(n_tok, H))     # gate weights sum to 1
+    assert ctx.device_status() == B.STRATA_OK
+    ctx.close()
+
+
+# ---- the five benchmark configurations --------------------------------------------
+
+def test_tiny_full():
+    run_full_case(wl.CONFIGS["tiny"])
+
+
+def test_decode_full():
+    run_full_case(wl.CONFIGS["decode"])
+
+
+def test_skew_full():
+    run_full_case(wl.CONFIGS["skew"])
+
+
+def test_fp8_full():
+    run_full_case(wl.CONFIGS["fp8"])
+
+
+def test_prefill_full_size_sampled():
+    """The benchmark's launch configuration at full size (7.5 GB receive buffer): layout compared
+    in full; dispatch and combine on sampled outputs the oracle computes one by one, plus the
+    properties that hold at any size (row equality through dst_row; identity experts return x)."""
+    cfg = wl.CONFIGS["prefill"]
+    inp = wl.generate(cfg)
+    ref_lay = oracle.layout(inp["ids"], cfg.E)
+    N, n_tok, H, K = cfg.n_items, cfg.n_tok, cfg.H, cfg.K
+    ctx = make_ctx(cfg)
+    ids_d, x_d, w_d = to_dev(inp["ids"]), to_dev(inp["x"]), to_dev(inp["w"])
+    lay = ctx.layout(ids_d)
+    assert_layout_equal(lay, ref_lay)
+
+    slab = torch.empty(N * H * 2 + 4096, dtype=torch.uint8, device=DEV)
+    rid = ctx.register(slab)
+    recv = ctx.carve(rid, (N, H), torch.int16)
+    recv.fill_(SENTINEL16)
+    ctx.dispatch(lay, x_d, recv)
+    torch.cuda.synchronize()
+
+    x2 = x_d.view(n_tok, H)
+    x_host = inp["x"].reshape(n_tok, H)
+    # sampled rows against the oracle's placement: row j holds the token of item src_of_row[j]
+    rng = np.random.default_rng(0)
+    rows = np.unique(np.concatenate([rng.integers(0, N, 4096), [0, N - 1],
+                                     ref_lay["expert_offset"][:-1].clip(0, N - 1)]))
+    got = u16(recv[torch.from_numpy(rows).to(DEV)])
+    want = x_host[ref_lay["src_of_row"][rows] // K]
+    assert np.array_equal(got, want)
+    # every row, on the device: recv[dst_row[i]] == x[i // K]
+    dst = lay.dst_row.view(n_tok, K).long()
+    for lo in range(0, n_tok, 8192):
+        hi = min(n_tok, lo + 8192)
+        for k in range(K):
+            assert torch.equal(recv[dst[lo:hi, k]], x2[lo:hi])
+
+    out = torch.empty((n_tok, H), dtype=torch.int16, device=DEV)
+    ctx.combine(lay, recv, w_d, out)
+    torch.cuda.synchronize()
+    # sampled tokens, one by one through the oracle (identity experts: the K rows are the token's own row)
+    toks = np.unique(np.concatenate([rng.integers(0, n_tok, 1024), [0, n_tok - 1]]))
+    y_mini = np.repeat(x_host[toks], K, axis=0)
+    d_mini = np.arange(toks.size * K, dtype=np.int32).reshape(-1, K)
+    want_out = oracle.combine(d_mini, y_mini, inp["w"].reshape(n_tok, K)[toks], nthreads=4)
+    got_out = u16(out[torch.from_numpy(toks).to(DEV)])
+    assert ulp_distance(got_out, want_out).max() <= 1
+    assert np.array_equal(got_out, want_out)
+    assert torch.equal(out, x2)                        # invariant at full size
+    assert ctx.device_status() == B.STRATA_OK
+    ctx.close()
+
+
+# ---- ragged, degenerate and extreme shapes -------------------------------------------
+
+RAGGED = [
+    dict(R=1, T=1, H=8, E=1, K=1),
+    dict(R=3, T=7, H=24, E=6, K=3),
+    dict(R=2, T=300, H=1000, E=10, K=5),            # T*K = 1500: two tiles per rank, ragged tail
+    dict(R=4, T=1030, H=256, E=64, K=1),
+    dict(R=2, T=65, H=8200, E=4, K=2),               # row of 16400 B: two chunks per row
+    dict(R=2, T=40, H=20000, E=8, K=4),              # three chunks, ragged last chunk
+    dict(R=8, T=33, H=512, E=1024, K=8),             # maximum expert count
+    dict(R=1, T=200, H=64, E=48, K=32),              # maximum top-k (generic combine path)
+    dict(R=2, T=129, H=136, E=12, K=9),
+    dict(R=5, T=50, H=4096, E=20, K=6),
+    dict(R=4, T=100, H=2048, E=16, K=4),
+]
+
+
+@pytest.mark.parametrize("kw", RAGGED, ids=lambda kw: "R{R}T{T}H{H}E{E}K{K}".format(**kw))
+def test_ragged_shapes(kw):
+    cfg = wl.shrink(wl.CONFIGS["decode"], seed=4242 + kw["T"], **kw)
+    run_full_case(cfg, threads=4)
+
+
+@pytest.mark.parametrize("kw", [dict(R=2, T=50, H=128, E=4, K=2), dict(R=4, T=300, H=1920, E=32, K=8),
+                                dict(R=1, T=9, H=4224, E=2, K=2), dict(R=2, T=20, H=8192 + 128, E=8, K=3)],
+                         ids=lambda kw: "R{R}T{T}H{H}E{E}K{K}".format(**kw))
+def test_ragged_shapes_fp8(kw):
+    cfg = wl.shrink(wl.CONFIGS["fp8"], seed=99 + kw["T"], **kw)
+    run_full_case(cfg, threads=4)
+
+
+def test_duplicate_ids_and_all_to_one_expert():
+    cfg = wl.shrink(wl.CONFIGS["tiny"], R=4, T=600, H=64, E=8, K=4, expert="scale")
+    inp = wl.generate(cfg)
+    rng = np.random.default_rng(1)
+    inp["ids"] = rng.integers(0, 3, size=inp["ids"].shape).astype(np.int32)      # duplicates, empty experts
+    run_full_case(cfg, inp)
+    inp["ids"][:] = 5                                                           # a single hot expert
+    run_full_case(cfg, inp)
+
+
+def test_zipf_small():
+    cfg = wl.shrink(wl.CONFIGS["skew"], R=8, T=200, H=512, E=32, K=8)
+    run_full_case(cfg)
+
+
+def test_fp8_extreme_values_every_bf16_pattern():
+    """All finite bf16 bit patterns as inputs, arranged so that blocks have very different amax
+    (and some are all zero): codes and scales must equal the oracle's bit for bit."""
+    cfg = wl.shrink(wl.CONFIGS["fp8"], R=2, T=128, H=512, E=4, K=2)
+    inp = wl.generate(cfg)
+    bits = np.arange(65536, dtype=np.uint32)
+    finite = bits[(bits & 0x7F80) != 0x7F80].astype(np.uint16)
+    rng = np.random.default_rng(7)
+    x = inp["x"].reshape(-1)
+    # sorted by magnitude so that a block holds values of similar size (exercises subnormal codes
+    # of tiny blocks as well as the saturating top), then some shuffled blocks for mixed ranges
+    mag = np.sort(finite & 0x7FFF)
+    sign = (rng.integers(0, 2, mag.size) << 15).astype(np.uint16)
+    x[:mag.size] = mag | sign
+    x[mag.size:2 * mag.size] = rng.permutation(finite)
+    x[2 * mag.size:2 * mag.size + 256] = 0
+    x[2 * mag.size + 256:2 * mag.size + 384] = 0x8000
+    run_full_case(cfg, inp)
+
+
+# ---- behaviour of the boundary on a real device ---------------------------------------
+
+def test_layout_is_deterministic():
+    cfg = wl.CONFIGS["skew"]
+    ids_d = to_dev(wl.gen_topk_ids(cfg))
+    ctx = make_ctx(cfg)
+    first = ctx.layout(ids_d)
+    torch.cuda.synchronize()
+    ref = {k: getattr(first, k).clone() for k in ("dst_row", "src_of_row", "expert_offset", "src_expert_count")}
+    lay = ctx.new_layout()
+    for _ in range(20):
+        ctx.layout(ids_d, lay)
+        torch.cuda.synchronize()
+        for k, v in ref.items():
+            assert torch.equal(getattr(lay, k), v), k
+    ctx.close()
+
+
+def test_bad_expert_id_is_skipped_and_reported():
+    cfg = wl.shrink(wl.CONFIGS["tiny"], H=64)
+    inp = wl.generate(cfg)
+    ids = inp["ids"].copy()
+    ids[1, 5, 0] = cfg.E          # out of range
+    ids[2, 9, 1] = -3
+    ctx = make_ctx(cfg)
+    lay = ctx.layout(to_dev(ids))
+    assert ctx.device_status() == B.STRATA_ERR_BAD_EXPERT_ID
+    assert ctx.device_status() == B.STRATA_OK                      # reading clears it
+    dst = lay.dst_row.cpu().numpy()
+    assert dst[1, 5, 0] == -1 and dst[2, 9, 1] == -1
+    valid = np.ones(ids.shape, bool)
+    valid[1, 5, 0] = valid[2, 9, 1] = False
+    N = cfg.n_items
+    assert lay.expert_count.sum().item() == N - 2
+    assert np.array_equal(np.sort(dst[valid]), np.arange(N - 2))   # the rest is still a packed bijection
+    # the valid items keep their relative (expert, rank, token, slot) order
+    order = np.lexsort((np.arange(N)[valid.ravel()], ids.ravel()[valid.ravel()]))
+    assert np.array_equal(dst.ravel()[valid.ravel()][order], np.arange(N - 2))
+    # dispatch skips the two items, reports a bad row, writes nothing out of bounds
+    whole, recv = guarded(N, cfg.H, torch.int16, -1)
+    ctx.register(whole)
+    ctx.dispatch(lay, to_dev(inp["x"]), recv)
+    assert ctx.device_status() == B.STRATA_ERR_BAD_ROW
+    hw = whole.cpu().numpy()
+    assert np.all(hw[:GUARD] == -1) and np.all(hw[GUARD + N - 2:] == -1)
+    x2 = inp["x"].reshape(cfg.n_tok, cfg.H)
+    got = hw[GUARD:GUARD + N - 2].view(np.uint16)
+    assert np.array_equal(got[dst.ravel()[valid.ravel()]], x2[(np.arange(N) // cfg.K)[valid.ravel()]])
+    # combine ignores the skipped slots
+    out = torch.zeros((cfg.n_tok, cfg.H), dtype=torch.int16, device=DEV)
+    ctx.combine(lay, recv, to_dev(inp["w"]), out)
+    assert ctx.device_status() == B.STRATA_ERR_BAD_ROW
+    ctx.close()
+
+
+def test_host_errors_on_device_context():
+    cfg = wl.shrink(wl.CONFIGS["tiny"], H=64)
+    ctx = make_ctx(cfg)
+    inp = wl.generate(cfg)
+    lay = ctx.layout(to_dev(inp["ids"]))
+    x_d = to_dev(inp["x"])
+    recv = torch.empty((cfg.n_items, cfg.H), dtype=torch.int16, device=DEV)
+    with pytest.raises(B.StrataError) as ei:
+        ctx.dispatch(lay, x_d, recv)                               # not registered
+    assert ei.value.code == B.STRATA_ERR_NOT_REGISTERED
+    ctx.register(recv)
+    with pytest.raises(B.StrataError) as ei:
+        ctx.dispatch(lay, x_d, recv[:-1])                          # too few rows
+    assert ei.value.code == B.STRATA_ERR_CAPACITY
+    with pytest.raises(B.StrataError) as ei:
+        ctx.dispatch(lay, x_d.view(-1)[4:], recv)                  # 8-byte offset
+    assert ei.value.code == B.STRATA_ERR_ALIGNMENT
+    ctx.dispatch(lay, x_d, recv)
+    assert ctx.device_status() == B.STRATA_OK
+    assert ctx.launch_count() == 3                                 # 2 (layout) + 1 (dispatch); failures launched nothing
+    ctx.close()
+
+
+def test_zero_copy_rank_partitions():
+    """The receive buffer is carved from a registered slab; rank d's partition is a plain view of it."""
+    cfg = wl.CONFIGS["tiny"]
+    inp = wl.generate(cfg)
+    ref_lay = oracle.layout(inp["ids"], cfg.E)
+    ctx = make_ctx(cfg)
+    slab = torch.zeros(cfg.n_items * cfg.H * 2 + 1024, dtype=torch.uint8, device=DEV)
+    rid = ctx.register(slab)
+    recv = ctx.carve(rid, (cfg.n_items, cfg.H), torch.int16)
+    assert recv.data_ptr() == slab.data_ptr()
+    lay = ctx.layout(to_dev(inp["ids"]))
+    ctx.dispatch(lay, to_dev(inp["x"]), recv)
+    torch.cuda.synchronize()
+    h_off = lay.rank_offset.cpu().numpy()
+    ref_recv = oracle.dispatch_bf16(ref_lay["dst_row"], inp["x"])
+    for d in range(cfg.R):
+        rc, base, rows = B.strata_moe_recv_view(ctx.h, h_off, d, recv.data_ptr())
+        assert rc == 0 and rows == ref_lay["rank_count"][d]
+        assert base == recv.data_ptr() + int(ref_lay["rank_offset"][d]) * cfg.H * 2
+        part = recv[h_off[d]:h_off[d + 1]]
+        assert part.data_ptr() == base
+        assert np.array_equal(u16(part), ref_recv[h_off[d]:h_off[d + 1]])
+    ctx.close()
+
+
+def test_roundtrip_from_host_buffers():
+    cfg = wl.CONFIGS["tiny"]
+    inp = wl.generate(cfg)
+    ctx = make_ctx(cfg)
+    lay = ctx.new_layout()
+    ids_d = torch.empty((cfg.R, cfg.T, cfg.K), dtype=torch.int32, device=DEV)
+    x_d = torch.empty((cfg.R, cfg.T, cfg.H), dtype=torch.int16, device=DEV)
+    w_d = torch.empty((cfg.R, cfg.T, cfg.K), dtype=torch.float32, device=DEV)
+    recv = torch.empty((cfg.n_items, cfg.H), dtype=torch.int16, device=DEV)
+    out_d = torch.empty((cfg.n_tok, cfg.H), dtype=torch.int16, device=DEV)
+    ctx.register(recv)
+    dev = B.strata_moe_device_buffers(ids_d.data_ptr(), x_d.data_ptr(), w_d.data_ptr(), recv.data_ptr(),
+                                      out_d.data_ptr(), lay.c)
+    h_ids = torch.from_numpy(inp["ids"]).pin_memory()
+    h_x = torch.from_numpy(inp["x"].view(np.int16)).pin_memory()
+    h_w = torch.from_numpy(inp["w"]).pin_memory()
+    h_out = torch.empty((cfg.n_tok, cfg.H), dtype=torch.int16).pin_memory()
+    rc = B.strata_moe_roundtrip_host(ctx.h, dev, h_ids.data_ptr(), h_x.data_ptr(), h_w.data_ptr(),
+                                     h_out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    assert rc == 0
+    ref_lay = oracle.layout(inp["ids"], cfg.E)
+    ref_recv = oracle.dispatch_bf16(ref_lay["dst_row"], inp["x"])
+    ref_out = oracle.combine(ref_lay["dst_row"], ref_recv, inp["w"])
+    assert np.array_equal(h_out.numpy().view(np.uint16), ref_out)
+    assert ctx.device_status() == B.STRATA_OK
+    ctx.close()
