@@ -137,8 +137,8 @@ strata_status strata_moe_layout(strata_ctx *ctx, const int32_t *topk_ids,
  *        per token and block of 128 columns: amax = max|x|, scale = amax/448 (IEEE binary32
  *        division), q = e4m3_rne_satfinite(x / (amax == 0 ? 1 : scale)); codes and the stored
  *        scale (amax/448) go to each of the token's K rows.
- * recv (and recv_scale) must lie inside a registered region (NOT_REGISTERED otherwise), be
- * 16-byte aligned, and capacity_rows >= N (CAPACITY otherwise).  Rows whose dst_row is outside
+ * recv (and recv_scale) must lie inside a registered region (NOT_REGISTERED otherwise); x and recv
+ * must be 16-byte aligned, recv_scale 4-byte aligned; capacity_rows >= N (CAPACITY otherwise).  Rows whose dst_row is outside
  * [0, capacity_rows) are skipped and raise BAD_ROW.  One kernel launch. */
 strata_status strata_moe_dispatch(strata_ctx *ctx, const strata_moe_layout_t *layout, const void *x,
                                   void *recv, float *recv_scale, size_t capacity_rows, void *stream);

@@ -288,7 +288,8 @@ strata_status strata_moe_dispatch(strata_ctx* ctx, const strata_moe_layout_t* la
     const strata_moe_shape& s = ctx->shape;
     const bool fp8 = s.dispatch_dtype == STRATA_FP8_E4M3_B128;
     if (fp8 != (recv_scale != nullptr)) return STRATA_ERR_INVALID_ARG;
-    if (!aligned16(x) || !aligned16(recv) || (fp8 && !aligned16(recv_scale))) return STRATA_ERR_ALIGNMENT;
+    if (!aligned16(x) || !aligned16(recv)) return STRATA_ERR_ALIGNMENT;
+    if (fp8 && (reinterpret_cast<uintptr_t>(recv_scale) & 3u) != 0) return STRATA_ERR_ALIGNMENT;
     if (!ctx->ws) return STRATA_ERR_WORKSPACE;
     const size_t n_rows = (size_t)s.R * s.T * s.K;
     if (capacity_rows < n_rows) return STRATA_ERR_CAPACITY;

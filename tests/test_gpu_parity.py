@@ -101,7 +101,8 @@ def run_full_case(cfg: wl.MoEConfig, inp=None, threads=8):
     ow = u16(out_whole)
     assert np.all(ow[:GUARD] == SENTINEL16) and np.all(ow[GUARD + n_tok:] == SENTINEL16)
     if cfg.expert == "identity" and not fp8:
-        assert np.array_equal(got_out, inp["x"].reshape(n_tok, H))     # gate weights sum to 1
+        # gate weights sum to 1: out == x as values (a -0 input comes back as +0: fma(w, -0, +0) = +0)
+        assert ulp_distance(got_out, inp["x"].reshape(n_tok, H)).max() == 0
     assert ctx.device_status() == B.STRATA_OK
     ctx.close()
 
@@ -171,7 +172,8 @@ def test_prefill_full_size_sampled():
     got_out = u16(out[torch.from_numpy(toks).to(DEV)])
     assert ulp_distance(got_out, want_out).max() <= 1
     assert np.array_equal(got_out, want_out)
-    assert torch.equal(out, x2)                        # invariant at full size
+    # invariant at full size, as values (-0 == +0)
+    assert bool((out.view(torch.bfloat16) == x2.view(torch.bfloat16)).all())
     assert ctx.device_status() == B.STRATA_OK
     ctx.close()
 
