@@ -38,11 +38,13 @@ UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch at the prefill shape, from the ncu
-# captures summarised under profiles/ (None until a capture exists for that kernel).
+# dram__bytes_read.sum + dram__bytes_write.sum per launch at the prefill shape.  Captured with
+# ncu --set full on the same recipe at T=512 tokens/rank (1/8 of the tokens) and scaled by 8, since
+# traffic grows in proportion to the tokens (profiles/*_prefill_T512.md); None = no capture yet.
 NCU_TRAFFIC_BYTES = {
-    "dispatch_bf16_kernel": None,
-    "combine_kernel": None,
+    "dispatch_bf16_kernel": 8 * (117_928_192 + 879_901_696),
+    "dispatch_fp8_kernel": None,
+    "combine_kernel": 8 * (940_062_208 + 98_784_768),
 }
 
 
@@ -283,7 +285,11 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
         if world > 1:
             dist.barrier()
 
-    cfg = wl.CONFIGS["prefill"]
+    cfg = wl.CONFIGS[args.workload]
+    if args.tokens_per_rank:
+        cfg = wl.shrink(cfg, T=args.tokens_per_rank)
+    if cfg.dispatch_dtype != wl.BF16:
+        args.no_e2e = True            # the host round trip is defined for bf16 dispatch only
     case = DeviceCase(cfg, local_rank)
     host_inp = case.inp
     disp_bytes, comb_bytes = cfg.dispatch_bytes(), cfg.combine_bytes()
@@ -377,8 +383,10 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
         return
 
     peak, peak_src = measured_peak()
+    traffic_ok = args.workload == "prefill" and not args.tokens_per_rank   # the captures are scaled to this shape
+    disp_name = "dispatch_bf16_kernel" if cfg.dispatch_dtype == wl.BF16 else "dispatch_fp8_kernel"
     kernels = {
-        "dispatch_bf16_kernel": {"bytes": disp_bytes, "ms": disp_ms},
+        disp_name: {"bytes": disp_bytes, "ms": disp_ms},
         "combine_kernel": {"bytes": comb_bytes, "ms": comb_ms},
     }
     for k, v in kernels.items():
@@ -389,11 +397,13 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
     roofline = {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["achieved"], "peak": peak,
                 "peak_source": f"{peak_src} (MEASURED_PEAKS.json hbm_gbs)" if peak_src == "measured"
                 else "fallback (recipe figure)",
-                "unit": "GB/s", "frac": kernels[dom]["frac"], "traffic": NCU_TRAFFIC_BYTES.get(dom),
+                "unit": "GB/s", "frac": kernels[dom]["frac"],
+                "traffic": NCU_TRAFFIC_BYTES.get(dom) if traffic_ok else None,
                 "algorithmic_bytes_per_launch": kernels[dom]["bytes"],
                 "kernels": {k: {"achieved": round(v["achieved"], 1), "frac": round(v["frac"], 4),
                                 "frac_of_nominal_8TBs": round(v["frac_of_nominal_8TBs"], 4),
-                                "avg_ms": round(v["ms"], 4), "traffic": NCU_TRAFFIC_BYTES.get(k)}
+                                "avg_ms": round(v["ms"], 4),
+                                "traffic": NCU_TRAFFIC_BYTES.get(k) if traffic_ok else None}
                             for k, v in kernels.items()},
                 "layout_avg_ms": round(lay_ms, 4)}
 
@@ -429,13 +439,15 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": "prefill: R=16 emulated ranks, T=4096 tokens/rank, H=7168 bf16, E=256, K=8 "
-                               "uniform distinct experts, softmax gates, identity experts (combine reads recv)",
+        "config": {"workload": f"{cfg.name}: R={cfg.R} emulated ranks, T={cfg.T} tokens/rank, H={cfg.H} bf16, "
+                               f"E={cfg.E}, K={cfg.K} {cfg.routing} distinct experts, softmax gates, "
+                               + ("identity experts (combine reads recv)" if cfg.dispatch_dtype == wl.BF16
+                                  else "e4m3 dispatch, bf16 expert outputs"),
                    "step": "strata_moe_layout + strata_moe_dispatch + strata_moe_combine",
                    "bytes_per_step": step_bytes, "l2": "inputs larger than L2 (8.4 GB working set), no flush",
                    "parallelism": "replicas only" if world > 1 else "1 GPU, 16 ranks emulated in HBM"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(n1 - n0), "roofline": roofline,
-        "pct_of_8TBs": {"dispatch": round(100 * kernels["dispatch_bf16_kernel"]["frac_of_nominal_8TBs"], 2),
+        "pct_of_8TBs": {"dispatch": round(100 * kernels[disp_name]["frac_of_nominal_8TBs"], 2),
                         "combine": round(100 * kernels["combine_kernel"]["frac_of_nominal_8TBs"], 2)},
         "other_configs": other, "cpu_baseline": cpu,
     }
@@ -453,8 +465,16 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-other", action="store_true")
+    ap.add_argument("--workload", default="prefill", choices=wl.CONFIG_ORDER,
+                    help="configuration to step through (the bench line is quoted on the default)")
+    ap.add_argument("--tokens-per-rank", type=int, default=0, help="shrink T (profiling captures only)")
+    ap.add_argument("--profile", action="store_true",
+                    help="for runs under a profiler: no e2e/cpu/other legs, warm-up not clamped")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "strata" else args.warmup
+    if args.profile:
+        args.no_e2e = args.no_cpu = args.no_other = True
+    elif args.impl == "strata":
+        args.warmup = max(args.warmup, 3)
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
