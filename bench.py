@@ -194,6 +194,26 @@ def run_reference(args, rank: int):
 
 
 # ---------------------------------------------------------------------------------------
+# replicas: the only cross-rank logic (no collective touches the data path)
+# ---------------------------------------------------------------------------------------
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The slowest rank's time: what the whole job took."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(bytes_per_replica_step: int, ms_per_step: float, world: int) -> float:
+    """Aggregate throughput of `world` independent replicas that all finish within ms_per_step."""
+    return world * bytes_per_replica_step / (ms_per_step * 1e-3) / 1e9
+
+
+# ---------------------------------------------------------------------------------------
 # GPU arm
 # ---------------------------------------------------------------------------------------
 
@@ -324,12 +344,9 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
     elapsed_ms = ev[0][0].elapsed_time(ev[K - 1][3])
     clocks = sampler.summary(t0, t1)
 
-    if world > 1:
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = max_over_ranks(elapsed_ms, world, "cuda")
     ms_per_step = elapsed_ms / K
-    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_gbs(step_bytes, ms_per_step, world)
 
     lay_ms = float(np.mean([ev[i][0].elapsed_time(ev[i][1]) for i in range(K)]))
     disp_ms = float(np.mean([ev[i][1].elapsed_time(ev[i][2]) for i in range(K)]))
@@ -365,14 +382,10 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
         torch.cuda.synchronize()
         barrier()
         e2e_ms = a.elapsed_time(b)
-        if world > 1:
-            t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        e2e_ms /= e2e_steps
+        e2e_ms = max_over_ranks(e2e_ms, world, "cuda") / e2e_steps
         h2d = h_ids.numel() * 4 + h_x.numel() * 2 + h_w.numel() * 4
         d2h = h_out.numel() * 2
-        e2e = {"value": world * step_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
+        e2e = {"value": whole_job_gbs(step_bytes, e2e_ms, world), "unit": UNIT, "ms_per_step": e2e_ms,
                "steps": e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "api": "strata_moe_roundtrip_host (pinned host buffers, copies in the timed region)"}
 
