@@ -130,6 +130,32 @@ strata_status strata_pool_reset(strata_ctx *ctx, uint64_t region_id);
 strata_status strata_moe_layout(strata_ctx *ctx, const int32_t *topk_ids,
                                 const strata_moe_layout_t *layout, void *stream);
 
+/* Routing layout without any allocation or workspace (the paper has no counterpart: this entry
+ * exists for this library's callers only).  It is for callers that cannot hand over a workspace
+ * because they cannot allocate device memory where they run: a serving process whose framework
+ * pool already owns all of the GPU's memory, a plug-in hook that must avoid the device-wide
+ * synchronisation cudaMalloc and cudaFree bring, or a binding with no device allocator of its own.
+ * Same inputs, outputs, ordering and error rules as strata_moe_layout, computed by the same kernels;
+ * the kernels' scratch lives in a fixed 2 MiB array inside the library (each GPU that loads the
+ * library holds it until the process exits) instead of a caller workspace.
+ *  - Runs on the CURRENT CUDA device; no context is needed.  `shape->H` and `dispatch_dtype` are ignored.
+ *  - Limit: 256 + ceil(T*K/1024) * R * E * 4 bytes must fit in 2 MiB (all five benchmark shapes do;
+ *    the prefill shape needs 0.5 MiB).  Larger shapes return STRATA_ERR_CAPACITY and launch nothing:
+ *    use strata_moe_layout with a workspace for those.
+ *  - device_status: device pointer to one int32 owned by the caller, zeroed by the caller; receives
+ *    STRATA_ERR_BAD_EXPERT_ID if an id outside [0,E) was skipped.  May be NULL (skipped items are then
+ *    only visible as dst_row = -1).
+ *  - The first call on each device resolves the array's device address and sets one kernel
+ *    attribute (no allocation).  Make that first call before any stream capture begins.
+ *  - All calls on a device share the one array, which keeps the previous call's contents; the
+ *    entry clears the words that must start at zero, in stream order.  Two calls whose kernels can
+ *    overlap on the GPU (different streams, no dependency between them) race on the array and give
+ *    wrong results: serialise them.
+ *  - Calls no cudaMalloc, cudaFree or any other allocating routine. */
+strata_status strata_moe_layout_noalloc(const strata_moe_shape *shape, const int32_t *topk_ids,
+                                        const strata_moe_layout_t *layout, int32_t *device_status,
+                                        void *stream);
+
 /* Dispatch (paper Sec. 6.2 / 7.1).  x: device bf16 [R,T,H].
  * BF16:  recv is device bf16 [capacity_rows, H]; recv[dst_row[i], :] = x[n(i), :] bit for bit;
  *        recv_scale must be NULL.

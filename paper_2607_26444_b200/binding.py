@@ -35,7 +35,7 @@ EXPORTS = [
     "strata_ctx_set_workspace", "strata_ctx_launch_count", "strata_pool_register", "strata_pool_is_ready",
     "strata_pool_unregister", "strata_pool_carve", "strata_pool_reset", "strata_moe_layout",
     "strata_moe_dispatch", "strata_moe_combine", "strata_moe_recv_view", "strata_device_status",
-    "strata_moe_roundtrip_host",
+    "strata_moe_roundtrip_host", "strata_moe_layout_noalloc",
 ]
 
 
@@ -95,6 +95,7 @@ def lib() -> ctypes.CDLL:
         "strata_moe_recv_view": [vp, vp, i32, vp, P(vp), P(ctypes.c_int64)],
         "strata_device_status": [vp, vp, P(i32)],
         "strata_moe_roundtrip_host": [vp, P(strata_moe_device_buffers), vp, vp, vp, vp, vp],
+        "strata_moe_layout_noalloc": [P(strata_moe_shape), vp, P(strata_moe_layout_t), vp, vp],
     }
     for name, args in sigs.items():
         fn = getattr(L, name)
@@ -191,6 +192,14 @@ def strata_device_status(ctx, stream: int) -> Tuple[int, int]:
 def strata_moe_roundtrip_host(ctx, dev: strata_moe_device_buffers, h_ids: int, h_x: int, h_w: int, h_out: int,
                               stream: int) -> int:
     return lib().strata_moe_roundtrip_host(ctx, ctypes.byref(dev), h_ids, h_x, h_w, h_out, stream)
+
+
+def strata_moe_layout_noalloc(shape: strata_moe_shape, topk_ids: int, layout: strata_moe_layout_t,
+                              device_status: Optional[int], stream: int) -> int:
+    """Routing layout on the current device with the library's built-in scratch: no context, no
+    workspace, nothing allocated.  For callers that cannot allocate device memory (see the header)."""
+    return lib().strata_moe_layout_noalloc(ctypes.byref(shape), topk_ids, ctypes.byref(layout), device_status,
+                                           stream)
 
 
 # ---- convenience wrapper over torch tensors (memory + streams only) ---------

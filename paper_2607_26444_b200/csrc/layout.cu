@@ -11,6 +11,8 @@
 //   2. layout_rank_kernel: one CTA per tile again; rank of an item inside its tile =
 //      (items with the same id in earlier warps) + (same id in earlier lanes), both
 //      from match.any masks, so the order is exact and no atomics decide a row.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace strata {
@@ -249,3 +251,108 @@ cudaError_t launch_layout(const strata_moe_shape& s, const int32_t* ids, const s
 }
 
 }  // namespace strata
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free routing layout.
+//
+// Some callers have no way to give this library a workspace: a serving process whose framework pool
+// has already claimed all device memory (a fresh cudaMalloc would fail or fragment it), a plug-in
+// hook that must not cause the device-wide synchronisation that cudaMalloc/cudaFree imply, or a thin
+// language binding that owns no device allocator at all.  For them the scratch of the layout kernels
+// (status word, ticket, per-tile histograms) lives in the fixed array below instead of a workspace.
+// Every GPU that loads this library holds the array (2 MiB) until the process exits.
+// ---------------------------------------------------------------------------------------------
+namespace strata {
+namespace {
+
+constexpr size_t kStaticScratchBytes = 2u << 20;       // header + int32[n_tiles, E]
+constexpr int kMaxDevices = 64;
+
+// In host code this name is only a handle for cudaGetSymbolAddress, never an address to pass on.
+static __device__ __align__(256) unsigned char g_layout_scratch[kStaticScratchBytes];
+
+std::mutex g_scratch_mu;
+int* g_scratch_ptr[kMaxDevices];                       // device address of the array, per device
+bool g_scratch_ready[kMaxDevices];
+
+// One-time set-up for the current device: resolve the array's device address and allow the rank
+// kernel its shared-memory table.  Neither call allocates.
+strata_status static_scratch_for_current_device(int** out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        return STRATA_ERR_CUDA;
+    }
+    if (dev < 0 || dev >= kMaxDevices) return STRATA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(g_scratch_mu);
+    if (!g_scratch_ready[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_layout_scratch) != cudaSuccess || ptr == nullptr) {
+            cudaGetLastError();
+            return STRATA_ERR_CUDA;
+        }
+        if (cudaFuncSetAttribute(layout_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 32 * kMaxExperts * (int)sizeof(int)) != cudaSuccess) {
+            cudaGetLastError();
+            return STRATA_ERR_CUDA;
+        }
+        g_scratch_ptr[dev] = static_cast<int*>(ptr);
+        g_scratch_ready[dev] = true;
+    }
+    *out = g_scratch_ptr[dev];
+    return STRATA_OK;
+}
+
+}  // namespace
+}  // namespace strata
+
+extern "C" strata_status strata_moe_layout_noalloc(const strata_moe_shape* shape, const int32_t* topk_ids,
+                                                   const strata_moe_layout_t* layout, int32_t* device_status,
+                                                   void* stream)
+{
+    using namespace strata;
+    if (!shape || !topk_ids || !layout) return STRATA_ERR_INVALID_ARG;
+    if (!layout->expert_count || !layout->expert_offset || !layout->rank_count || !layout->rank_offset ||
+        !layout->dst_row)
+        return STRATA_ERR_INVALID_ARG;
+    const strata_moe_shape& s = *shape;
+    if (s.R <= 0 || s.T <= 0 || s.E <= 0 || s.K <= 0) return STRATA_ERR_SHAPE;
+    if (s.E % s.R != 0 || s.E > kMaxExperts || s.K > kMaxTopK) return STRATA_ERR_SHAPE;
+    if ((long long)s.R * s.T * s.K >= (1ll << 31)) return STRATA_ERR_SHAPE;
+    const LayoutGeom g = layout_geom(s);
+    const size_t need = (size_t)kWsHeaderBytes + (size_t)g.n_tiles * s.E * sizeof(int);
+    if (need > kStaticScratchBytes) return STRATA_ERR_CAPACITY;     // beyond the fixed array: use a workspace
+
+    int* scratch = nullptr;
+    strata_status rc = static_scratch_for_current_device(&scratch);
+    if (rc != STRATA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // The array keeps whatever the previous call left: status word and ticket must start at zero.
+    if (cudaMemsetAsync(scratch, 0, kWsHeaderBytes, st) != cudaSuccess) {
+        cudaGetLastError();
+        return STRATA_ERR_CUDA;
+    }
+    LayoutParams p;
+    p.ids = topk_ids;
+    p.expert_count = layout->expert_count;
+    p.expert_offset = layout->expert_offset;
+    p.rank_count = layout->rank_count;
+    p.rank_offset = layout->rank_offset;
+    p.src_expert_count = layout->src_expert_count;
+    p.dst_row = layout->dst_row;
+    p.src_of_row = layout->src_of_row;
+    p.status = device_status ? device_status : scratch;
+    p.ticket = scratch + 1;
+    p.tile_cnt = scratch + kWsHeaderBytes / sizeof(int);
+    p.R = s.R;
+    p.E = s.E;
+    p.e_loc = s.E / s.R;
+    p.items_per_rank = g.items_per_rank;
+    p.tiles_per_rank = g.tiles_per_rank;
+    p.n_tiles = g.n_tiles;
+    layout_count_scan_kernel<<<g.n_tiles, kLayoutTile, count_scan_smem(s.E), st>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return STRATA_ERR_CUDA;
+    layout_rank_kernel<<<g.n_tiles, kLayoutTile, (size_t)32 * s.E * sizeof(int), st>>>(p);
+    return cudaGetLastError() == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
+}
