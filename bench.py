@@ -279,6 +279,9 @@ def per_call_us(case: DeviceCase, iters: int = 30, warmup: int = 3):
             fn()
         torch.cuda.synchronize()
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+        # Hold the stream for ~5 ms so that every call below is already queued when the first one
+        # runs: the events then bracket device time, not the host's enqueue pace.
+        torch.cuda._sleep(10_000_000)
         ev[0].record()
         for i in range(iters):
             fn()

@@ -126,7 +126,7 @@ strata_status strata_pool_reset(strata_ctx *ctx, uint64_t region_id);
  * then source rank, then token, then slot, packed without padding.
  * Duplicate ids inside a token are legal.  An id outside [0,E) is skipped
  * (dst_row = -1, not counted) and raises BAD_EXPERT_ID on the device status.
- * Needs a workspace.  Two kernel launches. */
+ * Needs a workspace.  One kernel launch for up to 4,096 items, two beyond. */
 strata_status strata_moe_layout(strata_ctx *ctx, const int32_t *topk_ids,
                                 const strata_moe_layout_t *layout, void *stream);
 
@@ -139,8 +139,8 @@ strata_status strata_moe_layout(strata_ctx *ctx, const int32_t *topk_ids,
  * the kernels' scratch lives in a fixed 2 MiB array inside the library (each GPU that loads the
  * library holds it until the process exits) instead of a caller workspace.
  *  - Runs on the CURRENT CUDA device; no context is needed.  `shape->H` and `dispatch_dtype` are ignored.
- *  - Limit: 256 + ceil(T*K/1024) * R * E * 4 bytes must fit in 2 MiB (all five benchmark shapes do;
- *    the prefill shape needs 0.5 MiB).  Larger shapes return STRATA_ERR_CAPACITY and launch nothing:
+ *  - Limit: 256 + ceil(T*K/4096) * R * E * 4 bytes must fit in 2 MiB (all five benchmark shapes do;
+ *    the prefill shape needs 0.13 MiB).  Larger shapes return STRATA_ERR_CAPACITY and launch nothing:
  *    use strata_moe_layout with a workspace for those.
  *  - device_status: device pointer to one int32 owned by the caller, zeroed by the caller; receives
  *    STRATA_ERR_BAD_EXPERT_ID if an id outside [0,E) was skipped.  May be NULL (skipped items are then

@@ -3,8 +3,9 @@
 //   out[n,c] = bf16_rne( fma(w[n,K-1], y[row(n,K-1),c], ... fma(w[n,0], y[row(n,0),c], +0) ) )
 // with binary32 fused multiply-adds in slot order 0..K-1.
 //
-// Work split: persistent CTAs take tokens round-robin; every token costs K row reads and one
-// row write, so the split is even whatever the expert popularity is.  A thread owns one
+// Work split: persistent CTAs take tokens round-robin, the grid sized so that every CTA gets the
+// same number of tokens (+-1); every token costs K row reads and one row write, so the split is
+// even whatever the expert popularity is.  A thread owns one
 // 16-byte column vector at a time: it issues the K independent 16-byte streaming loads first
 // (K requests in flight per thread), then runs the FMA chain in registers and writes 16 bytes.
 // The accumulation lives in registers; no atomics and no shared-memory staging are needed
@@ -139,7 +140,7 @@ cudaError_t launch_k(const CombineParams& p, int n_sm, cudaStream_t st)
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, combine_kernel<KT>, kCombineThreads, 0);
     if (err != cudaSuccess) return err;
     if (per_sm < 1) per_sm = 1;
-    const long long grid = min((long long)n_sm * per_sm, p.n_tok);
+    const long long grid = balanced_grid(p.n_tok, (long long)n_sm * per_sm);
     combine_kernel<KT><<<(unsigned)grid, kCombineThreads, 0, st>>>(p);
     return cudaGetLastError();
 }

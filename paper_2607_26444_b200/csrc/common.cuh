@@ -13,7 +13,9 @@ namespace strata {
 // word 1: ticket of the layout kernel (returns to 0 after every call)
 // bytes [256, ...): per-tile, per-expert counts, int32 [n_tiles, E]
 constexpr int kWsHeaderBytes = 256;
-constexpr int kLayoutTile = 1024;      // items per tile = threads per layout CTA
+constexpr int kLayoutThreads = 1024;   // threads per layout CTA
+constexpr int kItemsPerThread = 4;
+constexpr int kLayoutTile = kLayoutThreads * kItemsPerThread;   // items per tile
 constexpr int kMaxExperts = 1024;
 constexpr int kMaxTopK = 32;
 
@@ -30,6 +32,16 @@ inline LayoutGeom layout_geom(const strata_moe_shape& s)
     g.tiles_per_rank = (g.items_per_rank + kLayoutTile - 1) / kLayoutTile;
     g.n_tiles = s.R * g.tiles_per_rank;
     return g;
+}
+
+// Largest grid <= max_ctas in which round-robin dealing gives every CTA the same number of
+// units (the last CTA may get fewer): no CTA is left with one extra unit at the tail.
+inline long long balanced_grid(long long units, long long max_ctas)
+{
+    if (units <= 0) return 1;
+    if (max_ctas < 1) max_ctas = 1;
+    const long long per = (units + max_ctas - 1) / max_ctas;
+    return (units + per - 1) / per;
 }
 
 // ---- launchers (defined next to their kernels) -----------------------------

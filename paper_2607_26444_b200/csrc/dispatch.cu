@@ -2,8 +2,11 @@
 // the layout assigned, straight into the caller's (registered) receive buffer.
 //
 // Work split: a unit is one token (or one column chunk of a token when a row is larger than
-// a stage).  Units are dealt round-robin to a persistent grid, so every CTA moves the same
-// number of bytes whatever the expert popularity is: 1 row read + K row writes per unit.
+// a stage).  Units are dealt round-robin to a persistent grid whose size is chosen so that every
+// CTA gets the same number of units (+-1): every CTA moves the same bytes whatever the expert
+// popularity is, 1 row read + K row writes per unit.  Round-robin (rather than one contiguous
+// span per CTA) keeps the CTAs that run at the same time on neighbouring rows, which measured
+// 1..2 % faster for dispatch and far faster for combine.
 //
 // bf16: each CTA is a single warp that runs the SM's bulk-copy engine as a small DMA program
 //       (the on-SM counterpart of the paper's device-issued SDMA descriptors, Sec. 6.3):
@@ -80,8 +83,13 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
         const uint32_t bytes = min(p.chunk_cols, (uint32_t)p.H - col0) * 2u;
         const int s = (int)(j % kBf16Stages);
         mbar_expect_tx(&bars[s], bytes);
+#ifdef STRATA_EXP_XMOD
+        bulk_g2s(smem + (size_t)s * stage_bytes, p.x + (size_t)(tok % STRATA_EXP_XMOD) * row_bytes + (size_t)col0 * 2u, bytes, &bars[s],
+                 pol);
+#else
         bulk_g2s(smem + (size_t)s * stage_bytes, p.x + (size_t)tok * row_bytes + (size_t)col0 * 2u, bytes, &bars[s],
                  pol);
+#endif
     };
 
     if (lane == 0)
@@ -97,7 +105,11 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
         const int s = (int)(j % kBf16Stages);
         const uint32_t parity = (uint32_t)((j / kBf16Stages) & 1);
 
+#ifdef STRATA_EXP_SEQ
+        const int my_row = (lane < p.K) ? (int)(tok * p.K + lane) : -1;
+#else
         const int my_row = (lane < p.K) ? p.dst_row[tok * p.K + lane] : -1;
+#endif
         const bool row_ok = (lane >= p.K) || (my_row >= 0 && my_row < p.capacity_rows);
         if (!row_ok) report_status(p.status, STRATA_ERR_BAD_ROW);
 
@@ -302,7 +314,7 @@ cudaError_t launch_dispatch_bf16(const strata_moe_shape& s, const int32_t* dst_r
     if (err != cudaSuccess) return err;
     if (per_sm < 1) per_sm = 1;
     if (STRATA_BF16_MAX_CTAS_PER_SM > 0) per_sm = min(per_sm, STRATA_BF16_MAX_CTAS_PER_SM);
-    const long long grid = min((long long)n_sm * per_sm, p.n_units);
+    const long long grid = balanced_grid(p.n_units, (long long)n_sm * per_sm);
     dispatch_bf16_kernel<<<(unsigned)grid, 32, smem, st>>>(p);
     return cudaGetLastError();
 }
@@ -327,7 +339,7 @@ cudaError_t launch_dispatch_fp8(const strata_moe_shape& s, const int32_t* dst_ro
     cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dispatch_fp8_kernel, kFp8Threads, smem);
     if (err != cudaSuccess) return err;
     if (per_sm < 1) per_sm = 1;
-    const long long grid = min((long long)n_sm * per_sm, p.n_units);
+    const long long grid = balanced_grid(p.n_units, (long long)n_sm * per_sm);
     dispatch_fp8_kernel<<<(unsigned)grid, kFp8Threads, smem, st>>>(p);
     return cudaGetLastError();
 }

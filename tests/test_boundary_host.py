@@ -59,10 +59,10 @@ def test_bad_shapes_are_rejected(kw):
 
 def test_workspace_size():
     rc, n = B.strata_moe_workspace_bytes(shape())
-    # 4 ranks x ceil(128*2/1024)=1 tile, 16 experts, 256-byte header, rounded to 256
+    # 4 ranks x ceil(128*2/4096)=1 tile, 16 experts, 256-byte header, rounded to 256
     assert rc == 0 and n == 512
     rc, n = B.strata_moe_workspace_bytes(shape(R=16, T=4096, H=7168, E=256, K=8))
-    assert rc == 0 and n == 256 + 16 * 32 * 256 * 4
+    assert rc == 0 and n == 256 + 16 * 8 * 256 * 4
 
 
 @pytest.fixture

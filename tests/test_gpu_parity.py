@@ -192,6 +192,9 @@ RAGGED = [
     dict(R=2, T=129, H=136, E=12, K=9),
     dict(R=5, T=50, H=4096, E=20, K=6),
     dict(R=4, T=100, H=2048, E=16, K=4),
+    dict(R=4, T=256, H=64, E=32, K=4),               # 4,096 items: the largest single-CTA layout
+    dict(R=4, T=257, H=64, E=32, K=4),               # just above it: tiled layout
+    dict(R=64, T=3, H=64, E=64, K=7),                # warps straddle several source ranks
 ]
 
 
@@ -318,7 +321,7 @@ def test_host_errors_on_device_context():
     assert ei.value.code == B.STRATA_ERR_ALIGNMENT
     ctx.dispatch(lay, x_d, recv)
     assert ctx.device_status() == B.STRATA_OK
-    assert ctx.launch_count() == 3                                 # 2 (layout) + 1 (dispatch); failures launched nothing
+    assert ctx.launch_count() == 2                                 # 1 (small-batch layout) + 1 (dispatch); failures launched nothing
     ctx.close()
 
 

@@ -26,8 +26,8 @@ def test_shapes_beyond_the_built_in_scratch_are_refused():
     """2 MiB holds 256 + n_tiles*E*4 bytes; anything larger is refused before any CUDA call."""
     strata_build.build()
     lay = B.strata_moe_layout_t(16, 32, 48, 64, None, 80, None)       # never dereferenced
-    fits = B.strata_moe_shape(16, 4096, 7168, 256, 8, 0)               # prefill: 512 tiles * 256 experts
-    too_big = B.strata_moe_shape(64, 4096, 7168, 1024, 8, 0)           # 2048 tiles * 1024 experts = 8 MiB
+    fits = B.strata_moe_shape(16, 4096, 7168, 256, 8, 0)               # prefill: 128 tiles * 256 experts
+    too_big = B.strata_moe_shape(64, 16384, 7168, 1024, 8, 0)          # 2048 tiles * 1024 experts = 8 MiB
     assert B.strata_moe_layout_noalloc(too_big, 16, lay, None, None) == B.STRATA_ERR_CAPACITY
     assert "capacity" in B.strata_status_string(B.STRATA_ERR_CAPACITY)
     assert B.strata_moe_layout_noalloc(B.strata_moe_shape(3, 8, 64, 8, 2, 0), 16, lay, None, None) \
@@ -43,7 +43,7 @@ def test_noalloc_layout_matches_workspace_layout_twice_in_a_row():
     dev = "cuda:0"
     torch.cuda.set_device(0)
     stream = torch.cuda.current_stream().cuda_stream
-    cases = [wl.CONFIGS["skew"],                                                   # 128 tiles, hot expert
+    cases = [wl.CONFIGS["skew"],                                                   # 32 tiles, hot expert
              wl.shrink(wl.CONFIGS["decode"], R=4, T=300, E=64, K=5, seed=31)]       # ragged tiles, smaller E
     for cfg in cases:
         ids = torch.from_numpy(wl.gen_topk_ids(cfg)).to(dev)
