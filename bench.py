@@ -274,7 +274,12 @@ def per_call_us(case: DeviceCase, iters: int = 30, warmup: int = 3):
     """Median microseconds per call of each entry point (events on the calls' stream)."""
     torch = case.torch
     out = {}
-    for name, fn in (("layout", case.layout), ("dispatch", case.dispatch), ("combine", case.combine)):
+    def layout_dispatch():
+        case.layout()
+        case.dispatch()
+
+    for name, fn in (("layout", case.layout), ("dispatch", case.dispatch), ("combine", case.combine),
+                     ("layout+dispatch", layout_dispatch), ("step", case.step)):
         for _ in range(warmup):
             fn()
         torch.cuda.synchronize()
@@ -289,6 +294,27 @@ def per_call_us(case: DeviceCase, iters: int = 30, warmup: int = 3):
         torch.cuda.synchronize()
         ts = sorted(ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(iters))
         out[name] = {"median_us": ts[len(ts) // 2], "min_us": ts[0], "p95_us": ts[int(0.95 * (len(ts) - 1))]}
+    return out
+
+
+def cta_finish_spread(case: DeviceCase):
+    """Per-CTA probes (global timer at CTA start/end): relative gap between the first and the last
+    CTA to finish, (max_end - min_end) / (max_end - min_start), for dispatch and for combine."""
+    torch = case.torch
+    tr = case.ctx.trace(8192)
+    out = {}
+    for name, fn in (("dispatch", case.dispatch), ("combine", case.combine)):
+        vals = []
+        for _ in range(5):
+            tr.zero_()
+            fn()
+            torch.cuda.synchronize()
+            rec = tr.cpu().numpy()
+            used = rec[rec[:, 0] != 0]
+            total = float(used[:, 1].max() - used[:, 0].min())
+            vals.append(float(used[:, 1].max() - used[:, 1].min()) / total)
+        out[name] = round(float(np.median(vals)), 4)
+    case.ctx.trace_off()
     return out
 
 
@@ -438,9 +464,25 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
                 "layout_us": round(us["layout"]["median_us"], 2),
                 "dispatch_us": round(us["dispatch"]["median_us"], 2),
                 "combine_us": round(us["combine"]["median_us"], 2),
+                "layout+dispatch_us": round(us["layout+dispatch"]["median_us"], 2),
+                "step_us": round(us["step"]["median_us"], 2),
                 "dispatch_GBs": round(db / us["dispatch"]["median_us"] / 1e3, 1),
                 "combine_GBs": round(cb / us["combine"]["median_us"] / 1e3, 1),
             }
+            if name == "skew":
+                # load balance under Zipf routing: per-CTA finish-time spread, and the same shape with
+                # uniform routing for comparison
+                other[name]["cta_finish_spread"] = cta_finish_spread(dc)
+                del dc
+                torch.cuda.empty_cache()
+                uc = DeviceCase(wl.shrink(c, routing="uniform"), local_rank)
+                uu = per_call_us(uc)
+                other["skew_shape_uniform_routing"] = {
+                    "dispatch_GBs": round(db / uu["dispatch"]["median_us"] / 1e3, 1),
+                    "combine_GBs": round(cb / uu["combine"]["median_us"] / 1e3, 1),
+                    "cta_finish_spread": cta_finish_spread(uc),
+                }
+                dc = uc
             del dc
             torch.cuda.empty_cache()
 

@@ -35,7 +35,7 @@ EXPORTS = [
     "strata_ctx_set_workspace", "strata_ctx_launch_count", "strata_pool_register", "strata_pool_is_ready",
     "strata_pool_unregister", "strata_pool_carve", "strata_pool_reset", "strata_moe_layout",
     "strata_moe_dispatch", "strata_moe_combine", "strata_moe_recv_view", "strata_device_status",
-    "strata_moe_roundtrip_host", "strata_moe_layout_noalloc",
+    "strata_moe_roundtrip_host", "strata_moe_layout_noalloc", "strata_ctx_set_trace",
 ]
 
 
@@ -96,6 +96,7 @@ def lib() -> ctypes.CDLL:
         "strata_device_status": [vp, vp, P(i32)],
         "strata_moe_roundtrip_host": [vp, P(strata_moe_device_buffers), vp, vp, vp, vp, vp],
         "strata_moe_layout_noalloc": [P(strata_moe_shape), vp, P(strata_moe_layout_t), vp, vp],
+        "strata_ctx_set_trace": [vp, vp, sz],
     }
     for name, args in sigs.items():
         fn = getattr(L, name)
@@ -129,6 +130,10 @@ def strata_moe_workspace_bytes(shape: strata_moe_shape) -> Tuple[int, int]:
 
 def strata_ctx_set_workspace(ctx, dptr: int, nbytes: int) -> int:
     return lib().strata_ctx_set_workspace(ctx, dptr, nbytes)
+
+
+def strata_ctx_set_trace(ctx, dptr: Optional[int], capacity_ctas: int) -> int:
+    return lib().strata_ctx_set_trace(ctx, dptr, capacity_ctas)
 
 
 def strata_ctx_launch_count(ctx) -> Tuple[int, int]:
@@ -309,6 +314,18 @@ class MoEContext:
     def combine(self, layout: Layout, y, w, out) -> None:
         _check(strata_moe_combine(self.h, layout.c, y.data_ptr(), y.shape[0], w.data_ptr(), out.data_ptr(),
                                   self._stream()), "strata_moe_combine")
+
+    def trace(self, capacity_ctas: int = 4096):
+        """Turns per-CTA probes on; returns the uint64 tensor [capacity, 2] = (start_ns, end_ns)."""
+        import torch
+        t = torch.zeros((capacity_ctas, 2), dtype=torch.int64, device=self.device)
+        _check(strata_ctx_set_trace(self.h, t.data_ptr(), capacity_ctas), "strata_ctx_set_trace")
+        self._trace = t
+        return t
+
+    def trace_off(self) -> None:
+        _check(strata_ctx_set_trace(self.h, None, 0), "strata_ctx_set_trace")
+        self._trace = None
 
     def device_status(self) -> int:
         rc, st = strata_device_status(self.h, self._stream())

@@ -26,6 +26,8 @@ struct strata_ctx {
     size_t ws_bytes;
     uint64_t next_region;
     uint64_t launches;
+    uint64_t n_dispatch, n_combine;      // launches so far: their parity selects the work-claim counter
+    strata::TraceBuf trace;
     std::vector<strata_region> regions;
     std::mutex mu;
 };
@@ -52,6 +54,22 @@ size_t workspace_bytes(const strata_moe_shape& s)
     const LayoutGeom g = layout_geom(s);
     size_t b = (size_t)kWsHeaderBytes + (size_t)g.n_tiles * s.E * sizeof(int);
     return (b + 255) & ~(size_t)255;
+}
+
+// Counter pair of a kernel type; consecutive successful launches alternate (see WorkQueue).  The
+// parity only advances when a launch succeeded, so the counter a launch claims from is always the
+// one that the launch before it has zeroed.
+WorkQueue dispatch_queue(const strata_ctx* c)
+{
+    unsigned int* w = reinterpret_cast<unsigned int*>(c->ws) + 2;
+    const unsigned int k = (unsigned int)(c->n_dispatch & 1);
+    return WorkQueue{w + k, w + (k ^ 1)};
+}
+WorkQueue combine_queue(const strata_ctx* c)
+{
+    unsigned int* w = reinterpret_cast<unsigned int*>(c->ws) + 4;
+    const unsigned int k = (unsigned int)(c->n_combine & 1);
+    return WorkQueue{w + k, w + (k ^ 1)};
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -141,6 +159,8 @@ strata_status strata_ctx_create(strata_ctx** out, const strata_moe_shape* shape,
     c->ws_bytes = 0;
     c->next_region = 1;
     c->launches = 0;
+    c->n_dispatch = c->n_combine = 0;
+    c->trace = strata::TraceBuf{nullptr, 0};
     *out = c;
     return STRATA_OK;
 }
@@ -189,6 +209,17 @@ strata_status strata_ctx_launch_count(strata_ctx* ctx, uint64_t* count)
     if (!ctx || !count) return STRATA_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lk(ctx->mu);
     *count = ctx->launches;
+    return STRATA_OK;
+}
+
+strata_status strata_ctx_set_trace(strata_ctx* ctx, uint64_t* dptr, size_t capacity_ctas)
+{
+    if (!ctx) return STRATA_ERR_INVALID_ARG;
+    if (dptr && (reinterpret_cast<uintptr_t>(dptr) & 7u) != 0) return STRATA_ERR_ALIGNMENT;
+    if (dptr && (capacity_ctas == 0 || capacity_ctas > (size_t)1 << 24)) return STRATA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(ctx->mu);
+    ctx->trace.slots = reinterpret_cast<unsigned long long*>(dptr);
+    ctx->trace.capacity = dptr ? (int)capacity_ctas : 0;
     return STRATA_OK;
 }
 
@@ -304,13 +335,14 @@ strata_status strata_moe_dispatch(strata_ctx* ctx, const strata_moe_layout_t* la
     DeviceGuard g(ctx->device);
     if (!g.ok) return STRATA_ERR_CUDA;
     cudaError_t err =
-        fp8 ? launch_dispatch_fp8(s, layout->dst_row, x, recv, recv_scale, capacity_rows, ctx->ws, ctx->n_sm,
-                                  static_cast<cudaStream_t>(stream))
-            : launch_dispatch_bf16(s, layout->dst_row, x, recv, capacity_rows, ctx->ws, ctx->n_sm,
-                                   static_cast<cudaStream_t>(stream));
+        fp8 ? launch_dispatch_fp8(s, layout->dst_row, x, recv, recv_scale, capacity_rows, ctx->ws, dispatch_queue(ctx),
+                                  ctx->n_sm, ctx->trace, static_cast<cudaStream_t>(stream))
+            : launch_dispatch_bf16(s, layout->dst_row, x, recv, capacity_rows, ctx->ws, dispatch_queue(ctx), ctx->n_sm,
+                                   ctx->trace, static_cast<cudaStream_t>(stream));
     {
         std::lock_guard<std::mutex> lk(ctx->mu);
         ctx->launches += 1;
+        if (err == cudaSuccess) ctx->n_dispatch += 1;
     }
     return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
 }
@@ -326,11 +358,12 @@ strata_status strata_moe_combine(strata_ctx* ctx, const strata_moe_layout_t* lay
     if (ctx->device < 0) return STRATA_ERR_CUDA;
     DeviceGuard g(ctx->device);
     if (!g.ok) return STRATA_ERR_CUDA;
-    cudaError_t err = launch_combine(ctx->shape, layout->dst_row, y, y_rows, topk_w, out, ctx->ws, ctx->n_sm,
-                                     static_cast<cudaStream_t>(stream));
+    cudaError_t err = launch_combine(ctx->shape, layout->dst_row, y, y_rows, topk_w, out, ctx->ws, combine_queue(ctx),
+                                     ctx->n_sm, ctx->trace, static_cast<cudaStream_t>(stream));
     {
         std::lock_guard<std::mutex> lk(ctx->mu);
         ctx->launches += 1;
+        if (err == cudaSuccess) ctx->n_combine += 1;
     }
     return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
 }

@@ -3,9 +3,11 @@
 //   out[n,c] = bf16_rne( fma(w[n,K-1], y[row(n,K-1),c], ... fma(w[n,0], y[row(n,0),c], +0) ) )
 // with binary32 fused multiply-adds in slot order 0..K-1.
 //
-// Work split: persistent CTAs take tokens round-robin, the grid sized so that every CTA gets the
-// same number of tokens (+-1); every token costs K row reads and one row write, so the split is
-// even whatever the expert popularity is.  A thread owns one
+// Work split: a unit is one token, or one column part of a token when there are too few tokens to
+// give every CTA several units: K (part-)row reads and one write whatever the expert popularity is.
+// The CTAs of a persistent grid start on unit blockIdx.x and then claim units in order from a
+// counter in the workspace, one unit ahead of the one being worked on (the claim travels while the
+// rows stream in), so no CTA is left with a fixed share it cannot finish in time.  A thread owns one
 // 16-byte column vector at a time: it issues the K independent 16-byte streaming loads first
 // (K requests in flight per thread), then runs the FMA chain in registers and writes 16 bytes.
 // The accumulation lives in registers; no atomics and no shared-memory staging are needed
@@ -27,7 +29,11 @@ struct CombineParams {
     long long y_rows;
     int H;
     int K;
+    int parts;             // units per token
+    int vec_per_part;      // 16-byte vectors per unit, a multiple of the CTA size (last part may be shorter)
     int* status;
+    WorkQueue wq;
+    TraceBuf trace;
 };
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
@@ -56,20 +62,34 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
     const int tid = threadIdx.x;
     const int vpr = p.H / 8;                       // 16-byte vectors per row
     const size_t row_bytes = (size_t)p.H * 2u;
+    const unsigned int n_units = (unsigned int)(p.n_tok * p.parts);
+    __shared__ unsigned int s_next[2];             // the claim made during unit j is read for unit j+1
+    griddep_wait();
+    arm_next_queue(p.wq);
+    if (tid == 0) trace_begin(p.trace);
 
-    for (long long n = blockIdx.x; n < p.n_tok; n += gridDim.x) {
+    unsigned int u = blockIdx.x < n_units ? blockIdx.x : kNoUnit;
+    for (int j = 0; u != kNoUnit; ++j) {
+        if (tid == 0) {
+            const unsigned int nx = claim_unit(p.wq, n_units, gridDim.x);
+            s_next[j & 1] = nx;
+            if (nx == kNoUnit) griddep_launch_dependents();   // last unit of this CTA: let the next kernel in
+        }
+        const unsigned int n = u / (unsigned int)p.parts;
+        const int part = (int)(u - n * (unsigned int)p.parts);
+        const int v_begin = part * p.vec_per_part, v_end = min(v_begin + p.vec_per_part, vpr);
         const unsigned char* src[K];
         float wk[K];
 #pragma unroll
         for (int k = 0; k < K; ++k) {
-            const int row = p.dst_row[n * K + k];
+            const int row = p.dst_row[(long long)n * K + k];
             const bool row_ok = row >= 0 && row < p.y_rows;
-            if (!row_ok && tid == 0) report_status(p.status, STRATA_ERR_BAD_ROW);
+            if (!row_ok && tid == 0 && part == 0) report_status(p.status, STRATA_ERR_BAD_ROW);
             src[k] = row_ok ? p.y + (size_t)row * row_bytes : nullptr;
-            wk[k] = p.w[n * K + k];
+            wk[k] = p.w[(long long)n * K + k];
         }
         unsigned char* dst = p.out + (size_t)n * row_bytes;
-        for (int v = tid; v < vpr; v += kCombineThreads) {
+        for (int v = v_begin + tid; v < v_end; v += kCombineThreads) {
             uint4 d[K];
 #pragma unroll
             for (int k = 0; k < K; ++k)
@@ -85,27 +105,42 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
             o.w = pack_bf16x2(a[6], a[7]);
             st_stream16(dst + (size_t)v * 16, o);
         }
+        __syncthreads();                           // one barrier per unit: publishes the next claim
+        u = s_next[j & 1];
+    }
+    if (tid == 0) {
+        trace_end(p.trace);
     }
 }
 
-// Any K <= kMaxTopK: slots are taken in groups of up to 8, still in slot order.
+// Any K <= kMaxTopK: a CTA claims whole tokens; slots are taken in groups of up to 8, in slot order.
 template <>
 __global__ void __launch_bounds__(kCombineThreads) combine_kernel<0>(CombineParams p)
 {
     const int tid = threadIdx.x, K = p.K;
     const int vpr = p.H / 8;
     const size_t row_bytes = (size_t)p.H * 2u;
+    const unsigned int n_units = (unsigned int)p.n_tok;
     __shared__ long long s_off[kMaxTopK];          // byte offset of the row, -1 if skipped
     __shared__ float s_w[kMaxTopK];
+    __shared__ unsigned int s_tok;
+    griddep_wait();
+    arm_next_queue(p.wq);
+    if (tid == 0) trace_begin(p.trace);
 
-    for (long long n = blockIdx.x; n < p.n_tok; n += gridDim.x) {
+    for (int j = 0;; ++j) {
+        __syncthreads();                           // everyone is done with the previous token's tables
+        if (tid == 0) s_tok = j == 0 ? (blockIdx.x < n_units ? blockIdx.x : kNoUnit)
+                                     : claim_unit(p.wq, n_units, gridDim.x);
         __syncthreads();
+        const unsigned int n = s_tok;
+        if (n == kNoUnit) break;
         if (tid < K) {
-            const int row = p.dst_row[n * K + tid];
+            const int row = p.dst_row[(long long)n * K + tid];
             const bool row_ok = row >= 0 && row < p.y_rows;
             if (!row_ok) report_status(p.status, STRATA_ERR_BAD_ROW);
             s_off[tid] = row_ok ? (long long)row * (long long)row_bytes : -1;
-            s_w[tid] = p.w[n * K + tid];
+            s_w[tid] = p.w[(long long)n * K + tid];
         }
         __syncthreads();
         unsigned char* dst = p.out + (size_t)n * row_bytes;
@@ -130,6 +165,9 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel<0>(CombinePara
             st_stream16(dst + (size_t)v * 16, o);
         }
     }
+    if (tid == 0) {
+        trace_end(p.trace);
+    }
 }
 
 template <int KT>
@@ -140,17 +178,33 @@ cudaError_t launch_k(const CombineParams& p, int n_sm, cudaStream_t st)
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, combine_kernel<KT>, kCombineThreads, 0);
     if (err != cudaSuccess) return err;
     if (per_sm < 1) per_sm = 1;
-    const long long grid = balanced_grid(p.n_tok, (long long)n_sm * per_sm);
-    combine_kernel<KT><<<(unsigned)grid, kCombineThreads, 0, st>>>(p);
-    return cudaGetLastError();
+    CombineParams q = p;
+    const long long max_grid = (long long)n_sm * per_sm;
+    q.parts = 1;
+    q.vec_per_part = (p.H / 8 + kCombineThreads - 1) / kCombineThreads * kCombineThreads;
+    if (KT > 0) {
+        // split rows into column parts until every CTA can expect about 6 units (never below one
+        // vector per thread per unit)
+        const int m_full = q.vec_per_part / kCombineThreads;
+        int parts = 1;
+        while (parts < m_full && p.n_tok * parts < 6 * max_grid) ++parts;
+        q.vec_per_part = (m_full + parts - 1) / parts * kCombineThreads;
+        q.parts = (p.H / 8 + q.vec_per_part - 1) / q.vec_per_part;
+    }
+    const long long grid = max(1ll, min(max_grid, p.n_tok * q.parts));
+    const bool small = p.n_tok * p.H * 2 * (p.K + 1) < kPdlMaxBytes;
+    return STRATA_LAUNCH_LONG(small, combine_kernel<KT>, (unsigned)grid, kCombineThreads, 0, st, q);
 }
 
 }  // namespace
 
 cudaError_t launch_combine(const strata_moe_shape& s, const int32_t* dst_row, const void* y, size_t y_rows,
-                           const float* w, void* out, int* status, int n_sm, cudaStream_t st)
+                           const float* w, void* out, int* status, WorkQueue wq, int n_sm, TraceBuf trace,
+                           cudaStream_t st)
 {
     CombineParams p{};
+    p.trace = trace;
+    p.wq = wq;
     p.dst_row = dst_row;
     p.y = static_cast<const unsigned char*>(y);
     p.w = w;

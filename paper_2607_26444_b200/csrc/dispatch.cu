@@ -2,11 +2,10 @@
 // the layout assigned, straight into the caller's (registered) receive buffer.
 //
 // Work split: a unit is one token (or one column chunk of a token when a row is larger than
-// a stage).  Units are dealt round-robin to a persistent grid whose size is chosen so that every
-// CTA gets the same number of units (+-1): every CTA moves the same bytes whatever the expert
-// popularity is, 1 row read + K row writes per unit.  Round-robin (rather than one contiguous
-// span per CTA) keeps the CTAs that run at the same time on neighbouring rows, which measured
-// 1..2 % faster for dispatch and far faster for combine.
+// a stage): 1 row read + K row writes whatever the expert popularity is.  A persistent grid claims
+// units in order from a counter in the workspace, two units ahead of the one being stored, so the
+// claim latency is hidden, CTAs running together work on neighbouring rows, and no CTA is left
+// with a fixed share it cannot finish in time.
 //
 // bf16: each CTA is a single warp that runs the SM's bulk-copy engine as a small DMA program
 //       (the on-SM counterpart of the paper's device-issued SDMA descriptors, Sec. 6.3):
@@ -22,9 +21,13 @@ namespace strata {
 
 namespace {
 
-// Build-time tuning knobs.  Measured on B200 at the prefill shape: 2..4 stages, 2..5 CTAs per SM,
+// Build-time tuning knobs.  Measured on B200 at the prefill shape: 2..4 stages, 1..5 CTAs per SM,
 // 4..16 KB chunks and the store hint all land within 1% of each other (5.68..5.71 TB/s); a variant
 // that moved the payload through registers (16-byte loads, K 16-byte stores) reached 5.0 TB/s.
+// What bounds the kernel is HBM serving a 1:8 read:write mix: with the same stores and the source
+// rows resident in L2 the kernel writes at 6.3 TB/s (the rate of a pure bulk-store fill), with the
+// source in DRAM it runs at 5.7 TB/s whichever way the rows are loaded (bulk copy, cp.async, or
+// producer warps with plain loads), and clustering the reads with L2 prefetches made it slower.
 #ifndef STRATA_BF16_STAGES
 #define STRATA_BF16_STAGES 3
 #endif
@@ -32,7 +35,7 @@ namespace {
 #define STRATA_BF16_CHUNK_BYTES 16384
 #endif
 #ifndef STRATA_BF16_MAX_CTAS_PER_SM
-#define STRATA_BF16_MAX_CTAS_PER_SM 0          // 0: as many as fit
+#define STRATA_BF16_MAX_CTAS_PER_SM 2          // 0: as many as fit
 #endif
 #ifndef STRATA_BF16_STORE_HINT
 #define STRATA_BF16_STORE_HINT 0               // 1: L2 evict-first policy on the bulk stores
@@ -54,6 +57,8 @@ struct DispatchParams {
     int chunks_per_row;
     uint32_t chunk_cols;        // columns per chunk (last chunk of a row may be shorter)
     int* status;
+    WorkQueue wq;
+    TraceBuf trace;
 };
 
 __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
@@ -61,55 +66,71 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
     extern __shared__ __align__(128) unsigned char smem[];
     const uint32_t stage_bytes = p.chunk_cols * 2u;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kBf16Stages * stage_bytes);
+    unsigned int* s_unit = reinterpret_cast<unsigned int*>(bars + kBf16Stages);   // unit held by each stage
     const int lane = threadIdx.x;
     const size_t row_bytes = (size_t)p.H * 2u;
-
-    const long long first = blockIdx.x, stride = gridDim.x;
-    if (first >= p.n_units) return;
-    const long long n_my = (p.n_units - first + stride - 1) / stride;
+    const unsigned int n_units = (unsigned int)p.n_units;
 
     if (lane == 0) {
-        for (int s = 0; s < kBf16Stages; ++s) mbar_init(&bars[s], 1);
+        for (int s = 0; s < kBf16Stages; ++s) {
+            mbar_init(&bars[s], 1);
+            s_unit[s] = kNoUnit;
+        }
         mbar_fence_init();
     }
     __syncwarp();
     const uint64_t pol = policy_evict_first();
+    griddep_wait();                       // x and dst_row belong to earlier kernels in the stream
+    arm_next_queue(p.wq);
+    if (lane == 0) trace_begin(p.trace);
 
-    auto issue_load = [&](long long j) {   // lane 0 only
-        const long long u = first + j * stride;
-        const long long tok = u / p.chunks_per_row;
-        const int ch = (int)(u - tok * p.chunks_per_row);
-        const uint32_t col0 = (uint32_t)ch * p.chunk_cols;
-        const uint32_t bytes = min(p.chunk_cols, (uint32_t)p.H - col0) * 2u;
+    auto decode = [&](unsigned int u, long long& tok, uint32_t& col0, uint32_t& bytes) {
+        tok = u / (unsigned int)p.chunks_per_row;
+        const uint32_t ch = u - (unsigned int)tok * (unsigned int)p.chunks_per_row;
+        col0 = ch * p.chunk_cols;
+        bytes = min(p.chunk_cols, (uint32_t)p.H - col0) * 2u;
+    };
+    bool triggered = false;
+    // The first stages-1 units of a CTA are fixed (blockIdx + j*grid); the rest are claimed.
+    const unsigned int n_static = (unsigned int)(kBf16Stages - 1) * gridDim.x;
+    auto issue_load = [&](long long j) {   // lane 0 only: next unit into stage j % stages
         const int s = (int)(j % kBf16Stages);
+        unsigned int u;
+        if (j < kBf16Stages - 1) {
+            u = blockIdx.x + (unsigned int)j * gridDim.x;
+            if (u >= n_units) u = kNoUnit;
+        } else {
+            u = claim_unit(p.wq, n_units, n_static);
+        }
+        s_unit[s] = u;
+        if (u == kNoUnit) {
+            if (!triggered) griddep_launch_dependents();   // queue empty: the next kernel may be scheduled
+            triggered = true;
+            return;
+        }
+        long long tok;
+        uint32_t col0, bytes;
+        decode(u, tok, col0, bytes);
         mbar_expect_tx(&bars[s], bytes);
-#ifdef STRATA_EXP_XMOD
-        bulk_g2s(smem + (size_t)s * stage_bytes, p.x + (size_t)(tok % STRATA_EXP_XMOD) * row_bytes + (size_t)col0 * 2u, bytes, &bars[s],
-                 pol);
-#else
         bulk_g2s(smem + (size_t)s * stage_bytes, p.x + (size_t)tok * row_bytes + (size_t)col0 * 2u, bytes, &bars[s],
                  pol);
-#endif
     };
 
     if (lane == 0)
-        for (long long j = 0; j < kBf16Stages - 1 && j < n_my; ++j) issue_load(j);
+        for (long long j = 0; j < kBf16Stages - 1; ++j) issue_load(j);
+    __syncwarp();
 
     bool ok = true;
-    for (long long j = 0; j < n_my; ++j) {
-        const long long u = first + j * stride;
-        const long long tok = u / p.chunks_per_row;
-        const int ch = (int)(u - tok * p.chunks_per_row);
-        const uint32_t col0 = (uint32_t)ch * p.chunk_cols;
-        const uint32_t bytes = min(p.chunk_cols, (uint32_t)p.H - col0) * 2u;
+    for (long long j = 0;; ++j) {
         const int s = (int)(j % kBf16Stages);
         const uint32_t parity = (uint32_t)((j / kBf16Stages) & 1);
+        const unsigned int u = s_unit[s];
+        if (u == kNoUnit) break;          // claims fail in order: nothing is in flight behind this stage
+        long long tok;
+        uint32_t col0, bytes;
+        decode(u, tok, col0, bytes);
 
-#ifdef STRATA_EXP_SEQ
-        const int my_row = (lane < p.K) ? (int)(tok * p.K + lane) : -1;
-#else
         const int my_row = (lane < p.K) ? p.dst_row[tok * p.K + lane] : -1;
-#endif
         const bool row_ok = (lane >= p.K) || (my_row >= 0 && my_row < p.capacity_rows);
         if (!row_ok) report_status(p.status, STRATA_ERR_BAD_ROW);
 
@@ -131,17 +152,15 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
         if (lane == 0) {
             bulk_commit();
             // The stage that unit j-1 used is refilled next; its stores must have left shared memory.
-            const long long jn = j + kBf16Stages - 1;
-            if (jn < n_my) {
-                bulk_wait_read<1>();
-                issue_load(jn);
-            }
+            bulk_wait_read<1>();
+            issue_load(j + kBf16Stages - 1);
         }
         __syncwarp();
     }
     if (lane == 0) {
         if (!ok) report_status(p.status, STRATA_ERR_TIMEOUT);
         bulk_wait_read<0>();
+        trace_end(p.trace);
     }
 }
 
@@ -168,10 +187,11 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
     const int tid = threadIdx.x, lane = tid & 31;
     const size_t in_row_bytes = (size_t)p.H * 2u, out_row_bytes = (size_t)p.H;
     const int nb_row = p.H / 128;
+    const unsigned int n_units = (unsigned int)p.n_units;
 
-    const long long first = blockIdx.x, stride = gridDim.x;
-    if (first >= p.n_units) return;
-    const long long n_my = (p.n_units - first + stride - 1) / stride;
+    __shared__ unsigned int s_unit[2];     // unit held by each input stage
+    __shared__ int s_rows[kMaxTopK];
+    __shared__ float s_scale[kFp8MaxChunkCols / 128];
 
     if (tid == 0) {
         mbar_init(&bars[0], 1);
@@ -180,33 +200,54 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
     }
     __syncthreads();
     const uint64_t pol = policy_evict_first();
+    griddep_wait();
+    arm_next_queue(p.wq);
+    if (tid == 0) trace_begin(p.trace);
 
+    auto decode = [&](unsigned int u, long long& tok, uint32_t& col0, uint32_t& cols) {
+        tok = u / (unsigned int)p.chunks_per_row;
+        const uint32_t ch = u - (unsigned int)tok * (unsigned int)p.chunks_per_row;
+        col0 = ch * p.chunk_cols;
+        cols = min(p.chunk_cols, (uint32_t)p.H - col0);
+    };
+    bool triggered = false;
+    const unsigned int n_static = 2u * gridDim.x;   // the first two units of a CTA are fixed
     auto issue_load = [&](long long j) {   // thread 0 only
-        const long long u = first + j * stride;
-        const long long tok = u / p.chunks_per_row;
-        const int ch = (int)(u - tok * p.chunks_per_row);
-        const uint32_t col0 = (uint32_t)ch * p.chunk_cols;
-        const uint32_t cols = min(p.chunk_cols, (uint32_t)p.H - col0);
         const int s = (int)(j & 1);
+        unsigned int u;
+        if (j < 2) {
+            u = blockIdx.x + (unsigned int)j * gridDim.x;
+            if (u >= n_units) u = kNoUnit;
+        } else {
+            u = claim_unit(p.wq, n_units, n_static);
+        }
+        s_unit[s] = u;
+        if (u == kNoUnit) {
+            if (!triggered) griddep_launch_dependents();   // queue empty: the next kernel may be scheduled
+            triggered = true;
+            return;
+        }
+        long long tok;
+        uint32_t col0, cols;
+        decode(u, tok, col0, cols);
         mbar_expect_tx(&bars[s], cols * 2u);
         bulk_g2s(in_stage(s), p.x + (size_t)tok * in_row_bytes + (size_t)col0 * 2u, cols * 2u, &bars[s], pol);
     };
     if (tid == 0) {
         issue_load(0);
-        if (n_my > 1) issue_load(1);
+        issue_load(1);
     }
+    __syncthreads();
 
-    __shared__ int s_rows[kMaxTopK];
-    __shared__ float s_scale[kFp8MaxChunkCols / 128];
     bool ok = true;
-    for (long long j = 0; j < n_my; ++j) {
-        const long long u = first + j * stride;
-        const long long tok = u / p.chunks_per_row;
-        const int ch = (int)(u - tok * p.chunks_per_row);
-        const uint32_t col0 = (uint32_t)ch * p.chunk_cols;
-        const uint32_t cols = min(p.chunk_cols, (uint32_t)p.H - col0);
+    for (long long j = 0;; ++j) {
         const int s = (int)(j & 1);
         const uint32_t parity = (uint32_t)((j >> 1) & 1);
+        const unsigned int u = s_unit[s];
+        if (u == kNoUnit) break;
+        long long tok;
+        uint32_t col0, cols;
+        decode(u, tok, col0, cols);
 
         if (tid < p.K) {
             const int row = p.dst_row[tok * p.K + tid];
@@ -262,13 +303,14 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
                 if (row >= 0) bulk_s2g(p.recv + (size_t)row * out_row_bytes + col0, out_stage(s), cols);
             }
             bulk_commit();
-            if (j + 2 < n_my) issue_load(j + 2);    // in_stage(s) was fully consumed before the barrier above
+            issue_load(j + 2);                      // in_stage(s) was fully consumed before the barrier above
         }
-        __syncthreads();                            // s_rows is rewritten next iteration
+        __syncthreads();                            // s_rows, s_scale and s_unit[s] are rewritten next
     }
     if (tid == 0) {
         if (!ok) report_status(p.status, STRATA_ERR_TIMEOUT);
         bulk_wait_read<0>();
+        trace_end(p.trace);
     }
 }
 
@@ -294,9 +336,12 @@ cudaError_t configure_dispatch_kernels()
 }
 
 cudaError_t launch_dispatch_bf16(const strata_moe_shape& s, const int32_t* dst_row, const void* x, void* recv,
-                                 size_t capacity_rows, int* status, int n_sm, cudaStream_t st)
+                                 size_t capacity_rows, int* status, WorkQueue wq, int n_sm, TraceBuf trace,
+                                 cudaStream_t st)
 {
     DispatchParams p{};
+    p.trace = trace;
+    p.wq = wq;
     p.dst_row = dst_row;
     p.x = static_cast<const unsigned char*>(x);
     p.recv = static_cast<unsigned char*>(recv);
@@ -308,21 +353,24 @@ cudaError_t launch_dispatch_bf16(const strata_moe_shape& s, const int32_t* dst_r
     p.n_units = (long long)s.R * s.T * p.chunks_per_row;
     p.capacity_rows = (long long)capacity_rows;
     p.status = status;
-    const size_t smem = (size_t)kBf16Stages * p.chunk_cols * 2u + 64;
+    const size_t smem = (size_t)kBf16Stages * p.chunk_cols * 2u + 64;   // stages | mbarriers | unit ids
     int per_sm = 0;
     cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dispatch_bf16_kernel, 32, smem);
     if (err != cudaSuccess) return err;
     if (per_sm < 1) per_sm = 1;
     if (STRATA_BF16_MAX_CTAS_PER_SM > 0) per_sm = min(per_sm, STRATA_BF16_MAX_CTAS_PER_SM);
-    const long long grid = balanced_grid(p.n_units, (long long)n_sm * per_sm);
-    dispatch_bf16_kernel<<<(unsigned)grid, 32, smem, st>>>(p);
-    return cudaGetLastError();
+    const long long grid = max(1ll, min((long long)n_sm * per_sm, p.n_units));
+    const bool small = (long long)s.R * s.T * s.H * 2 * (s.K + 1) < kPdlMaxBytes;
+    return STRATA_LAUNCH_LONG(small, dispatch_bf16_kernel, (unsigned)grid, 32, smem, st, p);
 }
 
 cudaError_t launch_dispatch_fp8(const strata_moe_shape& s, const int32_t* dst_row, const void* x, void* recv_q,
-                                float* recv_scale, size_t capacity_rows, int* status, int n_sm, cudaStream_t st)
+                                float* recv_scale, size_t capacity_rows, int* status, WorkQueue wq, int n_sm,
+                                TraceBuf trace, cudaStream_t st)
 {
     DispatchParams p{};
+    p.trace = trace;
+    p.wq = wq;
     p.dst_row = dst_row;
     p.x = static_cast<const unsigned char*>(x);
     p.recv = static_cast<unsigned char*>(recv_q);
@@ -339,9 +387,9 @@ cudaError_t launch_dispatch_fp8(const strata_moe_shape& s, const int32_t* dst_ro
     cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dispatch_fp8_kernel, kFp8Threads, smem);
     if (err != cudaSuccess) return err;
     if (per_sm < 1) per_sm = 1;
-    const long long grid = balanced_grid(p.n_units, (long long)n_sm * per_sm);
-    dispatch_fp8_kernel<<<(unsigned)grid, kFp8Threads, smem, st>>>(p);
-    return cudaGetLastError();
+    const long long grid = max(1ll, min((long long)n_sm * per_sm, p.n_units));
+    const bool small = (long long)s.R * s.T * s.H * (s.K + 2) < kPdlMaxBytes;
+    return STRATA_LAUNCH_LONG(small, dispatch_fp8_kernel, (unsigned)grid, kFp8Threads, smem, st, p);
 }
 
 }  // namespace strata

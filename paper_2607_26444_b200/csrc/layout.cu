@@ -102,6 +102,8 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_count_scan_kernel(Layou
     for (int e = tid; e < E; e += kLayoutThreads) hist[e] = 0;
     __syncthreads();
     const int ebits = key_bits(E);
+    griddep_wait();
+    griddep_launch_dependents();          // the rank kernel may start its local pass now
 
     int ids[kItemsPerThread];
 #pragma unroll
@@ -293,6 +295,10 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_rank_kernel(LayoutParam
         }
     }
     __syncthreads();
+    // Everything above only read the ids (complete before the counting kernel was allowed to start
+    // us).  The tile prefixes and expert offsets below come from the counting kernel itself.
+    griddep_wait();
+    griddep_launch_dependents();
 #pragma unroll
     for (int q = 0; q < kItemsPerThread; ++q) {
         const int in_rank = warp_first + q * 32 + lane;
@@ -330,6 +336,8 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_small_kernel(LayoutPara
     int* mine = warp_cnt + wid * E;
     const int ebits = key_bits(E);
 
+    griddep_wait();
+    griddep_launch_dependents();
     // contiguous run per warp, a multiple of 32 items
     const int run = ((n_items + 31) / 32 + 31) / 32 * 32;      // ceil(ceil(N/32)/32)*32 >= N/32
     const int first = wid * run;
@@ -486,16 +494,13 @@ cudaError_t launch_layout(const strata_moe_shape& s, const int32_t* ids, const s
     const long long n_items = (long long)s.R * s.T * s.K;
     const size_t small_bytes = small_smem(s.E, s.R, L.src_expert_count != nullptr);
     if (n_items <= kSmallItems && small_bytes <= kSmallSmemLimit) {
-        layout_small_kernel<<<1, kLayoutThreads, small_bytes, st>>>(p, (int)n_items);
         *n_launches = 1;
-        return cudaGetLastError();
+        return launch_pdl(layout_small_kernel, 1, kLayoutThreads, small_bytes, st, p, (int)n_items);
     }
-    layout_count_scan_kernel<<<g.n_tiles, kLayoutThreads, count_scan_smem(s.E), st>>>(p);
-    cudaError_t err = cudaGetLastError();
-    if (err != cudaSuccess) return err;
-    layout_rank_kernel<<<g.n_tiles, kLayoutThreads, (size_t)32 * s.E * sizeof(int), st>>>(p);
     *n_launches = 2;
-    return cudaGetLastError();
+    cudaError_t err = launch_pdl(layout_count_scan_kernel, (unsigned)g.n_tiles, kLayoutThreads, count_scan_smem(s.E), st, p);
+    if (err != cudaSuccess) return err;
+    return launch_pdl(layout_rank_kernel, (unsigned)g.n_tiles, kLayoutThreads, (size_t)32 * s.E * sizeof(int), st, p);
 }
 
 }  // namespace strata

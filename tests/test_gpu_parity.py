@@ -376,3 +376,38 @@ def test_roundtrip_from_host_buffers():
     assert np.array_equal(h_out.numpy().view(np.uint16), ref_out)
     assert ctx.device_status() == B.STRATA_OK
     ctx.close()
+
+
+def test_per_cta_trace_probes():
+    """Stage probes: every CTA of a traced launch records start <= end on the global timer; the spread
+    of end times under Zipf routing stays small because tokens, not experts, are dealt to the CTAs."""
+    cfg = wl.shrink(wl.CONFIGS["skew"], T=256)
+    inp = wl.generate(cfg)
+    ctx = make_ctx(cfg)
+    lay = ctx.layout(to_dev(inp["ids"]))
+    x_d, w_d = to_dev(inp["x"]), to_dev(inp["w"])
+    recv = torch.empty((cfg.n_items, cfg.H), dtype=torch.int16, device=DEV)
+    out = torch.empty((cfg.n_tok, cfg.H), dtype=torch.int16, device=DEV)
+    ctx.register(recv)
+    for _ in range(2):
+        ctx.dispatch(lay, x_d, recv)
+    tr = ctx.trace(4096)
+    for name, call in (("dispatch", lambda: ctx.dispatch(lay, x_d, recv)),
+                       ("combine", lambda: ctx.combine(lay, recv, w_d, out))):
+        tr.zero_()
+        call()
+        torch.cuda.synchronize()
+        rec = tr.cpu().numpy()
+        used = rec[rec[:, 0] != 0]
+        assert 148 <= len(used) <= 4096, name
+        assert np.all(used[:, 1] >= used[:, 0]), name
+        total = used[:, 1].max() - used[:, 0].min()
+        spread = (used[:, 1].max() - used[:, 1].min()) / total
+        assert total > 0 and 0 <= spread < 0.5, (name, spread)
+    ctx.trace_off()
+    tr.zero_()
+    ctx.dispatch(lay, x_d, recv)
+    torch.cuda.synchronize()
+    assert int(tr.abs().sum().item()) == 0                   # probes off: nothing written
+    assert ctx.device_status() == B.STRATA_OK
+    ctx.close()
