@@ -18,7 +18,13 @@ namespace strata {
 
 namespace {
 
-constexpr int kCombineThreads = 128;
+#ifndef STRATA_COMBINE_THREADS
+#define STRATA_COMBINE_THREADS 128
+#endif
+#ifndef STRATA_COMBINE_MAX_CTAS_PER_SM
+#define STRATA_COMBINE_MAX_CTAS_PER_SM 0     // 0: as many as fit
+#endif
+constexpr int kCombineThreads = STRATA_COMBINE_THREADS;
 
 struct CombineParams {
     const int32_t* dst_row;
@@ -178,6 +184,7 @@ cudaError_t launch_k(const CombineParams& p, int n_sm, cudaStream_t st)
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, combine_kernel<KT>, kCombineThreads, 0);
     if (err != cudaSuccess) return err;
     if (per_sm < 1) per_sm = 1;
+    if (STRATA_COMBINE_MAX_CTAS_PER_SM > 0) per_sm = min(per_sm, STRATA_COMBINE_MAX_CTAS_PER_SM);
     CombineParams q = p;
     const long long max_grid = (long long)n_sm * per_sm;
     q.parts = 1;

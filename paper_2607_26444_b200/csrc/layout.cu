@@ -1,7 +1,7 @@
 // Routing layout (paper App. C, level 1 "token placement"): per-expert counts, prefix-sum
 // offsets and token-local offsets, as a stable counting sort of the items by expert id.
 //
-// Batches of up to 4,096 items take one launch of a single CTA (layout_small_kernel, below).
+// Batches of up to 32,768 items take one launch of one thread-block cluster (layout_cluster_kernel).
 // Larger batches take two launches, no device-side waiting anywhere:
 //   1. layout_count_scan_kernel: one CTA per tile of 4096 items (a tile never spans two
 //      source ranks).  Each warp aggregates equal ids with ballot-built same-id masks so a popular expert
@@ -12,6 +12,8 @@
 //   2. layout_rank_kernel: one CTA per tile again; rank of an item inside its tile =
 //      (items with the same id in earlier warps) + (same id in earlier lanes), both
 //      from same-id lane masks, so the order is exact and no atomics decide a row.
+#include <cooperative_groups.h>
+
 #include <mutex>
 
 #include "common.cuh"
@@ -315,22 +317,30 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_rank_kernel(LayoutParam
     }
 }
 
-// ---- small batches: the whole layout in one CTA, one launch ---------------------------------
-// Up to kSmallItems items: warp w owns a contiguous run of kSmallRounds*32 items, kept in
-// registers between the counting pass and the ranking pass; all intermediate tables live in
-// shared memory, so nothing waits on global memory in between.  One SM is issue bound beyond a
-// few thousand items (measured: 8 us at 1,024 items, 31 us at 16,384 against 19.5 us tiled).
+// ---- small and medium batches: the whole layout in one launch ---------------------------------
+// One thread-block cluster (1 CTA up to 4,096 items, 8 CTAs up to 32,768: the decode shape has
+// 16,384).  Warp w of CTA c owns a contiguous run of up to kSmallRounds*32 items, kept in registers
+// between the counting pass and the ranking pass; all tables live in shared memory, and the CTAs
+// of the cluster read each other's per-expert totals through distributed shared memory after one
+// hardware cluster barrier.  Nothing goes through global memory between the passes and nothing spins.
 constexpr int kSmallRounds = 4;
-constexpr int kSmallItems = 32 * 32 * kSmallRounds;
+constexpr int kSmallItems = 32 * 32 * kSmallRounds;      // per CTA
+constexpr int kLayoutCluster = 8;
 
-__global__ void __launch_bounds__(kLayoutThreads) layout_small_kernel(LayoutParams p, int n_items)
+
+__global__ void __launch_bounds__(kLayoutThreads) layout_cluster_kernel(LayoutParams p, int n_items)
 {
-    extern __shared__ int sm[];          // warp_cnt[32*E] | offs[E+1] | warp_sums[32] | total
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int n_cta = (int)cluster.num_blocks(), cta = (int)cluster.block_rank();
+
+    extern __shared__ int sm[];          // warp_cnt[32*E] | offs[E+1] | cta_cnt[E] | warp_sums[32] | total[2] | src_cnt[R*E]
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int E = p.E;
     int* warp_cnt = sm;
     int* offs = sm + 32 * E;
-    int* warp_sums = offs + E + 1;
+    int* cta_cnt = offs + E + 1;
+    int* warp_sums = cta_cnt + E;
     int* total = warp_sums + 32;
     int* src_cnt = total + 2;             // [R*E], only when src_expert_count is wanted
     int* mine = warp_cnt + wid * E;
@@ -338,9 +348,10 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_small_kernel(LayoutPara
 
     griddep_wait();
     griddep_launch_dependents();
-    // contiguous run per warp, a multiple of 32 items
-    const int run = ((n_items + 31) / 32 + 31) / 32 * 32;      // ceil(ceil(N/32)/32)*32 >= N/32
-    const int first = wid * run;
+    // contiguous run per warp over all warps of the cluster, a multiple of 32 items
+    const int n_warps = 32 * n_cta;
+    const int run = ((n_items + n_warps - 1) / n_warps + 31) / 32 * 32;
+    const int first = (cta * 32 + wid) * run;
 
     int ids[kSmallRounds];
 #pragma unroll
@@ -379,19 +390,14 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_small_kernel(LayoutPara
                 if (leader) atomicAdd(&src_cnt[r * E + e], __popc(peers));
             } else {
                 const unsigned peers2 = peers & same_key_lanes(r - r_lo_valid, 5);
-                if (valid && lane == __ffs(peers2) - 1)
-                    atomicAdd(&src_cnt[r * E + e], __popc(peers2));
+                if (valid && lane == __ffs(peers2) - 1) atomicAdd(&src_cnt[r * E + e], __popc(peers2));
             }
         }
         __syncwarp();
     }
     __syncthreads();
 
-    if (p.src_expert_count)
-        for (int x = tid; x < p.R * E; x += kLayoutThreads) p.src_expert_count[x] = src_cnt[x];
-
-    // exclusive prefix over the 32 warps per expert; totals are the per-expert counts
-    int count_e = 0;
+    // exclusive prefix over this CTA's 32 warps per expert; the totals go to cta_cnt for the cluster
     if (tid < E) {
         int running = 0;
 #pragma unroll 8
@@ -400,27 +406,61 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_small_kernel(LayoutPara
             warp_cnt[w * E + tid] = running;
             running += c;
         }
-        count_e = running;
+        cta_cnt[tid] = running;
+    }
+    cluster.sync();                       // every CTA's cta_cnt and src_cnt are complete and visible
+
+    // items with the same id in earlier CTAs of the cluster, and the cluster-wide count
+    int before = 0, count_e = 0;
+    if (tid < E) {
+        int v[kLayoutCluster];
+#pragma unroll
+        for (int c = 0; c < kLayoutCluster; ++c) v[c] = c < n_cta ? *cluster.map_shared_rank(&cta_cnt[tid], c) : 0;
+#pragma unroll
+        for (int c = 0; c < kLayoutCluster; ++c) {
+            if (c < cta) before += v[c];
+            count_e += v[c];
+        }
     }
     const int off = block_exclusive_scan_1024(count_e, warp_sums, total);
-    if (tid < E) {
-        p.expert_count[tid] = count_e;
-        p.expert_offset[tid] = off;
-        offs[tid] = off;
-    }
-    if (tid == 0) {
-        p.expert_offset[E] = *total;
-        p.rank_offset[p.R] = *total;
-        offs[E] = *total;
+    if (tid < E) offs[tid] = off;
+    if (tid == 0) offs[E] = *total;
+    if (cta == 0) {
+        if (tid < E) {
+            p.expert_count[tid] = count_e;
+            p.expert_offset[tid] = off;
+        }
+        if (tid == 0) {
+            p.expert_offset[E] = *total;
+            p.rank_offset[p.R] = *total;
+        }
     }
     __syncthreads();
-    for (int d = tid; d < p.R; d += kLayoutThreads) {
-        const int lo = offs[d * p.e_loc], hi = offs[(d + 1) * p.e_loc];
-        p.rank_offset[d] = lo;
-        p.rank_count[d] = hi - lo;
+    if (cta == 0)
+        for (int d = tid; d < p.R; d += kLayoutThreads) {
+            const int lo = offs[d * p.e_loc], hi = offs[(d + 1) * p.e_loc];
+            p.rank_offset[d] = lo;
+            p.rank_count[d] = hi - lo;
+        }
+    if (p.src_expert_count) {             // CTA c sums its contiguous slice of the per-source-rank table
+        const int slice = (p.R * E + n_cta - 1) / n_cta;
+        const int x_end = min(p.R * E, (cta + 1) * slice);
+        for (int x = cta * slice + tid; x < x_end; x += kLayoutThreads) {
+            int v[kLayoutCluster];
+#pragma unroll
+            for (int c = 0; c < kLayoutCluster; ++c)        // all remote reads in flight together
+                v[c] = c < n_cta ? *cluster.map_shared_rank(&src_cnt[x], c) : 0;
+            int sum = 0;
+#pragma unroll
+            for (int c = 0; c < kLayoutCluster; ++c) sum += v[c];
+            p.src_expert_count[x] = sum;
+        }
     }
+    __syncthreads();
+    if (tid < E) offs[tid] += before;     // first row of this CTA's items in each expert's segment
+    __syncthreads();
 
-    // pass 2: rows.  mine[e] now counts the same-id items of earlier warps and earlier rounds.
+    // pass 2: rows.  mine[e] counts the same-id items of earlier warps and earlier rounds of this CTA.
     const unsigned lt = (1u << lane) - 1u;
 #pragma unroll
     for (int q = 0; q < kSmallRounds; ++q) {
@@ -445,10 +485,14 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_small_kernel(LayoutPara
         }
         __syncwarp();
     }
+    cluster.sync();                       // no CTA leaves while another may still read its shared memory
 }
 
-// shared memory of the single-CTA kernel; the per-source-rank table is only there when asked for
-size_t small_smem(int E, int R, bool with_src) { return (size_t)(32 * E + E + 1 + 32 + 2 + (with_src ? R * E : 0)) * sizeof(int); }
+// shared memory of the cluster kernel; the per-source-rank table is only there when asked for
+size_t small_smem(int E, int R, bool with_src)
+{
+    return (size_t)(32 * E + E + 1 + E + 32 + 2 + (with_src ? R * E : 0)) * sizeof(int);
+}
 constexpr size_t kSmallSmemLimit = 200 * 1024;
 
 size_t count_scan_smem(int E)
@@ -464,7 +508,7 @@ cudaError_t configure_layout_kernels()
     cudaError_t err = cudaFuncSetAttribute(layout_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            32 * kMaxExperts * (int)sizeof(int));
     if (err != cudaSuccess) return err;
-    return cudaFuncSetAttribute(layout_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(layout_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)kSmallSmemLimit);
 }
 
@@ -493,9 +537,11 @@ cudaError_t launch_layout(const strata_moe_shape& s, const int32_t* ids, const s
 
     const long long n_items = (long long)s.R * s.T * s.K;
     const size_t small_bytes = small_smem(s.E, s.R, L.src_expert_count != nullptr);
-    if (n_items <= kSmallItems && small_bytes <= kSmallSmemLimit) {
+    if (n_items <= (long long)kSmallItems * kLayoutCluster && small_bytes <= kSmallSmemLimit) {
+        const unsigned n_cta = n_items <= kSmallItems ? 1u : (unsigned)kLayoutCluster;
         *n_launches = 1;
-        return launch_pdl(layout_small_kernel, 1, kLayoutThreads, small_bytes, st, p, (int)n_items);
+        return launch_pdl_cluster(layout_cluster_kernel, n_cta, kLayoutThreads, small_bytes, n_cta, st, p,
+                                  (int)n_items);
     }
     *n_launches = 2;
     cudaError_t err = launch_pdl(layout_count_scan_kernel, (unsigned)g.n_tiles, kLayoutThreads, count_scan_smem(s.E), st, p);
@@ -609,3 +655,4 @@ extern "C" strata_status strata_moe_layout_noalloc(const strata_moe_shape* shape
     layout_rank_kernel<<<g.n_tiles, kLayoutThreads, (size_t)32 * s.E * sizeof(int), st>>>(p);
     return cudaGetLastError() == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
 }
+

@@ -193,7 +193,10 @@ RAGGED = [
     dict(R=5, T=50, H=4096, E=20, K=6),
     dict(R=4, T=100, H=2048, E=16, K=4),
     dict(R=4, T=256, H=64, E=32, K=4),               # 4,096 items: the largest single-CTA layout
-    dict(R=4, T=257, H=64, E=32, K=4),               # just above it: tiled layout
+    dict(R=4, T=257, H=64, E=32, K=4),               # just above it: a cluster of 8 CTAs
+    dict(R=4, T=2048, H=64, E=32, K=4),              # 32,768 items: the largest cluster layout
+    dict(R=4, T=2049, H=64, E=32, K=4),              # just above it: tiled layout, two launches
+    dict(R=5, T=1111, H=64, E=1000, K=3),            # cluster layout, CTAs and warps straddle ranks, wide E
     dict(R=64, T=3, H=64, E=64, K=7),                # warps straddle several source ranks
 ]
 
