@@ -42,9 +42,9 @@ FALLBACK_HBM_GBS = 6650.0
 # ncu --set full on the same recipe at T=512 tokens/rank (1/8 of the tokens) and scaled by 8, since
 # traffic grows in proportion to the tokens (profiles/*_prefill_T512.md); None = no capture yet.
 NCU_TRAFFIC_BYTES = {
-    "dispatch_bf16_kernel": 8 * (117_928_192 + 879_901_696),
-    "dispatch_fp8_kernel": None,
-    "combine_kernel": 8 * (940_062_208 + 98_784_768),
+    "dispatch_bf16_kernel": 8 * (117_720_832 + 879_663_104),
+    "dispatch_fp8_kernel": None,      # captured at its own full size (fp8 config): 134.8 MB read + 494.1 MB written
+    "combine_kernel": 8 * (940_060_928 + 98_199_296),
 }
 
 
