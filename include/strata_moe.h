@@ -197,7 +197,10 @@ strata_status strata_device_status(strata_ctx *ctx, void *stream, strata_status 
 
 /* Whole path from HOST buffers with identity experts (BF16 contexts only): copies ids, x and
  * gate weights to the device buffers given in `dev`, runs layout -> dispatch -> combine with
- * y = recv, copies out back and synchronises the stream.  h_* are host pointers (pinned memory
+ * y = recv, copies out back and synchronises the stream.  Tokens travel in chunks of about 64 MB on
+ * two internal copy streams, so the upload of one chunk, the kernels of the previous one and the
+ * download of the one before overlap (streams and events are created on the first call; no device
+ * memory is allocated).  h_* are host pointers (pinned memory
  * makes the copies asynchronous); every member of `dev` is a device pointer owned by the caller,
  * dev->recv inside a registered region with room for N rows.  Used for end-to-end timing and
  * smoke checks; the paper has no counterpart (its operators take device buffers). */

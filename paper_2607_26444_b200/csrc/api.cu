@@ -1,5 +1,6 @@
 // C ABI: context, registration pool, argument validation and kernel launches.
 // Host-side only; every device-side step lives in layout.cu / dispatch.cu / combine.cu.
+#include <algorithm>
 #include <mutex>
 #include <new>
 #include <vector>
@@ -28,6 +29,10 @@ struct strata_ctx {
     uint64_t launches;
     uint64_t n_dispatch, n_combine;      // launches so far: their parity selects the work-claim counter
     strata::TraceBuf trace;
+    // host round trip only: copy streams and events, created on first use (no device memory)
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    std::vector<cudaEvent_t> ev_in, ev_done;
+    cudaEvent_t ev_entry = nullptr, ev_out = nullptr;
     std::vector<strata_region> regions;
     std::mutex mu;
 };
@@ -168,6 +173,15 @@ strata_status strata_ctx_create(strata_ctx** out, const strata_moe_shape* shape,
 strata_status strata_ctx_destroy(strata_ctx* ctx)
 {
     if (!ctx) return STRATA_ERR_INVALID_ARG;
+    if (ctx->device >= 0 && (ctx->s_in || ctx->ev_entry)) {
+        DeviceGuard g(ctx->device);
+        for (cudaEvent_t e : ctx->ev_in) cudaEventDestroy(e);
+        for (cudaEvent_t e : ctx->ev_done) cudaEventDestroy(e);
+        if (ctx->ev_entry) cudaEventDestroy(ctx->ev_entry);
+        if (ctx->ev_out) cudaEventDestroy(ctx->ev_out);
+        if (ctx->s_in) cudaStreamDestroy(ctx->s_in);
+        if (ctx->s_out) cudaStreamDestroy(ctx->s_out);
+    }
     delete ctx;
     return STRATA_OK;
 }
@@ -411,30 +425,98 @@ strata_status strata_moe_roundtrip_host(strata_ctx* ctx, const strata_moe_device
 {
     if (!ctx || !dev || !h_ids || !h_x || !h_w || !h_out) return STRATA_ERR_INVALID_ARG;
     if (!dev->ids || !dev->x || !dev->w || !dev->recv || !dev->out) return STRATA_ERR_INVALID_ARG;
+    strata_status rc = check_layout_ptrs(&dev->layout, true);
+    if (rc != STRATA_OK) return rc;
     const strata_moe_shape& s = ctx->shape;
     if (s.dispatch_dtype != STRATA_BF16) return STRATA_ERR_SHAPE;
+    if (!aligned16(dev->x) || !aligned16(dev->recv) || !aligned16(dev->out)) return STRATA_ERR_ALIGNMENT;
+    if (!ctx->ws) return STRATA_ERR_WORKSPACE;
+    const size_t n_tok = (size_t)s.R * s.T, n = n_tok * s.K, row_bytes = (size_t)s.H * 2;
+    {
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        if (!region_contains(ctx, dev->recv, n * row_bytes)) return STRATA_ERR_NOT_REGISTERED;
+    }
     if (ctx->device < 0) return STRATA_ERR_CUDA;
     DeviceGuard g(ctx->device);
     if (!g.ok) return STRATA_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t n_tok = (size_t)s.R * s.T, n = n_tok * s.K;
-    if (cudaMemcpyAsync(dev->ids, h_ids, n * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(dev->x, h_x, n_tok * s.H * 2, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(dev->w, h_w, n * sizeof(float), cudaMemcpyHostToDevice, st) != cudaSuccess) {
-        cudaGetLastError();
-        return STRATA_ERR_CUDA;
+
+    // Token chunks of about 64 MB of x: chunk c+1 travels to the device while chunk c is dispatched
+    // and combined and chunk c-1 travels back (the two copy directions use separate engines).
+    const size_t chunk_tok = std::max<size_t>(1, std::min(n_tok, ((size_t)64 << 20) / row_bytes));
+    const size_t n_chunks = (n_tok + chunk_tok - 1) / chunk_tok;
+#define STRATA_TRY(call) do { if ((call) != cudaSuccess) { cudaGetLastError(); return STRATA_ERR_CUDA; } } while (0)
+    if (!ctx->s_in) {
+        STRATA_TRY(cudaStreamCreateWithFlags(&ctx->s_in, cudaStreamNonBlocking));
+        STRATA_TRY(cudaStreamCreateWithFlags(&ctx->s_out, cudaStreamNonBlocking));
+        STRATA_TRY(cudaEventCreateWithFlags(&ctx->ev_entry, cudaEventDisableTiming));
+        STRATA_TRY(cudaEventCreateWithFlags(&ctx->ev_out, cudaEventDisableTiming));
     }
-    strata_status rc = strata_moe_layout(ctx, dev->ids, &dev->layout, stream);
-    if (rc != STRATA_OK) return rc;
-    rc = strata_moe_dispatch(ctx, &dev->layout, dev->x, dev->recv, nullptr, n, stream);
-    if (rc != STRATA_OK) return rc;
-    rc = strata_moe_combine(ctx, &dev->layout, dev->recv, n, dev->w, dev->out, stream);
-    if (rc != STRATA_OK) return rc;
-    if (cudaMemcpyAsync(h_out, dev->out, n_tok * s.H * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-        cudaStreamSynchronize(st) != cudaSuccess) {
-        cudaGetLastError();
-        return STRATA_ERR_CUDA;
+    while (ctx->ev_in.size() < n_chunks) {
+        cudaEvent_t a = nullptr, b = nullptr;
+        STRATA_TRY(cudaEventCreateWithFlags(&a, cudaEventDisableTiming));
+        ctx->ev_in.push_back(a);
+        STRATA_TRY(cudaEventCreateWithFlags(&b, cudaEventDisableTiming));
+        ctx->ev_done.push_back(b);
     }
+
+    // The copy-in stream starts where the caller's stream is now.  The small copies go first: copies
+    // in one direction are served in the order they were issued, whatever their stream.
+    STRATA_TRY(cudaEventRecord(ctx->ev_entry, st));
+    STRATA_TRY(cudaMemcpyAsync(dev->ids, h_ids, n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    STRATA_TRY(cudaMemcpyAsync(dev->w, h_w, n * sizeof(float), cudaMemcpyHostToDevice, st));
+    rc = strata_moe_layout(ctx, dev->ids, &dev->layout, stream);
+    if (rc != STRATA_OK) return rc;
+    STRATA_TRY(cudaStreamWaitEvent(ctx->s_in, ctx->ev_entry, 0));
+    const unsigned char* hx = static_cast<const unsigned char*>(h_x);
+    unsigned char* dx = static_cast<unsigned char*>(dev->x);
+    for (size_t c = 0; c < n_chunks; ++c) {
+        const size_t a = c * chunk_tok, cnt = std::min(chunk_tok, n_tok - a);
+        STRATA_TRY(cudaMemcpyAsync(dx + a * row_bytes, hx + a * row_bytes, cnt * row_bytes, cudaMemcpyHostToDevice,
+                                   ctx->s_in));
+        STRATA_TRY(cudaEventRecord(ctx->ev_in[c], ctx->s_in));
+    }
+
+    unsigned char* dout = static_cast<unsigned char*>(dev->out);
+    unsigned char* hout = static_cast<unsigned char*>(h_out);
+    for (size_t c = 0; c < n_chunks; ++c) {
+        const size_t a = c * chunk_tok, cnt = std::min(chunk_tok, n_tok - a);
+        strata_moe_shape sub = s;             // the chunk as a one-rank batch of cnt tokens
+        sub.R = 1;
+        sub.T = (int32_t)cnt;
+        STRATA_TRY(cudaStreamWaitEvent(st, ctx->ev_in[c], 0));
+        WorkQueue dq, cq;
+        {
+            std::lock_guard<std::mutex> lk(ctx->mu);
+            dq = dispatch_queue(ctx);
+            cq = combine_queue(ctx);
+        }
+        cudaError_t err = launch_dispatch_bf16(sub, dev->layout.dst_row + a * s.K, dx + a * row_bytes, dev->recv, n,
+                                               ctx->ws, dq, ctx->n_sm, TraceBuf{nullptr, 0}, st);
+        if (err == cudaSuccess)
+            err = launch_combine(sub, dev->layout.dst_row + a * s.K, dev->recv, n, dev->w + a * s.K,
+                                 dout + a * row_bytes, ctx->ws, cq, ctx->n_sm, TraceBuf{nullptr, 0}, st);
+        {
+            std::lock_guard<std::mutex> lk(ctx->mu);
+            ctx->launches += 2;
+            if (err == cudaSuccess) {
+                ctx->n_dispatch += 1;
+                ctx->n_combine += 1;
+            }
+        }
+        if (err != cudaSuccess) {
+            cudaGetLastError();
+            return STRATA_ERR_CUDA;
+        }
+        STRATA_TRY(cudaEventRecord(ctx->ev_done[c], st));
+        STRATA_TRY(cudaStreamWaitEvent(ctx->s_out, ctx->ev_done[c], 0));
+        STRATA_TRY(cudaMemcpyAsync(hout + a * row_bytes, dout + a * row_bytes, cnt * row_bytes, cudaMemcpyDeviceToHost,
+                                   ctx->s_out));
+    }
+    STRATA_TRY(cudaEventRecord(ctx->ev_out, ctx->s_out));
+    STRATA_TRY(cudaStreamWaitEvent(st, ctx->ev_out, 0));
+    STRATA_TRY(cudaStreamSynchronize(st));
+#undef STRATA_TRY
     return STRATA_OK;
 }
 

@@ -353,8 +353,11 @@ def test_zero_copy_rank_partitions():
     ctx.close()
 
 
-def test_roundtrip_from_host_buffers():
-    cfg = wl.CONFIGS["tiny"]
+@pytest.mark.parametrize("cfg", [wl.CONFIGS["tiny"],
+                                 # x is 168 MB: three upload chunks, the last one ragged
+                                 wl.shrink(wl.CONFIGS["tiny"], R=4, T=5000, H=4200, E=16, K=2, seed=5)],
+                         ids=["one-chunk", "three-chunks"])
+def test_roundtrip_from_host_buffers(cfg):
     inp = wl.generate(cfg)
     ctx = make_ctx(cfg)
     lay = ctx.new_layout()
@@ -374,8 +377,15 @@ def test_roundtrip_from_host_buffers():
                                      h_out.data_ptr(), torch.cuda.current_stream().cuda_stream)
     assert rc == 0
     ref_lay = oracle.layout(inp["ids"], cfg.E)
-    ref_recv = oracle.dispatch_bf16(ref_lay["dst_row"], inp["x"])
-    ref_out = oracle.combine(ref_lay["dst_row"], ref_recv, inp["w"])
+    ref_recv = oracle.dispatch_bf16(ref_lay["dst_row"], inp["x"], nthreads=8)
+    ref_out = oracle.combine(ref_lay["dst_row"], ref_recv, inp["w"], nthreads=8)
+    assert np.array_equal(h_out.numpy().view(np.uint16), ref_out)
+    assert np.array_equal(u16(recv), ref_recv)
+    # a second call on the same buffers (events and streams are reused)
+    h_out.zero_()
+    rc = B.strata_moe_roundtrip_host(ctx.h, dev, h_ids.data_ptr(), h_x.data_ptr(), h_w.data_ptr(),
+                                     h_out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    assert rc == 0
     assert np.array_equal(h_out.numpy().view(np.uint16), ref_out)
     assert ctx.device_status() == B.STRATA_OK
     ctx.close()
