@@ -44,6 +44,10 @@ def lib() -> ctypes.CDLL:
         L.oracle_combine.argtypes = [i64, i32, i32, vp, vp, vp, vp, i32]
         L.oracle_e4m3_encode.restype = ctypes.c_uint8
         L.oracle_e4m3_encode.argtypes = [ctypes.c_float]
+        L.oracle_partition.restype = i64
+        L.oracle_partition.argtypes = [i32, i32, i64, i32, vp, vp, vp, i32, i32, i32, i64, vp, vp, vp, vp, vp, vp]
+        L.oracle_dispatch_windows.restype = None
+        L.oracle_dispatch_windows.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.oracle_max_threads.restype = i32
         L.oracle_max_threads.argtypes = []
         _lib = L
@@ -143,3 +147,56 @@ def e4m3_encode(v: np.ndarray) -> np.ndarray:
     v = _c(v, np.float32)
     f = lib().oracle_e4m3_encode
     return np.fromiter((f(float(t)) for t in v.ravel()), dtype=np.uint8, count=v.size).reshape(v.shape)
+
+
+TIER_DTYPE = np.dtype([("alpha", np.int64), ("beta", np.int64), ("unit_rows", np.int64),
+                       ("fanout_cap", np.int32), ("pad", np.int32)])
+
+
+def make_tiers(tiers) -> np.ndarray:
+    """tiers: list of (alpha, beta, unit_rows, fanout_cap)."""
+    a = np.zeros(len(tiers), TIER_DTYPE)
+    for i, (al, be, ur, cap) in enumerate(tiers):
+        a[i] = (al, be, ur, cap, 0)
+    return a
+
+
+def partition(lay: Dict[str, np.ndarray], row_bytes: int, n_cores: int, tiers, g0: int = 1, g1: int = 1,
+              max_units: int = 1 << 16) -> Dict[str, np.ndarray]:
+    """Window partitioning + LPT-style list scheduling of dispatch (paper Sec. 6.2, App. B, C)."""
+    sec = _c(lay["src_expert_count"], np.int32)
+    R, E = sec.shape
+    off = _c(lay["expert_offset"], np.int32)
+    t = make_tiers(tiers)
+    out = {
+        "win_base": np.zeros((R, E), np.int32),
+        "unit_desc": np.zeros((max_units, 4), np.int32),
+        "unit_cost": np.zeros(max_units, np.int64),
+        "task_offset": np.zeros(n_cores + 1, np.int32),
+        "task_unit": np.zeros(max_units, np.int32),
+        "core_load": np.zeros(n_cores, np.int64),
+    }
+    U = lib().oracle_partition(R, E, row_bytes, n_cores, _p(sec), _p(off), _p(t), len(t), g0, g1, max_units,
+                               _p(out["win_base"]), _p(out["unit_desc"]), _p(out["unit_cost"]),
+                               _p(out["task_offset"]), _p(out["task_unit"]), _p(out["core_load"]))
+    if U < 0:
+        raise ValueError("more units than max_units")
+    out["n_units"] = int(U)
+    out["unit_desc"] = out["unit_desc"][:U]
+    out["unit_cost"] = out["unit_cost"][:U]
+    out["task_unit"] = out["task_unit"][:U]
+    return out
+
+
+def dispatch_windows(lay: Dict[str, np.ndarray], part: Dict[str, np.ndarray], x: np.ndarray, K: int) -> np.ndarray:
+    sec = _c(lay["src_expert_count"], np.int32)
+    R, E = sec.shape
+    H = x.shape[-1]
+    x2 = _c(x, np.uint16).reshape(-1, H)
+    n_cores = part["task_offset"].size - 1
+    recv = np.full((x2.shape[0] * K, H), 0xDEAD, np.uint16)
+    lib().oracle_dispatch_windows(R, E, K, H, n_cores, _p(sec), _p(_c(part["win_base"], np.int32)),
+                                  _p(_c(part["unit_desc"], np.int32)), _p(_c(part["task_offset"], np.int32)),
+                                  _p(_c(part["task_unit"], np.int32)), _p(_c(lay["src_of_row"], np.int32)),
+                                  _p(x2), _p(recv))
+    return recv

@@ -26,7 +26,10 @@
  * Pins (tests/test_oracle_*.py): sort-based brute force, a hand-worked
  * example, closed forms (E=1; round-robin ids), bijection/ordering invariants,
  * row-equality after dispatch, nearest-code brute force and a library cast for
- * the e4m3 encoder, identity/one-hot/K=1/doubling/fp64 checks for combine.
+ * the e4m3 encoder, identity/one-hot/K=1/doubling/fp64 checks for combine;
+ * for the partitioning: exact cover of the receive rows, Graham's tight LPT
+ * example, the 4/3 - 1/(3C) bound against a brute-force optimum, the fan-out
+ * cap, and equality of window-major with token-major dispatch.
  * No function here is "parity unpinned".
  *
  * Index convention: rank r in [0,R), token t in [0,T), slot k in [0,K),
@@ -273,6 +276,161 @@ void oracle_combine(int64_t n_tok, int32_t K, int32_t H,
                 acc = fmaf(w[n * K + k], bf16_to_f32(y[(size_t)row * H + c]), acc);
             }
             out[(size_t)n * H + c] = f32_to_bf16_rne(acc);
+        }
+}
+
+/* ------------------------------------------------------------------ */
+/* O5: hierarchical workload partitioning for dispatch (paper Sec. 6.2, */
+/* App. B and C).                                                       */
+/*  level 2, expert-window aggregation: the rows that source rank r     */
+/*    sends to expert e form one contiguous window of the receive       */
+/*    buffer, win_base[r][e] .. + src_expert_count[r][e].               */
+/*  level 3, peer-window partitioning: the expert windows of source r   */
+/*    towards the experts of destination rank d, concatenated in expert */
+/*    order, form the peer window (r,d) of B rows; it is cut into       */
+/*    n = ceil(B / S_t) transfer units of at most S_t rows, S_t the     */
+/*    unit size of the tier of (r,d).  Unit ids enumerate (r, d, k).    */
+/*  cost of a unit of s bytes (Sec. 6.2): tau = alpha_t + ceil(s/beta_t)*/
+/*    in integer cost units.                                            */
+/*  list scheduling (Sec. 6.2, App. B "LPT-style"): units sorted by     */
+/*    cost, largest first (ties: lower unit id first); each unit goes   */
+/*    to the least-loaded core (ties: lower core id) among the cores    */
+/*    whose next issue stripe still has room for the unit's destination */
+/*    rank, F[stripe][d] < H_t; a core's stripe index is the number of  */
+/*    units it already holds.  If no core is feasible the cap is        */
+/*    relaxed for that unit (this build's reading: the paper does not   */
+/*    say what happens then).                                           */
+/* Tiers (stand-in for the fabric's die / node / inter-node levels):    */
+/*   tier(r,d) = 0 if r/g0 == d/g0, else 1 if r/g1 == d/g1, else 2,     */
+/*   clamped to n_tiers-1.                                              */
+/* Returns the number of units, or -1 if it exceeds max_units.          */
+/* ------------------------------------------------------------------ */
+typedef struct {
+    int64_t alpha;        /* fixed cost of one unit                    */
+    int64_t beta;         /* bytes moved per cost unit                 */
+    int64_t unit_rows;    /* S_t in rows (>= 1)                        */
+    int32_t fanout_cap;   /* H_t                                       */
+    int32_t pad;
+} oracle_tier;
+
+static int32_t tier_of(int32_t r, int32_t d, int32_t g0, int32_t g1, int32_t n_tiers)
+{
+    int32_t t = (r / g0 == d / g0) ? 0 : (r / g1 == d / g1) ? 1 : 2;
+    return t < n_tiers ? t : n_tiers - 1;
+}
+
+int64_t oracle_partition(int32_t R, int32_t E, int64_t row_bytes, int32_t n_cores,
+                         const int32_t *src_expert_count,   /* [R,E]          */
+                         const int32_t *expert_offset,      /* [E+1]          */
+                         const oracle_tier *tiers, int32_t n_tiers, int32_t g0, int32_t g1,
+                         int64_t max_units,
+                         int32_t *win_base,                 /* [R,E]          */
+                         int32_t *unit_desc,                /* [max_units,4]: src, dst, first logical row, rows */
+                         int64_t *unit_cost,                /* [max_units]    */
+                         int32_t *task_offset,              /* [n_cores+1]    */
+                         int32_t *task_unit,                /* [max_units]    */
+                         int64_t *core_load)                /* [n_cores]      */
+{
+    const int32_t E_loc = E / R;
+    /* level 2: base row of every expert window */
+    for (int32_t e = 0; e < E; ++e) {
+        int32_t row = expert_offset[e];
+        for (int32_t r = 0; r < R; ++r) {
+            win_base[r * E + e] = row;
+            row += src_expert_count[r * E + e];
+        }
+    }
+    /* level 3: peer windows -> units with their cost */
+    int64_t U = 0;
+    for (int32_t r = 0; r < R; ++r)
+        for (int32_t d = 0; d < R; ++d) {
+            int64_t B = 0;
+            for (int32_t e = d * E_loc; e < (d + 1) * E_loc; ++e) B += src_expert_count[r * E + e];
+            const oracle_tier *t = &tiers[tier_of(r, d, g0, g1, n_tiers)];
+            for (int64_t a = 0; a < B; a += t->unit_rows) {
+                const int64_t rows = (B - a < t->unit_rows) ? B - a : t->unit_rows;
+                if (U >= max_units) return -1;
+                unit_desc[U * 4 + 0] = r;
+                unit_desc[U * 4 + 1] = d;
+                unit_desc[U * 4 + 2] = (int32_t)a;
+                unit_desc[U * 4 + 3] = (int32_t)rows;
+                unit_cost[U] = t->alpha + (rows * row_bytes + t->beta - 1) / t->beta;
+                ++U;
+            }
+        }
+    /* order: largest cost first, ties by unit id (insertion sort on an index array: plain and stable) */
+    int32_t *order = (int32_t *)malloc((size_t)(U > 0 ? U : 1) * sizeof(int32_t));
+    for (int64_t j = 0; j < U; ++j) {
+        int64_t k = j;
+        while (k > 0 && unit_cost[order[k - 1]] < unit_cost[j]) {
+            order[k] = order[k - 1];
+            --k;
+        }
+        order[k] = (int32_t)j;
+    }
+    /* list scheduling under the stripe-level fan-out cap */
+    int32_t *len = (int32_t *)calloc((size_t)n_cores, sizeof(int32_t));
+    int32_t *fan = (int32_t *)calloc((size_t)(U > 0 ? U : 1) * R, sizeof(int32_t));   /* F[stripe][d] */
+    int32_t *core_of = (int32_t *)malloc((size_t)(U > 0 ? U : 1) * sizeof(int32_t));
+    int32_t *stripe_of = (int32_t *)malloc((size_t)(U > 0 ? U : 1) * sizeof(int32_t));
+    for (int32_t c = 0; c < n_cores; ++c) core_load[c] = 0;
+    for (int64_t o = 0; o < U; ++o) {
+        const int32_t j = order[o];
+        const int32_t r = unit_desc[j * 4 + 0], d = unit_desc[j * 4 + 1];
+        const int32_t cap = tiers[tier_of(r, d, g0, g1, n_tiers)].fanout_cap;
+        int32_t best = -1, best_any = 0;
+        for (int32_t c = 0; c < n_cores; ++c) {
+            if (core_load[c] < core_load[best_any]) best_any = c;
+            if (fan[(int64_t)len[c] * R + d] < cap && (best < 0 || core_load[c] < core_load[best])) best = c;
+        }
+        if (best < 0) best = best_any;
+        core_of[j] = best;
+        stripe_of[j] = len[best];
+        fan[(int64_t)len[best] * R + d] += 1;
+        len[best] += 1;
+        core_load[best] += unit_cost[j];
+    }
+    /* per-core task lists in issue order */
+    task_offset[0] = 0;
+    for (int32_t c = 0; c < n_cores; ++c) task_offset[c + 1] = task_offset[c] + len[c];
+    for (int64_t j = 0; j < U; ++j) task_unit[task_offset[core_of[j]] + stripe_of[j]] = (int32_t)j;
+    free(order);
+    free(len);
+    free(fan);
+    free(core_of);
+    free(stripe_of);
+    return U;
+}
+
+/* O6: window-major dispatch following the task lists: every core copies the rows of its units,
+ * one source row per receive row (found through src_of_row).  Must produce exactly what O2 does. */
+void oracle_dispatch_windows(int32_t R, int32_t E, int32_t K, int32_t H, int32_t n_cores,
+                             const int32_t *src_expert_count, const int32_t *win_base,
+                             const int32_t *unit_desc, const int32_t *task_offset, const int32_t *task_unit,
+                             const int32_t *src_of_row, const uint16_t *x, uint16_t *recv)
+{
+    const int32_t E_loc = E / R;
+    for (int32_t c = 0; c < n_cores; ++c)
+        for (int32_t q = task_offset[c]; q < task_offset[c + 1]; ++q) {
+            const int32_t j = task_unit[q];
+            const int32_t r = unit_desc[j * 4 + 0], d = unit_desc[j * 4 + 1];
+            int64_t first = unit_desc[j * 4 + 2], rows = unit_desc[j * 4 + 3];
+            /* walk the peer window (r,d): expert windows of d's experts in order */
+            for (int32_t e = d * E_loc; e < (d + 1) * E_loc && rows > 0; ++e) {
+                const int64_t cnt = src_expert_count[r * E + e];
+                if (first >= cnt) {
+                    first -= cnt;
+                    continue;
+                }
+                const int64_t take = (cnt - first < rows) ? cnt - first : rows;
+                for (int64_t i = 0; i < take; ++i) {
+                    const int64_t row = win_base[r * E + e] + first + i;
+                    const int64_t tok = src_of_row[row] / K;
+                    memcpy(recv + (size_t)row * H, x + (size_t)tok * H, (size_t)H * 2);
+                }
+                rows -= take;
+                first = 0;
+            }
         }
 }
 
