@@ -318,6 +318,63 @@ def cta_finish_spread(case: DeviceCase):
     return out
 
 
+def window_partitioning_report(cfg: wl.MoEConfig, dev_index: int, unit_rows: int, n_cores: int = 296):
+    """The paper's static scheme (expert windows -> peer windows -> LPT-style task lists, Sec. 6.2) run on
+    the same inputs as the default path: policy generation time, window-major dispatch time, predicted
+    imbalance of the policy and measured per-CTA finish spread."""
+    import torch
+    from paper_2607_26444_b200 import binding as B
+    dev = torch.device("cuda", dev_index)
+    inp = wl.generate(cfg) if cfg.n_tok <= 20000 else None
+    ctx = B.MoEContext(cfg.R, cfg.T, cfg.H, cfg.E, cfg.K, device=dev_index)
+    ids = torch.from_numpy(inp["ids"] if inp else wl.gen_topk_ids(cfg)).to(dev)
+    x = (torch.from_numpy(inp["x"].view(np.int16)).to(dev) if inp
+         else torch.randint(-30000, 30000, (cfg.n_tok, cfg.H), dtype=torch.int16, device=dev))
+    lay = ctx.layout(ids)
+    recv = torch.empty((cfg.n_items, cfg.H), dtype=torch.int16, device=dev)
+    ctx.register(recv)
+    # one tier (HBM is uniform): cost in ns, alpha = 1 us per unit, beta = 22 B/ns per core
+    pol = B.make_policy([(1000, 22, unit_rows, n_cores)])
+    part = ctx.partition(lay, pol, n_cores)
+    torch.cuda.synchronize()
+
+    def timeit(fn, iters=10):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+        torch.cuda._sleep(10_000_000)
+        ev[0].record()
+        for i in range(iters):
+            fn()
+            ev[i + 1].record()
+        torch.cuda.synchronize()
+        ts = sorted(ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(iters))
+        return ts[len(ts) // 2]
+
+    policy_us = timeit(lambda: ctx.partition(lay, pol, n_cores, part))
+    win_us = timeit(lambda: ctx.dispatch_windows(lay, part, x, recv))
+    tok_us = timeit(lambda: ctx.dispatch(lay, x, recv))
+    load = part.core_load.cpu().numpy().astype(np.float64)
+    tr = ctx.trace(2048)
+    tr.zero_()
+    ctx.dispatch_windows(lay, part, x, recv)
+    torch.cuda.synchronize()
+    rec = tr.cpu().numpy()
+    used = rec[rec[:, 0] != 0]
+    spread = float(used[:, 1].max() - used[:, 1].min()) / float(used[:, 1].max() - used[:, 0].min())
+    ctx.trace_off()
+    st = ctx.device_status()
+    out = {"units": int(part.n_units.item()), "unit_rows": unit_rows, "cores": n_cores,
+           "policy_us": round(policy_us, 1), "window_dispatch_us": round(win_us, 1),
+           "window_dispatch_GBs": round(cfg.dispatch_bytes() / win_us / 1e3, 1),
+           "token_dispatch_us": round(tok_us, 1),
+           "predicted_imbalance_max_over_mean": round(float(load.max() / load.mean()), 4),
+           "cta_finish_spread": round(spread, 4), "device_status": st}
+    ctx.close()
+    return out
+
+
 def run_gpu(args, rank: int, local_rank: int, world: int):
     import torch
     import torch.distributed as dist
@@ -485,6 +542,13 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
                 dc = uc
             del dc
             torch.cuda.empty_cache()
+
+    if not args.no_other:
+        other["paper_window_partitioning"] = {
+            "skew": window_partitioning_report(wl.CONFIGS["skew"], local_rank, unit_rows=64),
+            "prefill": window_partitioning_report(wl.CONFIGS["prefill"], local_rank, unit_rows=128),
+        }
+        torch.cuda.empty_cache()
 
     cpu = None
     if not args.no_cpu:

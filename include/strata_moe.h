@@ -187,6 +187,62 @@ strata_status strata_moe_dispatch(strata_ctx *ctx, const strata_moe_layout_t *la
 strata_status strata_moe_combine(strata_ctx *ctx, const strata_moe_layout_t *layout, const void *y,
                                  size_t y_rows, const float *topk_w, void *out, void *stream);
 
+/* ---- optional: the paper's hierarchical workload partitioning (Sec. 6.2, App. B and C) -----------
+ * The default dispatch balances at run time by ordered work claiming.  These two calls build and run
+ * the paper's own static scheme instead, so that it can be compared on this hardware:
+ *   expert windows  (source rank r, expert e): src_expert_count[r][e] contiguous receive rows starting
+ *                   at win_base[r][e];
+ *   peer windows    (r -> destination rank d): the expert windows of d's experts in expert order, cut
+ *                   into transfer units of at most unit_rows rows of the tier of (r,d);
+ *                   tier(r,d) = 0 if r/g0 == d/g0, else 1 if r/g1 == d/g1, else 2 (clamped to n_tiers-1);
+ *   unit cost       tau = alpha + ceil(bytes / beta), integers;
+ *   policy          LPT-style list scheduling: units by decreasing cost (ties: lower unit id) onto the
+ *                   least-loaded core (ties: lower core id) among the cores whose next issue stripe
+ *                   (= number of units the core already holds) has fewer than fanout_cap units for the
+ *                   unit's destination rank; if no core qualifies the cap is waived for that unit.
+ * Unit ids enumerate (r, d, k) in that order. */
+typedef struct {
+    int64_t alpha;        /* fixed cost of a unit, 0 <= alpha < 2^30                      */
+    int64_t beta;         /* bytes per cost unit, >= 1                                    */
+    int64_t unit_rows;    /* S_t in rows, >= 1; unit_rows * row_bytes / beta < 2^36       */
+    int32_t fanout_cap;   /* H_t >= 1                                                     */
+    int32_t reserved;
+} strata_tier;
+typedef struct {
+    int32_t n_tiers;      /* 1..3 */
+    int32_t g0, g1;       /* ranks per innermost group and per middle group, >= 1         */
+    int32_t reserved;
+    strata_tier tiers[3];
+} strata_partition_policy;
+typedef struct {            /* all device pointers, caller-owned */
+    int32_t *win_base;      /* [R,E]            first receive row of expert window (r,e)              */
+    int32_t *unit_desc;     /* [max_units,4]    source rank, destination rank, first logical row, rows */
+    int64_t *unit_cost;     /* [max_units]                                                            */
+    int32_t *n_units;       /* [1]              number of units; -1 if they did not fit                */
+    int32_t *task_offset;   /* [n_cores+1]      core c's list is task_unit[task_offset[c] .. [c+1])    */
+    int32_t *task_unit;     /* [max_units]      unit ids, core-major, in issue order                   */
+    int64_t *core_load;     /* [n_cores]        predicted load of each core                            */
+    int32_t *scratch;       /* [max_units*(R+2)] working memory of the policy kernel                   */
+} strata_partition_t;
+
+/* Upper bound of the unit count for a shape and policy (host arithmetic only):
+ * sum over tiers is bounded by N / min(unit_rows) + R*R. */
+strata_status strata_moe_partition_max_units(const strata_moe_shape *shape, const strata_partition_policy *policy,
+                                             size_t *max_units);
+/* Generates the policy on the GPU (one launch, one CTA) from a layout that includes src_expert_count.
+ * Limits: at most 8192 units and 1024 cores; more units raise STRATA_ERR_CAPACITY on the device status
+ * and set *n_units = -1 (choose larger units).  Host errors: INVALID_ARG, SHAPE, WORKSPACE, CAPACITY. */
+strata_status strata_moe_partition(strata_ctx *ctx, const strata_moe_layout_t *layout,
+                                   const strata_partition_policy *policy, int32_t n_cores,
+                                   const strata_partition_t *out, size_t max_units, void *stream);
+/* Window-major bf16 dispatch: n_cores one-warp CTAs, CTA c copies the rows of the units in its task
+ * list in order, one source row (found through layout->src_of_row, which must be present) per
+ * receive row.  Writes exactly what strata_moe_dispatch writes.  Same registration, alignment and
+ * capacity rules; rows of at most 16 KB. */
+strata_status strata_moe_dispatch_windows(strata_ctx *ctx, const strata_moe_layout_t *layout,
+                                          const strata_partition_t *partition, int32_t n_cores, const void *x,
+                                          void *recv, size_t capacity_rows, void *stream);
+
 /* Host helper: rank d's partition of the receive buffer, from a HOST copy of rank_offset[R+1]:
  * *rank_base = recv + rank_offset[d] * row_bytes, *rows = rank_offset[d+1] - rank_offset[d]. */
 strata_status strata_moe_recv_view(strata_ctx *ctx, const int32_t *h_rank_offset, int rank,

@@ -36,6 +36,7 @@ EXPORTS = [
     "strata_pool_unregister", "strata_pool_carve", "strata_pool_reset", "strata_moe_layout",
     "strata_moe_dispatch", "strata_moe_combine", "strata_moe_recv_view", "strata_device_status",
     "strata_moe_roundtrip_host", "strata_moe_layout_noalloc", "strata_ctx_set_trace",
+    "strata_moe_partition_max_units", "strata_moe_partition", "strata_moe_dispatch_windows",
 ]
 
 
@@ -54,6 +55,31 @@ class strata_moe_layout_t(ctypes.Structure):
 class strata_moe_device_buffers(ctypes.Structure):
     _fields_ = [("ids", ctypes.c_void_p), ("x", ctypes.c_void_p), ("w", ctypes.c_void_p),
                 ("recv", ctypes.c_void_p), ("out", ctypes.c_void_p), ("layout", strata_moe_layout_t)]
+
+
+class strata_tier(ctypes.Structure):
+    _fields_ = [("alpha", ctypes.c_int64), ("beta", ctypes.c_int64), ("unit_rows", ctypes.c_int64),
+                ("fanout_cap", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class strata_partition_policy(ctypes.Structure):
+    _fields_ = [("n_tiers", ctypes.c_int32), ("g0", ctypes.c_int32), ("g1", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("tiers", strata_tier * 3)]
+
+
+class strata_partition_t(ctypes.Structure):
+    _fields_ = [("win_base", ctypes.c_void_p), ("unit_desc", ctypes.c_void_p), ("unit_cost", ctypes.c_void_p),
+                ("n_units", ctypes.c_void_p), ("task_offset", ctypes.c_void_p), ("task_unit", ctypes.c_void_p),
+                ("core_load", ctypes.c_void_p), ("scratch", ctypes.c_void_p)]
+
+
+def make_policy(tiers, g0: int = 1, g1: int = 1) -> strata_partition_policy:
+    """tiers: list of (alpha, beta, unit_rows, fanout_cap), at most 3."""
+    p = strata_partition_policy()
+    p.n_tiers, p.g0, p.g1 = len(tiers), g0, g1
+    for i, (a, be, ur, cap) in enumerate(tiers):
+        p.tiers[i] = strata_tier(a, be, ur, cap, 0)
+    return p
 
 
 class StrataError(RuntimeError):
@@ -97,6 +123,10 @@ def lib() -> ctypes.CDLL:
         "strata_moe_roundtrip_host": [vp, P(strata_moe_device_buffers), vp, vp, vp, vp, vp],
         "strata_moe_layout_noalloc": [P(strata_moe_shape), vp, P(strata_moe_layout_t), vp, vp],
         "strata_ctx_set_trace": [vp, vp, sz],
+        "strata_moe_partition_max_units": [P(strata_moe_shape), P(strata_partition_policy), P(sz)],
+        "strata_moe_partition": [vp, P(strata_moe_layout_t), P(strata_partition_policy), i32,
+                                 P(strata_partition_t), sz, vp],
+        "strata_moe_dispatch_windows": [vp, P(strata_moe_layout_t), P(strata_partition_t), i32, vp, vp, sz, vp],
     }
     for name, args in sigs.items():
         fn = getattr(L, name)
@@ -207,6 +237,24 @@ def strata_moe_layout_noalloc(shape: strata_moe_shape, topk_ids: int, layout: st
                                            stream)
 
 
+def strata_moe_partition_max_units(shape: strata_moe_shape, policy: strata_partition_policy) -> Tuple[int, int]:
+    n = ctypes.c_size_t()
+    rc = lib().strata_moe_partition_max_units(ctypes.byref(shape), ctypes.byref(policy), ctypes.byref(n))
+    return rc, n.value
+
+
+def strata_moe_partition(ctx, layout: strata_moe_layout_t, policy: strata_partition_policy, n_cores: int,
+                         out: strata_partition_t, max_units: int, stream: int) -> int:
+    return lib().strata_moe_partition(ctx, ctypes.byref(layout), ctypes.byref(policy), n_cores, ctypes.byref(out),
+                                      max_units, stream)
+
+
+def strata_moe_dispatch_windows(ctx, layout: strata_moe_layout_t, partition: strata_partition_t, n_cores: int,
+                                x: int, recv: int, capacity_rows: int, stream: int) -> int:
+    return lib().strata_moe_dispatch_windows(ctx, ctypes.byref(layout), ctypes.byref(partition), n_cores, x, recv,
+                                             capacity_rows, stream)
+
+
 # ---- convenience wrapper over torch tensors (memory + streams only) ---------
 
 def _check(rc: int, where: str) -> None:
@@ -233,6 +281,27 @@ class Layout:
             self.src_expert_count.data_ptr() if with_optional else None,
             self.dst_row.data_ptr(),
             self.src_of_row.data_ptr() if with_optional else None)
+
+
+class Partition:
+    """Device tensors of a window-partitioning policy, plus the C struct pointing at them."""
+
+    def __init__(self, R: int, E: int, n_cores: int, max_units: int, device):
+        import torch
+        i32 = dict(dtype=torch.int32, device=device)
+        i64 = dict(dtype=torch.int64, device=device)
+        self.n_cores, self.max_units = n_cores, max_units
+        self.win_base = torch.zeros((R, E), **i32)
+        self.unit_desc = torch.zeros((max_units, 4), **i32)
+        self.unit_cost = torch.zeros(max_units, **i64)
+        self.n_units = torch.zeros(1, **i32)
+        self.task_offset = torch.zeros(n_cores + 1, **i32)
+        self.task_unit = torch.zeros(max_units, **i32)
+        self.core_load = torch.zeros(n_cores, **i64)
+        self.scratch = torch.zeros(max_units * (R + 2), **i32)
+        self.c = strata_partition_t(self.win_base.data_ptr(), self.unit_desc.data_ptr(), self.unit_cost.data_ptr(),
+                                    self.n_units.data_ptr(), self.task_offset.data_ptr(), self.task_unit.data_ptr(),
+                                    self.core_load.data_ptr(), self.scratch.data_ptr())
 
 
 class MoEContext:
@@ -326,6 +395,21 @@ class MoEContext:
     def trace_off(self) -> None:
         _check(strata_ctx_set_trace(self.h, None, 0), "strata_ctx_set_trace")
         self._trace = None
+
+    # the paper's static window partitioning, as an alternative to run-time work claiming ------------
+    def partition(self, layout: Layout, policy: strata_partition_policy, n_cores: int,
+                  part: Optional[Partition] = None) -> Partition:
+        if part is None:
+            rc, mu = strata_moe_partition_max_units(self.shape, policy)
+            _check(rc, "strata_moe_partition_max_units")
+            part = Partition(self.R, self.E, n_cores, mu, self.device)
+        _check(strata_moe_partition(self.h, layout.c, policy, n_cores, part.c, part.max_units, self._stream()),
+               "strata_moe_partition")
+        return part
+
+    def dispatch_windows(self, layout: Layout, part: Partition, x, recv) -> None:
+        _check(strata_moe_dispatch_windows(self.h, layout.c, part.c, part.n_cores, x.data_ptr(), recv.data_ptr(),
+                                           recv.shape[0], self._stream()), "strata_moe_dispatch_windows")
 
     def device_status(self) -> int:
         rc, st = strata_device_status(self.h, self._stream())

@@ -10,6 +10,7 @@
 namespace strata {
 cudaError_t configure_layout_kernels();
 cudaError_t configure_dispatch_kernels();
+cudaError_t configure_partition_kernels();
 }  // namespace strata
 
 struct strata_region {
@@ -150,7 +151,8 @@ strata_status strata_ctx_create(strata_ctx** out, const strata_moe_shape* shape,
         if (!g.ok) return STRATA_ERR_CUDA;
         if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
             return STRATA_ERR_CUDA;
-        if (configure_layout_kernels() != cudaSuccess || configure_dispatch_kernels() != cudaSuccess) {
+        if (configure_layout_kernels() != cudaSuccess || configure_dispatch_kernels() != cudaSuccess ||
+            configure_partition_kernels() != cudaSuccess) {
             cudaGetLastError();
             return STRATA_ERR_CUDA;
         }
@@ -378,6 +380,94 @@ strata_status strata_moe_combine(strata_ctx* ctx, const strata_moe_layout_t* lay
         std::lock_guard<std::mutex> lk(ctx->mu);
         ctx->launches += 1;
         if (err == cudaSuccess) ctx->n_combine += 1;
+    }
+    return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
+}
+
+namespace {
+strata_status check_policy(const strata_moe_shape& s, const strata_partition_policy* pol)
+{
+    if (!pol) return STRATA_ERR_INVALID_ARG;
+    if (pol->n_tiers < 1 || pol->n_tiers > 3 || pol->g0 < 1 || pol->g1 < 1) return STRATA_ERR_INVALID_ARG;
+    for (int t = 0; t < pol->n_tiers; ++t) {
+        const strata_tier& q = pol->tiers[t];
+        if (q.alpha < 0 || q.alpha >= (1ll << 30) || q.beta < 1 || q.unit_rows < 1 || q.fanout_cap < 1)
+            return STRATA_ERR_INVALID_ARG;
+        if (q.unit_rows > (1ll << 31)) return STRATA_ERR_INVALID_ARG;
+        if (q.unit_rows * ((long long)s.H * 2) / q.beta >= (1ll << 36)) return STRATA_ERR_INVALID_ARG;
+    }
+    return STRATA_OK;
+}
+}  // namespace
+
+strata_status strata_moe_partition_max_units(const strata_moe_shape* shape, const strata_partition_policy* policy,
+                                             size_t* max_units)
+{
+    if (!max_units) return STRATA_ERR_INVALID_ARG;
+    strata_status st = check_shape(shape);
+    if (st != STRATA_OK) return st;
+    st = check_policy(*shape, policy);
+    if (st != STRATA_OK) return st;
+    long long smin = policy->tiers[0].unit_rows;
+    for (int t = 1; t < policy->n_tiers; ++t) smin = std::min<long long>(smin, policy->tiers[t].unit_rows);
+    const long long n = (long long)shape->R * shape->T * shape->K;
+    *max_units = (size_t)(n / smin + (long long)shape->R * shape->R);
+    return STRATA_OK;
+}
+
+strata_status strata_moe_partition(strata_ctx* ctx, const strata_moe_layout_t* layout,
+                                   const strata_partition_policy* policy, int32_t n_cores,
+                                   const strata_partition_t* out, size_t max_units, void* stream)
+{
+    if (!ctx || !layout || !out) return STRATA_ERR_INVALID_ARG;
+    if (!layout->src_expert_count || !layout->expert_offset) return STRATA_ERR_INVALID_ARG;
+    if (!out->win_base || !out->unit_desc || !out->unit_cost || !out->n_units || !out->task_offset ||
+        !out->task_unit || !out->core_load || !out->scratch)
+        return STRATA_ERR_INVALID_ARG;
+    strata_status st = check_policy(ctx->shape, policy);
+    if (st != STRATA_OK) return st;
+    if (n_cores < 1 || n_cores > partition_max_cores_supported()) return STRATA_ERR_SHAPE;
+    if (max_units < 1 || max_units > (size_t)1 << 20) return STRATA_ERR_CAPACITY;
+    if (!ctx->ws) return STRATA_ERR_WORKSPACE;
+    if (ctx->device < 0) return STRATA_ERR_CUDA;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return STRATA_ERR_CUDA;
+    cudaError_t err = launch_partition(ctx->shape, *layout, *policy, n_cores, *out, max_units, ctx->ws,
+                                       static_cast<cudaStream_t>(stream));
+    {
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        ctx->launches += 1;
+    }
+    return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
+}
+
+strata_status strata_moe_dispatch_windows(strata_ctx* ctx, const strata_moe_layout_t* layout,
+                                          const strata_partition_t* partition, int32_t n_cores, const void* x,
+                                          void* recv, size_t capacity_rows, void* stream)
+{
+    if (!ctx || !layout || !partition || !x || !recv) return STRATA_ERR_INVALID_ARG;
+    if (!layout->src_expert_count || !layout->src_of_row) return STRATA_ERR_INVALID_ARG;
+    if (!partition->win_base || !partition->unit_desc || !partition->task_offset || !partition->task_unit)
+        return STRATA_ERR_INVALID_ARG;
+    const strata_moe_shape& s = ctx->shape;
+    if (s.dispatch_dtype != STRATA_BF16 || (uint32_t)s.H * 2u > windows_max_row_bytes()) return STRATA_ERR_SHAPE;
+    if (n_cores < 1 || n_cores > partition_max_cores_supported()) return STRATA_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(recv)) return STRATA_ERR_ALIGNMENT;
+    if (!ctx->ws) return STRATA_ERR_WORKSPACE;
+    const size_t n_rows = (size_t)s.R * s.T * s.K;
+    if (capacity_rows < n_rows) return STRATA_ERR_CAPACITY;
+    {
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        if (!region_contains(ctx, recv, capacity_rows * (size_t)s.H * 2)) return STRATA_ERR_NOT_REGISTERED;
+    }
+    if (ctx->device < 0) return STRATA_ERR_CUDA;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return STRATA_ERR_CUDA;
+    cudaError_t err = launch_dispatch_windows(s, *layout, *partition, n_cores, x, recv, capacity_rows, ctx->ws,
+                                              ctx->trace, static_cast<cudaStream_t>(stream));
+    {
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        ctx->launches += 1;
     }
     return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
 }

@@ -72,7 +72,15 @@ cudaError_t launch_dispatch_fp8(const strata_moe_shape& s, const int32_t* dst_ro
 cudaError_t launch_combine(const strata_moe_shape& s, const int32_t* dst_row, const void* y, size_t y_rows,
                            const float* w, void* out, int* status, WorkQueue wq, int n_sm, TraceBuf trace,
                            cudaStream_t st);
-cudaError_t configure_kernels(int device);
+cudaError_t launch_partition(const strata_moe_shape& s, const strata_moe_layout_t& L,
+                             const strata_partition_policy& pol, int n_cores, const strata_partition_t& out,
+                             size_t max_units, int* status, cudaStream_t st);
+cudaError_t launch_dispatch_windows(const strata_moe_shape& s, const strata_moe_layout_t& L,
+                                    const strata_partition_t& part, int n_cores, const void* x, void* recv,
+                                    size_t capacity_rows, int* status, TraceBuf trace, cudaStream_t st);
+int partition_max_units_supported();
+int partition_max_cores_supported();
+uint32_t windows_max_row_bytes();
 
 #ifdef __CUDACC__
 // ---- programmatic dependent launch ---------------------------------------------

@@ -1,0 +1,540 @@
+// Hierarchical workload partitioning for dispatch, the paper's own scheme (Sec. 6.2, App. B and C), as
+// an optional work-assignment variant next to the default ordered work claiming:
+//   level 2  expert-window aggregation: rows that source rank r sends to expert e are one contiguous
+//            window of the receive buffer (win_base[r][e], src_expert_count[r][e] rows);
+//   level 3  peer-window partitioning: the expert windows of (source r -> destination rank d),
+//            concatenated in expert order, are cut into transfer units of at most S_t rows, t the tier
+//            of (r,d); cost tau = alpha_t + ceil(bytes / beta_t);
+//   policy   LPT-style list scheduling: units by decreasing cost onto the least-loaded core whose next
+//            issue stripe still has room for the unit's destination rank (fan-out cap H_t); the output
+//            is one task list per core, which the window-major dispatch kernel simply follows.
+// The policy is generated ON the GPU by one CTA (no host round trip): a bitonic sort of the units and a
+// sequential greedy loop whose "least-loaded feasible core" step is a block-wide arg-min.
+#include "common.cuh"
+
+namespace strata {
+
+namespace {
+
+constexpr int kPartThreads = 1024;
+constexpr int kPartMaxUnits = 8192;       // sort keys live in shared memory
+constexpr int kPartMaxCores = 1024;       // one thread per core in the arg-min
+constexpr int kFanSmemInts = 12288;       // fan-out counts F[stripe][dest] kept in shared memory
+constexpr int kMaxTiers = 3;
+
+struct PartitionParams {
+    const int32_t* src_expert_count;   // [R,E]
+    const int32_t* expert_offset;      // [E+1]
+    int32_t* win_base;                 // [R,E]
+    int32_t* unit_desc;                // [max_units,4]
+    long long* unit_cost;              // [max_units]
+    int32_t* n_units;                  // [1]
+    int32_t* task_offset;              // [n_cores+1]
+    int32_t* task_unit;                // [max_units]
+    long long* core_load;              // [n_cores]
+    int32_t* scratch;                  // [2*max_units + max_units*R]: core_of | stripe_of | fan-out overflow
+    int* status;
+    int R, E, e_loc, n_cores, max_units, n_tiers, g0, g1;
+    long long row_bytes;
+    long long alpha[kMaxTiers], beta[kMaxTiers], unit_rows[kMaxTiers];
+    int cap[kMaxTiers];
+};
+
+__device__ __forceinline__ int tier_of(const PartitionParams& p, int r, int d)
+{
+    const int t = (r / p.g0 == d / p.g0) ? 0 : (r / p.g1 == d / p.g1) ? 1 : 2;
+    return min(t, p.n_tiers - 1);
+}
+
+__global__ void __launch_bounds__(kPartThreads) partition_kernel(PartitionParams p)
+{
+    extern __shared__ unsigned long long sm64[];
+    unsigned long long* keys = sm64;                                   // [kPartMaxUnits] sort keys
+    long long* load = reinterpret_cast<long long*>(keys + kPartMaxUnits);   // [kPartMaxCores]
+    int* len = reinterpret_cast<int*>(load + kPartMaxCores);               // [kPartMaxCores]
+    int* fan = len + kPartMaxCores;                                         // [kFanSmemInts]
+    int* scan = fan + kFanSmemInts;                                         // [kPartThreads + 34]
+    __shared__ int s_total;
+
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int R = p.R, E = p.E;
+    griddep_wait();
+    griddep_launch_dependents();
+
+    // ---- level 2: base row of every expert window ----
+    for (int e = tid; e < E; e += kPartThreads) {
+        int row = p.expert_offset[e];
+        for (int r = 0; r < R; ++r) {
+            p.win_base[r * E + e] = row;
+            row += p.src_expert_count[r * E + e];
+        }
+    }
+
+    // ---- level 3: units per peer window, exclusive scan over (r,d) in id order ----
+    // R*R <= 4096 peer windows, up to 4 per thread, each thread's windows consecutive
+    const int n_win = R * R;
+    const int per_thread = (n_win + kPartThreads - 1) / kPartThreads;
+    int my_units = 0;
+    for (int i = 0; i < per_thread; ++i) {
+        const int w = tid * per_thread + i;
+        if (w < n_win) {
+            const int r = w / R, d = w - r * R;
+            long long B = 0;
+            for (int e = d * p.e_loc; e < (d + 1) * p.e_loc; ++e) B += p.src_expert_count[r * E + e];
+            const long long S = p.unit_rows[tier_of(p, r, d)];
+            my_units += (int)((B + S - 1) / S);
+        }
+    }
+    {   // block exclusive scan of my_units
+        int inc = my_units;
+#pragma unroll
+        for (int dlt = 1; dlt < 32; dlt <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, inc, dlt);
+            if (lane >= dlt) inc += t;
+        }
+        if (lane == 31) scan[wid] = inc;
+        __syncthreads();
+        if (wid == 0) {
+            const int s = scan[lane];
+            int si = s;
+#pragma unroll
+            for (int dlt = 1; dlt < 32; dlt <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, si, dlt);
+                if (lane >= dlt) si += t;
+            }
+            scan[lane] = si - s;
+            if (lane == 31) s_total = si;
+        }
+        __syncthreads();
+        my_units = scan[wid] + inc - my_units;     // now: first unit id of this thread's windows
+    }
+    const int U = s_total;
+    if (U > p.max_units || U > kPartMaxUnits) {
+        if (tid == 0) {
+            report_status(p.status, STRATA_ERR_CAPACITY);
+            *p.n_units = -1;
+        }
+        return;
+    }
+    // unit descriptors and costs
+    {
+        int j = my_units;
+        for (int i = 0; i < per_thread; ++i) {
+            const int w = tid * per_thread + i;
+            if (w < n_win) {
+                const int r = w / R, d = w - r * R;
+                long long B = 0;
+                for (int e = d * p.e_loc; e < (d + 1) * p.e_loc; ++e) B += p.src_expert_count[r * E + e];
+                const int t = tier_of(p, r, d);
+                const long long S = p.unit_rows[t];
+                for (long long a = 0; a < B; a += S, ++j) {
+                    const long long rows = min(S, B - a);
+                    const long long cost = p.alpha[t] + (rows * p.row_bytes + p.beta[t] - 1) / p.beta[t];
+                    p.unit_desc[j * 4 + 0] = r;
+                    p.unit_desc[j * 4 + 1] = d;
+                    p.unit_desc[j * 4 + 2] = (int)a;
+                    p.unit_desc[j * 4 + 3] = (int)rows;
+                    p.unit_cost[j] = cost;
+                    // largest cost first, ties by lower unit id: ascending order of this key
+                    keys[j] = ((unsigned long long)((1ll << 43) - 1 - cost) << 20) | (unsigned)j;
+                }
+            }
+        }
+    }
+    int P = 1;
+    while (P < U) P <<= 1;
+    for (int j = U + tid; j < P; j += kPartThreads) keys[j] = ~0ull;
+    for (int c = tid; c < p.n_cores; c += kPartThreads) {
+        load[c] = 0;
+        len[c] = 0;
+    }
+    for (int x = tid; x < kFanSmemInts; x += kPartThreads) fan[x] = 0;
+    int* core_of = p.scratch;
+    int* stripe_of = p.scratch + p.max_units;
+    int* fan_global = p.scratch + 2 * p.max_units;     // stripes beyond shared memory
+    const int smem_stripes = kFanSmemInts / R;
+    for (int x = tid; x < U * R; x += kPartThreads) fan_global[x] = 0;
+    __syncthreads();
+
+    // ---- bitonic sort of the keys ----
+    for (int k = 2; k <= P; k <<= 1)
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = tid; i < P; i += kPartThreads) {
+                const int ixj = i ^ j;
+                if (ixj > i) {
+                    const unsigned long long a = keys[i], b = keys[ixj];
+                    const bool up = (i & k) == 0;
+                    if ((a > b) == up) {
+                        keys[i] = b;
+                        keys[ixj] = a;
+                    }
+                }
+            }
+            __syncthreads();
+        }
+
+    // After the sort every key is replaced by what the greedy loop needs, so that the loop touches
+    // shared memory only: cost (37 bits) | destination rank (12) | unit id (13) | tier (2).
+    {
+        unsigned long long meta[kPartMaxUnits / kPartThreads];
+#pragma unroll
+        for (int i = 0; i < kPartMaxUnits / kPartThreads; ++i) {
+            const int o = tid + i * kPartThreads;
+            if (o < U) {
+                const int j = (int)(keys[o] & 0xfffffu);
+                const int r = p.unit_desc[j * 4 + 0], d = p.unit_desc[j * 4 + 1];
+                meta[i] = ((unsigned long long)p.unit_cost[j] << 27) | ((unsigned long long)d << 15) |
+                          ((unsigned long long)j << 2) | (unsigned)tier_of(p, r, d);
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < kPartMaxUnits / kPartThreads; ++i) {
+            const int o = tid + i * kPartThreads;
+            if (o < U) keys[o] = meta[i];
+        }
+        __syncthreads();
+    }
+
+    // ---- list scheduling: one warp, one unit per iteration; lane l speaks for cores l, l+32, ... ----
+    // The loop is sequential in the units and a lone warp pays full ALU latency on every dependent
+    // instruction, so the arithmetic is kept narrow: while every core's load fits 21 bits the key
+    // (infeasible | load | core) is one 32-bit word and the arg-min is one redux instruction; the
+    // first load that would not fit switches the rest of the run to 64-bit keys.
+    if (wid == 0) {
+        // narrow state of a core: load (21 bits) << 11 | list length (11 bits); slots past the last core
+        // (the table is padded to a multiple of 128) hold all ones and can never win
+        unsigned int* st32 = reinterpret_cast<unsigned int*>(scan);        // [kPartMaxCores] (scan[] is free here)
+        const int padded = (p.n_cores + 127) / 128 * 128;
+        for (int c = lane; c < padded; c += 32) st32[c] = c < p.n_cores ? 0u : 0xffffffffu;
+        __syncwarp();
+        int o = 0;
+        for (; o < U; ++o) {
+            const unsigned long long m = keys[o];
+            const unsigned int cost = (unsigned int)min(m >> 27, (unsigned long long)0x7fffffffu);
+            const int d = (int)((m >> 15) & 0xfffu), j = (int)((m >> 2) & 0x1fffu);
+            const int cap = (m & 3u) == 0 ? p.cap[0] : (m & 3u) == 1 ? p.cap[1] : p.cap[2];
+            const int* fan_d = fan + d;
+            unsigned int best = 0xffffffffu;
+            for (int c0 = lane; c0 < padded; c0 += 128) {
+                unsigned int st[4];
+                int f[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) st[u] = st32[c0 + 32 * u];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) f[u] = fan_d[min((int)(st[u] & 2047u), smem_stripes - 1) * R];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    unsigned int key = ((st[u] >> 1) & 0x7ffffc00u) | (unsigned)(c0 + 32 * u);
+                    if (f[u] >= cap) key |= 0x80000000u;                        // infeasible cores sort last
+                    best = min(best, st[u] == 0xffffffffu ? 0xffffffffu : key);
+                }
+            }
+            best = __reduce_min_sync(0xffffffffu, best);
+            const int win = (int)(best & 1023u);    // if every core was infeasible this is the least loaded overall
+            const unsigned int sw = st32[win];
+            const unsigned int new_load = (sw >> 11) + cost, kk = sw & 2047u;
+            // leave the narrow mode before anything stops fitting: load in 21 bits, list length in 11
+            // bits and inside the shared-memory part of the fan-out table
+            if (new_load >= (1u << 21) || kk + 1 >= 2047u || (int)kk + 1 >= smem_stripes) break;
+            if (lane == (win & 31)) {
+                fan[kk * R + d] += 1;
+                core_of[j] = win;
+                stripe_of[j] = (int)kk;
+                st32[win] = (new_load << 11) | (kk + 1);
+            }
+            __syncwarp();
+        }
+        for (int c = lane; c < p.n_cores; c += 32) {
+            len[c] = (int)(st32[c] & 2047u);
+            load[c] = (long long)(st32[c] >> 11);
+        }
+
+        __syncwarp();
+        const int cores_per_lane_w = (p.n_cores + 31) / 32;
+        for (; o < U; ++o) {                        // wide keys: load << 10 | core in 64 bits (load < 2^53)
+            const unsigned long long m = keys[o];
+            const long long cost = (long long)(m >> 27);
+            const int d = (int)((m >> 15) & 0xfffu), j = (int)((m >> 2) & 0x1fffu);
+            const int cap = (m & 3u) == 0 ? p.cap[0] : (m & 3u) == 1 ? p.cap[1] : p.cap[2];
+            unsigned long long best = ~0ull;
+            for (int i = 0; i < cores_per_lane_w; ++i) {
+                const int c = lane + 32 * i;
+                if (c < p.n_cores) {
+                    const int kk = len[c];
+                    const int f = kk < smem_stripes ? fan[kk * R + d] : fan_global[(size_t)kk * R + d];
+                    unsigned long long key = ((unsigned long long)load[c] << 10) | (unsigned)c;
+                    if (f >= cap) key |= 1ull << 63;
+                    best = min(best, key);
+                }
+            }
+#pragma unroll
+            for (int dlt = 16; dlt > 0; dlt >>= 1) {
+                const unsigned lo = __shfl_xor_sync(0xffffffffu, (unsigned)best, dlt);
+                const unsigned hi = __shfl_xor_sync(0xffffffffu, (unsigned)(best >> 32), dlt);
+                best = min(best, ((unsigned long long)hi << 32) | lo);
+            }
+            const int win = (int)(best & 1023u);
+            if (lane == (win & 31)) {
+                const int kk = len[win];
+                if (kk < smem_stripes) fan[kk * R + d] += 1;
+                else fan_global[(size_t)kk * R + d] += 1;
+                core_of[j] = win;
+                stripe_of[j] = kk;
+                len[win] = kk + 1;
+                load[win] += cost;
+            }
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+
+    // ---- per-core task lists in issue order ----
+    {
+        const int v = tid < p.n_cores ? len[tid] : 0;
+        int inc = v;
+#pragma unroll
+        for (int dlt = 1; dlt < 32; dlt <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, inc, dlt);
+            if (lane >= dlt) inc += t;
+        }
+        if (lane == 31) scan[wid] = inc;
+        __syncthreads();
+        if (wid == 0) {
+            const int s = scan[lane];
+            int si = s;
+#pragma unroll
+            for (int dlt = 1; dlt < 32; dlt <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, si, dlt);
+                if (lane >= dlt) si += t;
+            }
+            scan[lane] = si - s;
+        }
+        __syncthreads();
+        const int off = scan[wid] + inc - v;
+        if (tid < p.n_cores) {
+            p.task_offset[tid] = off;
+            p.core_load[tid] = load[tid];
+            scan[34 + tid] = off;              // scan[] has room for kPartThreads + 34 ints
+        }
+        if (tid == 0) {
+            p.task_offset[p.n_cores] = U;
+            *p.n_units = U;
+        }
+        __syncthreads();
+        for (int j = tid; j < U; j += kPartThreads) p.task_unit[scan[34 + core_of[j]] + stripe_of[j]] = j;
+    }
+}
+
+constexpr size_t kPartSmem = (size_t)kPartMaxUnits * 8 + (size_t)kPartMaxCores * 8 + (size_t)kPartMaxCores * 4 +
+                             (size_t)kFanSmemInts * 4 + (size_t)(kPartThreads + 34) * 4;
+
+// ---- window-major dispatch: every CTA follows its task list ---------------------------------
+constexpr int kWinStages = 4;
+constexpr uint32_t kWinMaxRowBytes = 16384;
+
+struct WindowsParams {
+    const int32_t* src_expert_count;
+    const int32_t* win_base;
+    const int32_t* unit_desc;
+    const int32_t* task_offset;
+    const int32_t* task_unit;
+    const int32_t* src_of_row;
+    const unsigned char* x;
+    unsigned char* recv;
+    long long capacity_rows, n_tok;
+    int E, e_loc, K, H;
+    int* status;
+    TraceBuf trace;
+};
+
+// One warp per core.  Rows are produced in batches of 32 (receive-row ids by lane 0 walking the task
+// list, their source tokens by all lanes from src_of_row), then lane 0 runs them through a ring of
+// stages: bulk load of the source row, then a bulk store to the receive row.  Ring protocol, with
+// `issued` loads and `stored` stores so far: never more than stages-1 loaded rows wait for their
+// store; before a stage is reloaded, wait_group.read<1> retires every store but the newest, which
+// includes the one that last read this stage.
+__global__ void __launch_bounds__(32) dispatch_windows_kernel(WindowsParams p)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    const uint32_t row_bytes = (uint32_t)p.H * 2u;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kWinStages * row_bytes);
+    __shared__ int s_row[32];
+    __shared__ int s_dst[kWinStages];          // receive row of the load held by each stage
+    const int lane = threadIdx.x;
+    const int core = blockIdx.x;
+
+    if (lane == 0) {
+        for (int s = 0; s < kWinStages; ++s) mbar_init(&bars[s], 1);
+        mbar_fence_init();
+    }
+    __syncwarp();
+    const uint64_t pol = policy_evict_first();
+    griddep_wait();
+    griddep_launch_dependents();
+    if (lane == 0) trace_begin(p.trace);
+
+    // lane 0 only: store the oldest loaded row
+    long long issued = 0, stored = 0;
+    auto store_oldest = [&]() -> bool {
+        const int s = (int)(stored % kWinStages);
+        if (!mbar_wait_bounded(&bars[s], (uint32_t)((stored / kWinStages) & 1))) return false;
+        bulk_s2g(p.recv + (size_t)s_dst[s] * row_bytes, smem + (size_t)s * row_bytes, row_bytes);
+        bulk_commit();
+        ++stored;
+        return true;
+    };
+
+    // cursor over this core's rows (lane 0)
+    int q = p.task_offset[core];
+    const int q_end = p.task_offset[core + 1];
+    int r = 0, e = 0, e_end = 0, first = 0, rows_left = 0;
+    bool ok = true;
+
+    while (ok) {
+        // ---- next batch of up to 32 receive rows ----
+        int n = 0;
+        if (lane == 0) {
+            while (n < 32) {
+                if (rows_left == 0) {
+                    if (q >= q_end) break;
+                    const int j = p.task_unit[q++];
+                    r = p.unit_desc[j * 4 + 0];
+                    const int d = p.unit_desc[j * 4 + 1];
+                    first = p.unit_desc[j * 4 + 2];
+                    rows_left = p.unit_desc[j * 4 + 3];
+                    e = d * p.e_loc;
+                    e_end = e + p.e_loc;
+                }
+                int cnt = p.src_expert_count[r * p.E + e];
+                while (first >= cnt && e + 1 < e_end) {     // expert windows in front of the first logical row
+                    first -= cnt;
+                    ++e;
+                    cnt = p.src_expert_count[r * p.E + e];
+                }
+                const int take = min(min(cnt - first, rows_left), 32 - n);
+                if (take <= 0) {                            // inconsistent lists: report, never loop forever
+                    report_status(p.status, STRATA_ERR_INVALID_ARG);
+                    rows_left = 0;
+                    q = q_end;
+                    break;
+                }
+                const int base = p.win_base[r * p.E + e] + first;
+                for (int i = 0; i < take; ++i) s_row[n + i] = base + i;
+                n += take;
+                first += take;
+                rows_left -= take;
+            }
+        }
+        n = __shfl_sync(0xffffffffu, n, 0);
+        if (n == 0) break;
+        __syncwarp();
+        const int my_row = lane < n ? s_row[lane] : -1;
+        const bool row_ok = my_row >= 0 && my_row < p.capacity_rows;
+        long long my_tok = row_ok ? (long long)p.src_of_row[my_row] / p.K : -1;
+        if (lane < n && (!row_ok || my_tok < 0 || my_tok >= p.n_tok)) {
+            report_status(p.status, STRATA_ERR_BAD_ROW);
+            my_tok = -1;
+        }
+        // ---- run the batch through the ring ----
+        for (int i = 0; i < n; ++i) {
+            const int row = __shfl_sync(0xffffffffu, my_row, i);
+            const long long tok = __shfl_sync(0xffffffffu, my_tok, i);
+            if (lane == 0 && tok >= 0 && ok) {
+                if (issued - stored == kWinStages - 1) ok = store_oldest();
+                if (ok) {
+                    if (issued >= kWinStages) bulk_wait_read<1>();
+                    const int s = (int)(issued % kWinStages);
+                    s_dst[s] = row;
+                    mbar_expect_tx(&bars[s], row_bytes);
+                    bulk_g2s(smem + (size_t)s * row_bytes, p.x + (size_t)tok * row_bytes, row_bytes, &bars[s], pol);
+                    ++issued;
+                }
+            }
+        }
+        ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+        __syncwarp();
+    }
+    if (lane == 0) {
+        while (ok && stored < issued) ok = store_oldest();
+        if (!ok) report_status(p.status, STRATA_ERR_TIMEOUT);
+        bulk_wait_read<0>();
+        trace_end(p.trace);
+    }
+}
+
+}  // namespace
+
+cudaError_t configure_partition_kernels()
+{
+    cudaError_t err =
+        cudaFuncSetAttribute(partition_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPartSmem);
+    if (err != cudaSuccess) return err;
+    return cudaFuncSetAttribute(dispatch_windows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                kWinStages * (int)kWinMaxRowBytes + 64);
+}
+
+cudaError_t launch_partition(const strata_moe_shape& s, const strata_moe_layout_t& L,
+                             const strata_partition_policy& pol, int n_cores, const strata_partition_t& out,
+                             size_t max_units, int* status, cudaStream_t st)
+{
+    PartitionParams p{};
+    p.src_expert_count = L.src_expert_count;
+    p.expert_offset = L.expert_offset;
+    p.win_base = out.win_base;
+    p.unit_desc = out.unit_desc;
+    p.unit_cost = reinterpret_cast<long long*>(out.unit_cost);
+    p.n_units = out.n_units;
+    p.task_offset = out.task_offset;
+    p.task_unit = out.task_unit;
+    p.core_load = reinterpret_cast<long long*>(out.core_load);
+    p.scratch = out.scratch;
+    p.status = status;
+    p.R = s.R;
+    p.E = s.E;
+    p.e_loc = s.E / s.R;
+    p.n_cores = n_cores;
+    p.max_units = (int)max_units;
+    p.n_tiers = pol.n_tiers;
+    p.g0 = pol.g0;
+    p.g1 = pol.g1;
+    p.row_bytes = (long long)s.H * 2;
+    for (int t = 0; t < pol.n_tiers; ++t) {
+        p.alpha[t] = pol.tiers[t].alpha;
+        p.beta[t] = pol.tiers[t].beta;
+        p.unit_rows[t] = pol.tiers[t].unit_rows;
+        p.cap[t] = pol.tiers[t].fanout_cap;
+    }
+    return launch_pdl(partition_kernel, 1, kPartThreads, kPartSmem, st, p);
+}
+
+cudaError_t launch_dispatch_windows(const strata_moe_shape& s, const strata_moe_layout_t& L,
+                                    const strata_partition_t& part, int n_cores, const void* x, void* recv,
+                                    size_t capacity_rows, int* status, TraceBuf trace, cudaStream_t st)
+{
+    WindowsParams p{};
+    p.src_expert_count = L.src_expert_count;
+    p.win_base = part.win_base;
+    p.unit_desc = part.unit_desc;
+    p.task_offset = part.task_offset;
+    p.task_unit = part.task_unit;
+    p.src_of_row = L.src_of_row;
+    p.x = static_cast<const unsigned char*>(x);
+    p.recv = static_cast<unsigned char*>(recv);
+    p.capacity_rows = (long long)capacity_rows;
+    p.n_tok = (long long)s.R * s.T;
+    p.E = s.E;
+    p.e_loc = s.E / s.R;
+    p.K = s.K;
+    p.H = s.H;
+    p.status = status;
+    p.trace = trace;
+    const size_t smem = (size_t)kWinStages * s.H * 2 + 64;
+    return launch_plain(dispatch_windows_kernel, (unsigned)n_cores, 32, smem, st, p);
+}
+
+int partition_max_units_supported() { return kPartMaxUnits; }
+int partition_max_cores_supported() { return kPartMaxCores; }
+uint32_t windows_max_row_bytes() { return kWinMaxRowBytes; }
+
+}  // namespace strata
