@@ -180,15 +180,7 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
 // One thread per CTA calls these; slot = blockIdx.x.
 __device__ __forceinline__ void trace_begin(const TraceBuf& t)
 {
-#ifdef STRATA_TRACE_SMID
-    if (t.slots && (int)blockIdx.x < t.capacity) {   // experiment build: record the SM id instead of the start time
-        unsigned int smid;
-        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-        t.slots[2 * blockIdx.x] = smid + 1;
-    }
-#else
     if (t.slots && (int)blockIdx.x < t.capacity) t.slots[2 * blockIdx.x] = global_timer_ns();
-#endif
 }
 __device__ __forceinline__ void trace_end(const TraceBuf& t)
 {
@@ -287,11 +279,6 @@ template <int N>
 __device__ __forceinline__ void bulk_wait_read()
 {
     asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
-}
-template <int N>
-__device__ __forceinline__ void bulk_wait_all()
-{
-    asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
 }
 // generic-proxy writes to shared memory become visible to the async proxy
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }

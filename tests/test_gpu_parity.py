@@ -424,3 +424,22 @@ def test_per_cta_trace_probes():
     assert int(tr.abs().sum().item()) == 0                   # probes off: nothing written
     assert ctx.device_status() == B.STRATA_OK
     ctx.close()
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_shapes(seed):
+    """Seeded random shapes through the whole path: odd sizes hit every work-distribution branch
+    (all-static grids, column-part units, chunked rows, cluster and tiled layouts)."""
+    rng = np.random.default_rng(1234 + seed)
+    R = int(rng.choice([1, 2, 3, 4, 6, 8, 16]))
+    e_loc = int(rng.integers(1, 9))
+    E = R * e_loc
+    K = int(rng.integers(1, min(E, 10) + 1))
+    T = int(rng.choice([1, 5, 37, 130, 700, 3000]))
+    H = int(rng.choice([8, 64, 520, 1024, 2056, 7168, 9000])) // 8 * 8
+    if R * T * K * H * 2 > 600e6:          # keep every case under ~0.6 GB of receive buffer
+        T = max(1, int(600e6 // (R * K * H * 2)))
+    cfg = wl.shrink(wl.CONFIGS["decode"], R=R, T=T, H=H, E=E, K=K, seed=9000 + seed,
+                    routing="zipf" if seed % 3 == 0 else "uniform",
+                    expert=["identity", "scale", "affine"][seed % 3])
+    run_full_case(cfg, threads=8)
