@@ -35,7 +35,7 @@ def lib() -> ctypes.CDLL:
         L = ctypes.CDLL(build())
         i32, i64, vp = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p
         L.oracle_layout.restype = i64
-        L.oracle_layout.argtypes = [i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.oracle_layout.argtypes = [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.oracle_dispatch_bf16.restype = None
         L.oracle_dispatch_bf16.argtypes = [i64, i32, i32, vp, vp, vp, i32]
         L.oracle_dispatch_fp8.restype = None
@@ -73,11 +73,13 @@ class BadExpertId(ValueError):
         self.item = item
 
 
-def layout(ids: np.ndarray, E: int) -> Dict[str, np.ndarray]:
-    """Routing layout of ids int32 [R,T,K]; raises BadExpertId for an id outside [0,E)."""
+def layout(ids: np.ndarray, E: int, segment_align: int = 1, allow_unrouted: bool = False) -> Dict[str, np.ndarray]:
+    """Routing layout of ids int32 [R,T,K]; raises BadExpertId for an id outside [0,E) (-1 is accepted
+    as "not routed" with allow_unrouted).  segment_align > 1 pads every expert segment to that many rows."""
     ids = _c(ids, np.int32)
     R, T, K = ids.shape
     N = R * T * K
+    A = max(1, int(segment_align))
     out = {
         "expert_count": np.zeros(E, np.int32),
         "expert_offset": np.zeros(E + 1, np.int32),
@@ -85,21 +87,23 @@ def layout(ids: np.ndarray, E: int) -> Dict[str, np.ndarray]:
         "rank_offset": np.zeros(R + 1, np.int32),
         "src_expert_count": np.zeros((R, E), np.int32),
         "dst_row": np.full((R, T, K), -1, np.int32),
-        "src_of_row": np.full(N, -1, np.int32),
+        "src_of_row": np.full(N + E * (A - 1), -1, np.int32),
     }
-    rc = lib().oracle_layout(R, T, K, E, _p(ids), _p(out["expert_count"]), _p(out["expert_offset"]),
-                             _p(out["rank_count"]), _p(out["rank_offset"]), _p(out["src_expert_count"]),
-                             _p(out["dst_row"]), _p(out["src_of_row"]))
+    rc = lib().oracle_layout(R, T, K, E, A, int(bool(allow_unrouted)), _p(ids), _p(out["expert_count"]),
+                             _p(out["expert_offset"]), _p(out["rank_count"]), _p(out["rank_offset"]),
+                             _p(out["src_expert_count"]), _p(out["dst_row"]), _p(out["src_of_row"]))
     if rc < 0:
         if rc < -(1 << 40):
             raise ValueError("invalid shape (need R,K,E > 0 and E % R == 0)")
         raise BadExpertId(int(-rc - 1))
+    out["src_of_row"] = out["src_of_row"][:int(out["expert_offset"][E])]
     return out
 
 
 def dispatch_bf16(dst_row: np.ndarray, x: np.ndarray, nthreads: int = 1,
-                  recv: Optional[np.ndarray] = None) -> np.ndarray:
-    """recv uint16 [N,H] with recv[dst_row[i]] = x[i // K]."""
+                  recv: Optional[np.ndarray] = None, n_rows: Optional[int] = None) -> np.ndarray:
+    """recv uint16 [n_rows,H] (default n_rows = N) with recv[dst_row[i]] = x[i // K]; rows that no item
+    maps to (padding) keep 0xDEAD."""
     dst_row = _c(dst_row, np.int32)
     K = dst_row.shape[-1]
     H = x.shape[-1]
@@ -107,14 +111,14 @@ def dispatch_bf16(dst_row: np.ndarray, x: np.ndarray, nthreads: int = 1,
     n_tok = x2.shape[0]
     assert dst_row.size == n_tok * K
     if recv is None:
-        recv = np.empty((n_tok * K, H), np.uint16)
+        recv = np.full((n_rows if n_rows is not None else n_tok * K, H), 0xDEAD, np.uint16)
     assert recv.dtype == np.uint16 and recv.flags.c_contiguous
     lib().oracle_dispatch_bf16(n_tok, K, H, _p(dst_row), _p(x2), _p(recv), nthreads)
     return recv
 
 
-def dispatch_fp8(dst_row: np.ndarray, x: np.ndarray, nthreads: int = 1):
-    """(recv_q uint8 [N,H], recv_scale float32 [N,H/128])."""
+def dispatch_fp8(dst_row: np.ndarray, x: np.ndarray, nthreads: int = 1, n_rows: Optional[int] = None):
+    """(recv_q uint8 [n_rows,H], recv_scale float32 [n_rows,H/128]); padding rows keep 0x7F / -7."""
     dst_row = _c(dst_row, np.int32)
     K = dst_row.shape[-1]
     H = x.shape[-1]
@@ -122,8 +126,9 @@ def dispatch_fp8(dst_row: np.ndarray, x: np.ndarray, nthreads: int = 1):
     x2 = _c(x, np.uint16).reshape(-1, H)
     n_tok = x2.shape[0]
     assert dst_row.size == n_tok * K
-    q = np.empty((n_tok * K, H), np.uint8)
-    s = np.empty((n_tok * K, H // 128), np.float32)
+    rows = n_rows if n_rows is not None else n_tok * K
+    q = np.full((rows, H), 0x7F, np.uint8)
+    s = np.full((rows, H // 128), -7.0, np.float32)
     lib().oracle_dispatch_fp8(n_tok, K, H, _p(dst_row), _p(x2), _p(q), _p(s), nthreads)
     return q, s
 

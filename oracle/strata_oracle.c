@@ -49,10 +49,22 @@
 /* O1: routing layout = stable counting sort of items by expert id.    */
 /* Returns 0, or -(i+1) where i is the first item whose id is outside  */
 /* [0,E) (nothing is written for a rejected input beyond the counts    */
-/* seen so far), or -2^31 for an invalid shape.                        */
+/* seen so far), or -2^62 for an invalid shape.                        */
 /* Optional outputs (src_expert_count, src_of_row) may be NULL.        */
+/* Production variants (this build's readings; the paper only names    */
+/* the metadata):                                                      */
+/*  segment_align A > 1: every expert segment starts at a multiple of  */
+/*    A rows: offset[e+1] = round_up(offset[e] + count[e], A); the     */
+/*    rows between a segment's end and the next start are padding      */
+/*    (src_of_row = -1 there); rank_offset follows the padded offsets, */
+/*    rank_count stays the number of real rows.  src_of_row then has   */
+/*    offset[E] entries.                                               */
+/*  allow_unrouted: an id of -1 means "not routed": the item gets      */
+/*    dst_row = -1, is not counted, and is skipped by dispatch and     */
+/*    combine.  Without the flag -1 is rejected like any bad id.       */
 /* ------------------------------------------------------------------ */
 int64_t oracle_layout(int32_t R, int32_t T, int32_t K, int32_t E,
+                      int32_t segment_align, int32_t allow_unrouted,
                       const int32_t *ids,           /* [R,T,K] */
                       int32_t *expert_count,        /* [E]     */
                       int32_t *expert_offset,       /* [E+1]   */
@@ -60,12 +72,13 @@ int64_t oracle_layout(int32_t R, int32_t T, int32_t K, int32_t E,
                       int32_t *rank_offset,         /* [R+1]   */
                       int32_t *src_expert_count,    /* [R,E] or NULL */
                       int32_t *dst_row,             /* [R,T,K] */
-                      int32_t *src_of_row)          /* [N] or NULL */
+                      int32_t *src_of_row)          /* [offset[E]] or NULL */
 {
     if (R <= 0 || T < 0 || K <= 0 || E <= 0 || E % R != 0) return INT64_MIN / 2;
     const int64_t N = (int64_t)R * T * K;
     const int64_t per_rank = (int64_t)T * K;
     const int32_t E_loc = E / R;
+    const int32_t A = segment_align > 1 ? segment_align : 1;
 
     /* per-expert counts (and per-(source rank, expert) counts) */
     for (int32_t e = 0; e < E; ++e) expert_count[e] = 0;
@@ -73,14 +86,18 @@ int64_t oracle_layout(int32_t R, int32_t T, int32_t K, int32_t E,
         for (int64_t j = 0; j < (int64_t)R * E; ++j) src_expert_count[j] = 0;
     for (int64_t i = 0; i < N; ++i) {
         const int32_t e = ids[i];
+        if (allow_unrouted && e == -1) continue;
         if (e < 0 || e >= E) return -(i + 1);
         expert_count[e] += 1;
         if (src_expert_count) src_expert_count[(i / per_rank) * E + e] += 1;
     }
 
-    /* prefix-sum offsets: segment of expert e is rows [offset[e], offset[e+1]) */
+    /* prefix-sum offsets: segment of expert e is rows [offset[e], offset[e] + count[e]) */
     expert_offset[0] = 0;
-    for (int32_t e = 0; e < E; ++e) expert_offset[e + 1] = expert_offset[e] + expert_count[e];
+    for (int32_t e = 0; e < E; ++e) {
+        const int64_t end = (int64_t)expert_offset[e] + expert_count[e];
+        expert_offset[e + 1] = (int32_t)((end + A - 1) / A * A);
+    }
 
     /* rows received per destination rank; rank d owns experts [d*E_loc,(d+1)*E_loc) */
     for (int32_t d = 0; d < R; ++d) {
@@ -89,14 +106,20 @@ int64_t oracle_layout(int32_t R, int32_t T, int32_t K, int32_t E,
         rank_count[d] = s;
         rank_offset[d] = expert_offset[d * E_loc];
     }
-    rank_offset[R] = (int32_t)N;
+    rank_offset[R] = expert_offset[E];
 
     /* token-local offsets: the j-th item (in increasing i) that chose expert e
        lands in row offset[e] + j.  Increasing i is lexicographic (r,t,k). */
     int32_t *seen = (int32_t *)calloc((size_t)E, sizeof(int32_t));
     if (!seen) return INT64_MIN / 2;
+    if (src_of_row)
+        for (int64_t j = 0; j < expert_offset[E]; ++j) src_of_row[j] = -1;
     for (int64_t i = 0; i < N; ++i) {
         const int32_t e = ids[i];
+        if (e == -1) {
+            dst_row[i] = -1;
+            continue;
+        }
         const int32_t row = expert_offset[e] + seen[e];
         seen[e] += 1;
         dst_row[i] = row;
@@ -120,6 +143,7 @@ void oracle_dispatch_bf16(int64_t n_tok, int32_t K, int32_t H,
     for (int64_t n = 0; n < n_tok; ++n)
         for (int32_t k = 0; k < K; ++k) {
             const int64_t row = dst_row[n * K + k];
+            if (row < 0) continue;                  /* not routed */
             memcpy(recv + (size_t)row * H, x + (size_t)n * H, (size_t)H * 2);
         }
 }
@@ -237,6 +261,7 @@ void oracle_dispatch_fp8(int64_t n_tok, int32_t K, int32_t H,
         }
         for (int32_t k = 0; k < K; ++k) {
             const int64_t row = dst_row[n * K + k];
+            if (row < 0) continue;                  /* not routed */
             memcpy(recv_q + (size_t)row * H, q, (size_t)H);
             memcpy(recv_scale + (size_t)row * nb, sc, (size_t)nb * sizeof(float));
         }
@@ -273,6 +298,7 @@ void oracle_combine(int64_t n_tok, int32_t K, int32_t H,
             float acc = 0.0f;
             for (int32_t k = 0; k < K; ++k) {
                 const int64_t row = dst_row[n * K + k];
+                if (row < 0) continue;              /* not routed: the slot contributes nothing */
                 acc = fmaf(w[n * K + k], bf16_to_f32(y[(size_t)row * H + c]), acc);
             }
             out[(size_t)n * H + c] = f32_to_bf16_rne(acc);

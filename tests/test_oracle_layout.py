@@ -147,3 +147,98 @@ def test_invariants_on_tiny_config():
     check_invariants(ids, cfg.E, lay)
     dst, cnt, _ = brute_force_layout(ids, cfg.E)
     assert np.array_equal(lay["dst_row"], dst)
+
+
+# ---- production variants: aligned segments and the "not routed" sentinel ----------------------
+
+def brute_force_layout_variants(ids, E, A, allow_unrouted):
+    """Independent formulation: sort the routed item tuples; row = aligned segment start + position."""
+    R, T, K = ids.shape
+    tuples = [(int(ids[r, t, k]), r, t, k) for r in range(R) for t in range(T) for k in range(K)
+              if not (allow_unrouted and ids[r, t, k] == -1)]
+    cnt = np.zeros(E, np.int64)
+    for e, _, _, _ in tuples:
+        cnt[e] += 1
+    off = np.zeros(E + 1, np.int64)
+    for e in range(E):
+        off[e + 1] = -(-(off[e] + cnt[e]) // A) * A
+    dst = np.full((R, T, K), -1, np.int32)
+    pos = np.zeros(E, np.int64)
+    for e, r, t, k in sorted(tuples):
+        dst[r, t, k] = off[e] + pos[e]
+        pos[e] += 1
+    return dst, cnt, off
+
+
+def test_worked_example_padded_unrouted():
+    rows = {}
+    with open(os.path.join(GOLDEN, "layout_padded_unrouted_example.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].split()
+            if line:
+                rows[line[0]] = np.array(line[1:], dtype=np.int64)
+    R, T, K, E = rows["shape"]
+    lay = oracle.layout(rows["ids"].astype(np.int32).reshape(R, T, K), int(E), segment_align=int(rows["align"][0]),
+                        allow_unrouted=True)
+    for key in ("expert_count", "expert_offset", "rank_count", "rank_offset", "src_expert_count", "dst_row",
+                "src_of_row"):
+        assert np.array_equal(lay[key].ravel(), rows[key]), key
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_variants_match_brute_force(seed):
+    rng = np.random.default_rng(100 + seed)
+    R = int(rng.choice([1, 2, 4]))
+    E = R * int(rng.integers(1, 5))
+    T, K = int(rng.integers(1, 40)), int(rng.integers(1, 5))
+    A = int(rng.choice([1, 2, 8, 16, 128]))
+    ids = rng.integers(-1, E, size=(R, T, K)).astype(np.int32)
+    lay = oracle.layout(ids, E, segment_align=A, allow_unrouted=True)
+    dst, cnt, off = brute_force_layout_variants(ids, E, A, True)
+    assert np.array_equal(lay["dst_row"], dst)
+    assert np.array_equal(lay["expert_count"], cnt)
+    assert np.array_equal(lay["expert_offset"], off)
+    assert np.all(lay["expert_offset"] % A == 0)
+    assert lay["rank_count"].sum() == (ids >= 0).sum()
+    assert lay["rank_offset"][R] == off[E] and np.array_equal(lay["rank_offset"][:R], off[0:E:E // R])
+    # inverse map: padding rows and nothing else hold -1
+    src = lay["src_of_row"]
+    assert src.size == off[E]
+    routed = np.flatnonzero(ids.ravel() >= 0)
+    assert np.array_equal(np.sort(src[src >= 0]), routed)
+    assert np.array_equal(lay["dst_row"].ravel()[src[src >= 0]], np.flatnonzero(src >= 0))
+    # without the flag, -1 is rejected like any bad id
+    if (ids == -1).any():
+        with pytest.raises(oracle.BadExpertId):
+            oracle.layout(ids, E, segment_align=A)
+    # align 1 without unrouted items is the plain layout
+    ids2 = np.where(ids < 0, 0, ids).astype(np.int32)
+    a = oracle.layout(ids2, E)
+    b = oracle.layout(ids2, E, segment_align=1, allow_unrouted=True)
+    assert all(np.array_equal(a[k], b[k]) for k in a)
+
+
+def test_dispatch_and_combine_skip_unrouted_and_leave_padding():
+    from paper_2607_26444_b200 import workloads as wl
+    cfg = wl.shrink(wl.CONFIGS["tiny"], R=2, T=40, H=64, E=8, K=3)
+    inp = wl.generate(cfg)
+    ids = inp["ids"].copy()
+    rng = np.random.default_rng(3)
+    ids[rng.random(ids.shape) < 0.3] = -1
+    ids[0, 0, :] = -1                                   # a token with no expert at all
+    lay = oracle.layout(ids, cfg.E, segment_align=16, allow_unrouted=True)
+    n_rows = int(lay["expert_offset"][cfg.E])
+    recv = oracle.dispatch_bf16(lay["dst_row"], inp["x"], n_rows=n_rows)
+    x2 = inp["x"].reshape(cfg.n_tok, cfg.H)
+    src = lay["src_of_row"]
+    assert np.all(recv[src < 0] == 0xDEAD)              # padding rows untouched
+    assert np.array_equal(recv[src >= 0], x2[src[src >= 0] // cfg.K])
+    out = oracle.combine(lay["dst_row"], recv, inp["w"])
+    assert np.all(out[0] == 0)                          # nothing routed: the sum is empty, +0
+    # against float64 over the routed slots only
+    rows = lay["dst_row"].reshape(cfg.n_tok, cfg.K)
+    w = inp["w"].reshape(cfg.n_tok, cfg.K).astype(np.float64)
+    xv = wl.bf16_bits_to_f32(x2).astype(np.float64)
+    exact = ((rows >= 0) * w).sum(axis=1, keepdims=True) * xv
+    got = wl.bf16_bits_to_f32(out).astype(np.float64)
+    assert np.all(np.abs(got - exact) <= np.abs(exact) * 2.0 ** -8 + 1e-30)
