@@ -55,10 +55,21 @@ typedef enum {
 
 /* Problem shape.  Requirements: R,T,H,E,K > 0; E % R == 0; E <= 1024; K <= 32;
  * H % 8 == 0 (rows are whole 16-byte vectors); H % 128 == 0 for FP8;
- * R*T*K < 2^31. */
+ * R*T*K + E*(segment_align-1) < 2^31.
+ * Two production variants of the layout (zero = off, the packed strict layout):
+ *  segment_align A > 1: every expert segment starts at a multiple of A rows (what a grouped GEMM
+ *    with A-row tiles wants): expert_offset[e+1] = round_up(expert_offset[e] + expert_count[e], A).
+ *    Rows between a segment's end and the next start are padding: dispatch never writes them and
+ *    src_of_row is -1 there.  rank_offset follows the padded offsets, rank_count and expert_count
+ *    stay the numbers of real rows.  The receive buffer needs strata_moe_recv_rows() rows.
+ *  STRATA_FLAG_ALLOW_UNROUTED: an id of -1 means "not routed" (dropped token slot): dst_row = -1,
+ *    counted nowhere, skipped by dispatch, contributes nothing in combine, and is not an error. */
+#define STRATA_FLAG_ALLOW_UNROUTED 1
 typedef struct {
     int32_t R, T, H, E, K;
     int32_t dispatch_dtype;        /* a strata_dtype */
+    int32_t segment_align;         /* rows; 0 or 1 = packed segments; at most 65536 */
+    int32_t flags;                 /* STRATA_FLAG_* */
 } strata_moe_shape;
 
 typedef struct strata_ctx strata_ctx;   /* opaque, host side */
@@ -73,8 +84,8 @@ typedef struct {
     int32_t *rank_count;        /* [R]    rows received by rank d                        */
     int32_t *rank_offset;       /* [R+1]  rank d's partition = rows [off[d],off[d+1])    */
     int32_t *src_expert_count;  /* [R,E]  items of source rank r routed to e; may be NULL */
-    int32_t *dst_row;           /* [R,T,K] receive row of item i (-1 for a skipped item) */
-    int32_t *src_of_row;        /* [N]    inverse of dst_row; may be NULL                */
+    int32_t *dst_row;           /* [R,T,K] receive row of item i (-1 for a skipped or unrouted item) */
+    int32_t *src_of_row;        /* [strata_moe_recv_rows] inverse of dst_row, -1 on padding rows; may be NULL */
 } strata_moe_layout_t;
 
 const char *strata_status_string(strata_status s);
@@ -96,6 +107,9 @@ strata_status strata_ctx_destroy(strata_ctx *ctx);
  * strata_ctx_set_workspace, which zeroes it (synchronously).  It must stay
  * valid and unshared while calls on this context are in flight. */
 strata_status strata_moe_workspace_bytes(const strata_moe_shape *shape, size_t *bytes);
+/* Rows the receive buffer (and src_of_row) must hold: R*T*K + E*(segment_align-1), the worst case of
+ * the padded layout (R*T*K for packed segments).  Host arithmetic only. */
+strata_status strata_moe_recv_rows(const strata_moe_shape *shape, size_t *rows);
 strata_status strata_ctx_set_workspace(strata_ctx *ctx, void *dptr, size_t bytes);
 
 /* Number of kernels this context has launched so far (for accounting). */
@@ -134,7 +148,8 @@ strata_status strata_pool_reset(strata_ctx *ctx, uint64_t region_id);
  * expert_offset[e_i] + #{j < i : e_j = e_i}, i.e. segments ordered by expert,
  * then source rank, then token, then slot, packed without padding.
  * Duplicate ids inside a token are legal.  An id outside [0,E) is skipped
- * (dst_row = -1, not counted) and raises BAD_EXPERT_ID on the device status.
+ * (dst_row = -1, not counted) and raises BAD_EXPERT_ID on the device status
+ * (except -1 under STRATA_FLAG_ALLOW_UNROUTED, which is legal).
  * Needs a workspace.  One kernel launch for up to 32,768 items, two beyond. */
 strata_status strata_moe_layout(strata_ctx *ctx, const int32_t *topk_ids,
                                 const strata_moe_layout_t *layout, void *stream);
@@ -147,7 +162,8 @@ strata_status strata_moe_layout(strata_ctx *ctx, const int32_t *topk_ids,
  * Same inputs, outputs, ordering and error rules as strata_moe_layout, computed by the same kernels;
  * the kernels' scratch lives in a fixed 2 MiB array inside the library (each GPU that loads the
  * library holds it until the process exits) instead of a caller workspace.
- *  - Runs on the CURRENT CUDA device; no context is needed.  `shape->H` and `dispatch_dtype` are ignored.
+ *  - Runs on the CURRENT CUDA device; no context is needed.  `shape->H` and `dispatch_dtype` are ignored;
+ *    segment_align and flags are honoured.
  *  - Limit: 256 + ceil(T*K/4096) * R * E * 4 bytes must fit in 2 MiB (all five benchmark shapes do;
  *    the prefill shape needs 0.13 MiB).  Larger shapes return STRATA_ERR_CAPACITY and launch nothing:
  *    use strata_moe_layout with a workspace for those.
@@ -173,8 +189,9 @@ strata_status strata_moe_layout_noalloc(const strata_moe_shape *shape, const int
  *        division), q = e4m3_rne_satfinite(x / (amax == 0 ? 1 : scale)); codes and the stored
  *        scale (amax/448) go to each of the token's K rows.
  * recv (and recv_scale) must lie inside a registered region (NOT_REGISTERED otherwise); x and recv
- * must be 16-byte aligned, recv_scale 4-byte aligned; capacity_rows >= N (CAPACITY otherwise).  Rows whose dst_row is outside
- * [0, capacity_rows) are skipped and raise BAD_ROW.  One kernel launch. */
+ * must be 16-byte aligned, recv_scale 4-byte aligned; capacity_rows >= strata_moe_recv_rows (CAPACITY
+ * otherwise).  Items with dst_row = -1 are skipped silently; any other dst_row outside
+ * [0, capacity_rows) is skipped and raises BAD_ROW.  One kernel launch. */
 strata_status strata_moe_dispatch(strata_ctx *ctx, const strata_moe_layout_t *layout, const void *x,
                                   void *recv, float *recv_scale, size_t capacity_rows, void *stream);
 
@@ -182,8 +199,9 @@ strata_status strata_moe_dispatch(strata_ctx *ctx, const strata_moe_layout_t *la
  * outputs, row j answers receive row j; may be the receive buffer itself), topk_w: device
  * float [R,T,K], out: device bf16 [R,T,H].
  * out[n,c] = bf16_rne( fma(w[n,K-1], y[dst_row[n,K-1],c], ... fma(w[n,0], y[dst_row[n,0],c], +0)) ):
- * binary32 fused multiply-add chain in slot order, one rounding to bf16.  Slots whose dst_row is
- * outside [0, y_rows) contribute nothing and raise BAD_ROW.  One kernel launch. */
+ * binary32 fused multiply-add chain in slot order, one rounding to bf16.  Slots with dst_row = -1
+ * contribute nothing; any other dst_row outside [0, y_rows) contributes nothing and raises BAD_ROW.
+ * One kernel launch. */
 strata_status strata_moe_combine(strata_ctx *ctx, const strata_moe_layout_t *layout, const void *y,
                                  size_t y_rows, const float *topk_w, void *out, void *stream);
 

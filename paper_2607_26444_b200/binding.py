@@ -29,6 +29,7 @@ STRATA_ERR_BAD_ROW = 10
 
 STRATA_BF16 = 0
 STRATA_FP8_E4M3_B128 = 1
+STRATA_FLAG_ALLOW_UNROUTED = 1
 
 EXPORTS = [
     "strata_status_string", "strata_ctx_create", "strata_ctx_destroy", "strata_moe_workspace_bytes",
@@ -37,12 +38,14 @@ EXPORTS = [
     "strata_moe_dispatch", "strata_moe_combine", "strata_moe_recv_view", "strata_device_status",
     "strata_moe_roundtrip_host", "strata_moe_layout_noalloc", "strata_ctx_set_trace",
     "strata_moe_partition_max_units", "strata_moe_partition", "strata_moe_dispatch_windows",
+    "strata_moe_recv_rows",
 ]
 
 
 class strata_moe_shape(ctypes.Structure):
     _fields_ = [("R", ctypes.c_int32), ("T", ctypes.c_int32), ("H", ctypes.c_int32),
-                ("E", ctypes.c_int32), ("K", ctypes.c_int32), ("dispatch_dtype", ctypes.c_int32)]
+                ("E", ctypes.c_int32), ("K", ctypes.c_int32), ("dispatch_dtype", ctypes.c_int32),
+                ("segment_align", ctypes.c_int32), ("flags", ctypes.c_int32)]
 
 
 class strata_moe_layout_t(ctypes.Structure):
@@ -108,6 +111,7 @@ def lib() -> ctypes.CDLL:
         "strata_ctx_create": [P(vp), P(strata_moe_shape), i32],
         "strata_ctx_destroy": [vp],
         "strata_moe_workspace_bytes": [P(strata_moe_shape), P(sz)],
+        "strata_moe_recv_rows": [P(strata_moe_shape), P(sz)],
         "strata_ctx_set_workspace": [vp, vp, sz],
         "strata_ctx_launch_count": [vp, P(u64)],
         "strata_pool_register": [vp, vp, sz, P(u64)],
@@ -155,6 +159,12 @@ def strata_ctx_destroy(ctx) -> int:
 def strata_moe_workspace_bytes(shape: strata_moe_shape) -> Tuple[int, int]:
     n = ctypes.c_size_t()
     rc = lib().strata_moe_workspace_bytes(ctypes.byref(shape), ctypes.byref(n))
+    return rc, n.value
+
+
+def strata_moe_recv_rows(shape: strata_moe_shape) -> Tuple[int, int]:
+    n = ctypes.c_size_t()
+    rc = lib().strata_moe_recv_rows(ctypes.byref(shape), ctypes.byref(n))
     return rc, n.value
 
 
@@ -265,7 +275,8 @@ def _check(rc: int, where: str) -> None:
 class Layout:
     """Device tensors holding the routing metadata, plus the C struct pointing at them."""
 
-    def __init__(self, R: int, T: int, K: int, E: int, device, with_optional: bool = True):
+    def __init__(self, R: int, T: int, K: int, E: int, device, with_optional: bool = True,
+                 recv_rows: Optional[int] = None):
         import torch
         i32 = dict(dtype=torch.int32, device=device)
         self.expert_count = torch.empty(E, **i32)
@@ -274,7 +285,7 @@ class Layout:
         self.rank_offset = torch.empty(R + 1, **i32)
         self.src_expert_count = torch.empty((R, E), **i32) if with_optional else None
         self.dst_row = torch.empty((R, T, K), **i32)
-        self.src_of_row = torch.empty(R * T * K, **i32) if with_optional else None
+        self.src_of_row = torch.empty(recv_rows or R * T * K, **i32) if with_optional else None
         self.c = strata_moe_layout_t(
             self.expert_count.data_ptr(), self.expert_offset.data_ptr(), self.rank_count.data_ptr(),
             self.rank_offset.data_ptr(),
@@ -308,11 +319,12 @@ class MoEContext:
     """One shape on one GPU.  Owns a strata_ctx and its workspace tensor."""
 
     def __init__(self, R: int, T: int, H: int, E: int, K: int, dispatch_dtype: int = STRATA_BF16,
-                 device: int = 0):
+                 device: int = 0, segment_align: int = 0, allow_unrouted: bool = False):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("MoEContext needs a CUDA device (there is no CPU fallback)")
-        self.shape = strata_moe_shape(R, T, H, E, K, dispatch_dtype)
+        self.shape = strata_moe_shape(R, T, H, E, K, dispatch_dtype, segment_align,
+                                      STRATA_FLAG_ALLOW_UNROUTED if allow_unrouted else 0)
         self.R, self.T, self.H, self.E, self.K = R, T, H, E, K
         self.fp8 = dispatch_dtype == STRATA_FP8_E4M3_B128
         self.n_tok, self.n_items = R * T, R * T * K
@@ -320,6 +332,8 @@ class MoEContext:
         rc, h = strata_ctx_create(self.shape, device)
         _check(rc, "strata_ctx_create")
         self.h = h
+        rc, self.recv_rows = strata_moe_recv_rows(self.shape)     # rows a receive buffer must hold
+        _check(rc, "strata_moe_recv_rows")
         rc, nbytes = strata_moe_workspace_bytes(self.shape)
         _check(rc, "strata_moe_workspace_bytes")
         self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
@@ -367,7 +381,7 @@ class MoEContext:
         return base.view(torch.uint8).reshape(-1)[off:off + nbytes].view(dtype).reshape(*shape)
 
     def new_layout(self, with_optional: bool = True) -> Layout:
-        return Layout(self.R, self.T, self.K, self.E, self.device, with_optional)
+        return Layout(self.R, self.T, self.K, self.E, self.device, with_optional, self.recv_rows)
 
     # hot path ---------------------------------------------------------------
     def layout(self, ids, layout: Optional[Layout] = None) -> Layout:

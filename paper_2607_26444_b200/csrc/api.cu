@@ -42,6 +42,13 @@ namespace {
 
 using namespace strata;
 
+// rows of the receive buffer: all items plus the worst-case padding of aligned segments
+long long recv_rows(const strata_moe_shape& s)
+{
+    const long long pad = s.segment_align > 1 ? s.segment_align - 1 : 0;
+    return (long long)s.R * s.T * s.K + (long long)s.E * pad;
+}
+
 strata_status check_shape(const strata_moe_shape* s)
 {
     if (!s) return STRATA_ERR_INVALID_ARG;
@@ -50,8 +57,9 @@ strata_status check_shape(const strata_moe_shape* s)
     if (s->H % 8 != 0) return STRATA_ERR_SHAPE;
     if (s->dispatch_dtype != STRATA_BF16 && s->dispatch_dtype != STRATA_FP8_E4M3_B128) return STRATA_ERR_SHAPE;
     if (s->dispatch_dtype == STRATA_FP8_E4M3_B128 && s->H % 128 != 0) return STRATA_ERR_SHAPE;
-    const long long n = (long long)s->R * s->T * s->K;
-    if (n >= (1ll << 31)) return STRATA_ERR_SHAPE;
+    if (s->segment_align < 0 || s->segment_align > 65536) return STRATA_ERR_SHAPE;
+    if ((s->flags & ~STRATA_FLAG_ALLOW_UNROUTED) != 0) return STRATA_ERR_SHAPE;
+    if (recv_rows(*s) >= (1ll << 31)) return STRATA_ERR_SHAPE;
     return STRATA_OK;
 }
 
@@ -197,6 +205,15 @@ strata_status strata_moe_workspace_bytes(const strata_moe_shape* shape, size_t* 
     return STRATA_OK;
 }
 
+strata_status strata_moe_recv_rows(const strata_moe_shape* shape, size_t* rows)
+{
+    if (!rows) return STRATA_ERR_INVALID_ARG;
+    strata_status st = check_shape(shape);
+    if (st != STRATA_OK) return st;
+    *rows = (size_t)recv_rows(*shape);
+    return STRATA_OK;
+}
+
 strata_status strata_ctx_set_workspace(strata_ctx* ctx, void* dptr, size_t bytes)
 {
     if (!ctx || !dptr) return STRATA_ERR_INVALID_ARG;
@@ -338,7 +355,7 @@ strata_status strata_moe_dispatch(strata_ctx* ctx, const strata_moe_layout_t* la
     if (!aligned16(x) || !aligned16(recv)) return STRATA_ERR_ALIGNMENT;
     if (fp8 && (reinterpret_cast<uintptr_t>(recv_scale) & 3u) != 0) return STRATA_ERR_ALIGNMENT;
     if (!ctx->ws) return STRATA_ERR_WORKSPACE;
-    const size_t n_rows = (size_t)s.R * s.T * s.K;
+    const size_t n_rows = (size_t)recv_rows(s);
     if (capacity_rows < n_rows) return STRATA_ERR_CAPACITY;
     const size_t row_bytes = fp8 ? (size_t)s.H : (size_t)s.H * 2;
     {
@@ -454,7 +471,7 @@ strata_status strata_moe_dispatch_windows(strata_ctx* ctx, const strata_moe_layo
     if (n_cores < 1 || n_cores > partition_max_cores_supported()) return STRATA_ERR_SHAPE;
     if (!aligned16(x) || !aligned16(recv)) return STRATA_ERR_ALIGNMENT;
     if (!ctx->ws) return STRATA_ERR_WORKSPACE;
-    const size_t n_rows = (size_t)s.R * s.T * s.K;
+    const size_t n_rows = (size_t)recv_rows(s);
     if (capacity_rows < n_rows) return STRATA_ERR_CAPACITY;
     {
         std::lock_guard<std::mutex> lk(ctx->mu);
@@ -522,9 +539,10 @@ strata_status strata_moe_roundtrip_host(strata_ctx* ctx, const strata_moe_device
     if (!aligned16(dev->x) || !aligned16(dev->recv) || !aligned16(dev->out)) return STRATA_ERR_ALIGNMENT;
     if (!ctx->ws) return STRATA_ERR_WORKSPACE;
     const size_t n_tok = (size_t)s.R * s.T, n = n_tok * s.K, row_bytes = (size_t)s.H * 2;
+    const size_t n_recv = (size_t)recv_rows(s);
     {
         std::lock_guard<std::mutex> lk(ctx->mu);
-        if (!region_contains(ctx, dev->recv, n * row_bytes)) return STRATA_ERR_NOT_REGISTERED;
+        if (!region_contains(ctx, dev->recv, n_recv * row_bytes)) return STRATA_ERR_NOT_REGISTERED;
     }
     if (ctx->device < 0) return STRATA_ERR_CUDA;
     DeviceGuard g(ctx->device);
@@ -581,10 +599,10 @@ strata_status strata_moe_roundtrip_host(strata_ctx* ctx, const strata_moe_device
             dq = dispatch_queue(ctx);
             cq = combine_queue(ctx);
         }
-        cudaError_t err = launch_dispatch_bf16(sub, dev->layout.dst_row + a * s.K, dx + a * row_bytes, dev->recv, n,
+        cudaError_t err = launch_dispatch_bf16(sub, dev->layout.dst_row + a * s.K, dx + a * row_bytes, dev->recv, n_recv,
                                                ctx->ws, dq, ctx->n_sm, TraceBuf{nullptr, 0}, st);
         if (err == cudaSuccess)
-            err = launch_combine(sub, dev->layout.dst_row + a * s.K, dev->recv, n, dev->w + a * s.K,
+            err = launch_combine(sub, dev->layout.dst_row + a * s.K, dev->recv, n_recv, dev->w + a * s.K,
                                  dout + a * row_bytes, ctx->ws, cq, ctx->n_sm, TraceBuf{nullptr, 0}, st);
         {
             std::lock_guard<std::mutex> lk(ctx->mu);

@@ -90,7 +90,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
         for (int k = 0; k < K; ++k) {
             const int row = p.dst_row[(long long)n * K + k];
             const bool row_ok = row >= 0 && row < p.y_rows;
-            if (!row_ok && tid == 0 && part == 0) report_status(p.status, STRATA_ERR_BAD_ROW);
+            if (!row_ok && row != -1 && tid == 0 && part == 0) report_status(p.status, STRATA_ERR_BAD_ROW);
             src[k] = row_ok ? p.y + (size_t)row * row_bytes : nullptr;
             wk[k] = p.w[(long long)n * K + k];
         }
@@ -144,7 +144,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel<0>(CombinePara
         if (tid < K) {
             const int row = p.dst_row[(long long)n * K + tid];
             const bool row_ok = row >= 0 && row < p.y_rows;
-            if (!row_ok) report_status(p.status, STRATA_ERR_BAD_ROW);
+            if (!row_ok && row != -1) report_status(p.status, STRATA_ERR_BAD_ROW);
             s_off[tid] = row_ok ? (long long)row * (long long)row_bytes : -1;
             s_w[tid] = p.w[(long long)n * K + tid];
         }

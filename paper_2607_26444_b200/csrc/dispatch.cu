@@ -132,7 +132,7 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
 
         const int my_row = (lane < p.K) ? p.dst_row[tok * p.K + lane] : -1;
         const bool row_ok = (lane >= p.K) || (my_row >= 0 && my_row < p.capacity_rows);
-        if (!row_ok) report_status(p.status, STRATA_ERR_BAD_ROW);
+        if (!row_ok && my_row != -1) report_status(p.status, STRATA_ERR_BAD_ROW);
 
         ok = mbar_wait_bounded(&bars[s], parity);
         ok = __all_sync(0xffffffffu, ok);
@@ -252,7 +252,7 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
         if (tid < p.K) {
             const int row = p.dst_row[tok * p.K + tid];
             const bool row_ok = row >= 0 && row < p.capacity_rows;
-            if (!row_ok) report_status(p.status, STRATA_ERR_BAD_ROW);
+            if (!row_ok && row != -1) report_status(p.status, STRATA_ERR_BAD_ROW);
             s_rows[tid] = row_ok ? row : -1;
         }
         if (tid == 0) bulk_wait_read<1>();     // stores of unit j-2 have left out_stage(s)

@@ -36,7 +36,11 @@ struct LayoutParams {
     int* tile_cnt;
     int R, E, e_loc;
     int items_per_rank, tiles_per_rank, n_tiles;
+    int align;            // >= 1: rows every expert segment is padded to
+    int allow_unrouted;   // id -1 is legal and means "not routed"
 };
+
+__device__ __forceinline__ int round_up_rows(int n, int a) { return (n + a - 1) / a * a; }
 
 // Lanes of the warp holding the same key (0 <= key < 2^nbits), from nbits ballots.  Invalid lanes
 // (key < 0) get a mask of the other invalid lanes, which callers ignore.  Measured several times
@@ -119,7 +123,7 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_count_scan_kernel(Layou
         bool valid = in_rank < p.items_per_rank;
         int e = ids[q];
         if (valid && (unsigned)e >= (unsigned)E) {
-            report_status(p.status, STRATA_ERR_BAD_EXPERT_ID);
+            if (!(p.allow_unrouted && e == -1)) report_status(p.status, STRATA_ERR_BAD_EXPERT_ID);
             valid = false;
             e = -1;
         }
@@ -186,13 +190,15 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_count_scan_kernel(Layou
         }
     }
 
-    // exclusive scan over experts (one expert per thread of group 0)
-    const int v = (tid < E) ? count_e : 0;
+    // exclusive scan over experts of the padded segment lengths (one expert per thread of group 0)
+    const int v = (tid < E) ? round_up_rows(count_e, p.align) : 0;
     const int off = block_exclusive_scan_1024(v, warp_sums, total);
     if (tid < E) {
         p.expert_count[tid] = count_e;
         p.expert_offset[tid] = off;
         offs[tid] = off;
+        if (p.src_of_row)                 // padding rows of this segment have no source item
+            for (int row = off + count_e; row < off + v; ++row) p.src_of_row[row] = -1;
     }
     if (tid == 0) {
         p.expert_offset[E] = *total;
@@ -201,9 +207,10 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_count_scan_kernel(Layou
     }
     __syncthreads();
     for (int d = tid; d < p.R; d += kLayoutThreads) {
-        const int lo = offs[d * p.e_loc], hi = offs[(d + 1) * p.e_loc];
-        p.rank_offset[d] = lo;
-        p.rank_count[d] = hi - lo;
+        p.rank_offset[d] = offs[d * p.e_loc];
+        int real = 0;
+        for (int e2 = d * p.e_loc; e2 < (d + 1) * p.e_loc; ++e2) real += p.expert_count[e2];
+        p.rank_count[d] = real;
     }
 
     // per-tile exclusive prefix (within the expert, across tiles in order).  The prefix at the first
@@ -334,13 +341,14 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_cluster_kernel(LayoutPa
     cg::cluster_group cluster = cg::this_cluster();
     const int n_cta = (int)cluster.num_blocks(), cta = (int)cluster.block_rank();
 
-    extern __shared__ int sm[];          // warp_cnt[32*E] | offs[E+1] | cta_cnt[E] | warp_sums[32] | total[2] | src_cnt[R*E]
+    extern __shared__ int sm[];          // warp_cnt[32*E] | offs[E+1] | cta_cnt[E] | all_cnt[E] | warp_sums[32] | total[2] | src_cnt[R*E]
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int E = p.E;
     int* warp_cnt = sm;
     int* offs = sm + 32 * E;
-    int* cta_cnt = offs + E + 1;
-    int* warp_sums = cta_cnt + E;
+    int* cta_cnt = offs + E + 1;          // this CTA's per-expert totals, read by the other CTAs of the cluster
+    int* all_cnt = cta_cnt + E;           // cluster-wide per-expert counts (local copy)
+    int* warp_sums = all_cnt + E;
     int* total = warp_sums + 32;
     int* src_cnt = total + 2;             // [R*E], only when src_expert_count is wanted
     int* mine = warp_cnt + wid * E;
@@ -372,7 +380,7 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_cluster_kernel(LayoutPa
         int e = ids[q];
         bool valid = i < n_items;
         if (valid && (unsigned)e >= (unsigned)E) {
-            report_status(p.status, STRATA_ERR_BAD_EXPERT_ID);
+            if (!(p.allow_unrouted && e == -1)) report_status(p.status, STRATA_ERR_BAD_EXPERT_ID);
             valid = false;
         }
         if (!valid) e = -1;
@@ -422,13 +430,19 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_cluster_kernel(LayoutPa
             count_e += v[c];
         }
     }
-    const int off = block_exclusive_scan_1024(count_e, warp_sums, total);
-    if (tid < E) offs[tid] = off;
+    const int padded = round_up_rows(count_e, p.align);
+    const int off = block_exclusive_scan_1024(tid < E ? padded : 0, warp_sums, total);
+    if (tid < E) {
+        offs[tid] = off;
+        all_cnt[tid] = count_e;
+    }
     if (tid == 0) offs[E] = *total;
     if (cta == 0) {
         if (tid < E) {
             p.expert_count[tid] = count_e;
             p.expert_offset[tid] = off;
+            if (p.src_of_row)             // padding rows of this segment have no source item
+                for (int row = off + count_e; row < off + padded; ++row) p.src_of_row[row] = -1;
         }
         if (tid == 0) {
             p.expert_offset[E] = *total;
@@ -438,9 +452,10 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_cluster_kernel(LayoutPa
     __syncthreads();
     if (cta == 0)
         for (int d = tid; d < p.R; d += kLayoutThreads) {
-            const int lo = offs[d * p.e_loc], hi = offs[(d + 1) * p.e_loc];
-            p.rank_offset[d] = lo;
-            p.rank_count[d] = hi - lo;
+            p.rank_offset[d] = offs[d * p.e_loc];
+            int real = 0;
+            for (int e2 = d * p.e_loc; e2 < (d + 1) * p.e_loc; ++e2) real += all_cnt[e2];
+            p.rank_count[d] = real;
         }
     if (p.src_expert_count) {             // CTA c sums its contiguous slice of the per-source-rank table
         const int slice = (p.R * E + n_cta - 1) / n_cta;
@@ -491,7 +506,7 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_cluster_kernel(LayoutPa
 // shared memory of the cluster kernel; the per-source-rank table is only there when asked for
 size_t small_smem(int E, int R, bool with_src)
 {
-    return (size_t)(32 * E + E + 1 + E + 32 + 2 + (with_src ? R * E : 0)) * sizeof(int);
+    return (size_t)(32 * E + E + 1 + E + E + 32 + 2 + (with_src ? R * E : 0)) * sizeof(int);
 }
 constexpr size_t kSmallSmemLimit = 200 * 1024;
 
@@ -534,6 +549,8 @@ cudaError_t launch_layout(const strata_moe_shape& s, const int32_t* ids, const s
     p.items_per_rank = g.items_per_rank;
     p.tiles_per_rank = g.tiles_per_rank;
     p.n_tiles = g.n_tiles;
+    p.align = s.segment_align > 1 ? s.segment_align : 1;
+    p.allow_unrouted = (s.flags & STRATA_FLAG_ALLOW_UNROUTED) ? 1 : 0;
 
     const long long n_items = (long long)s.R * s.T * s.K;
     const size_t small_bytes = small_smem(s.E, s.R, L.src_expert_count != nullptr);
@@ -618,7 +635,9 @@ extern "C" strata_status strata_moe_layout_noalloc(const strata_moe_shape* shape
     const strata_moe_shape& s = *shape;
     if (s.R <= 0 || s.T <= 0 || s.E <= 0 || s.K <= 0) return STRATA_ERR_SHAPE;
     if (s.E % s.R != 0 || s.E > kMaxExperts || s.K > kMaxTopK) return STRATA_ERR_SHAPE;
-    if ((long long)s.R * s.T * s.K >= (1ll << 31)) return STRATA_ERR_SHAPE;
+    if (s.segment_align < 0 || s.segment_align > 65536) return STRATA_ERR_SHAPE;
+    if ((long long)s.R * s.T * s.K + (long long)s.E * (s.segment_align > 1 ? s.segment_align - 1 : 0) >= (1ll << 31))
+        return STRATA_ERR_SHAPE;
     const LayoutGeom g = layout_geom(s);
     const size_t need = (size_t)kWsHeaderBytes + (size_t)g.n_tiles * s.E * sizeof(int);
     if (need > kStaticScratchBytes) return STRATA_ERR_CAPACITY;     // beyond the fixed array: use a workspace
@@ -650,6 +669,8 @@ extern "C" strata_status strata_moe_layout_noalloc(const strata_moe_shape* shape
     p.items_per_rank = g.items_per_rank;
     p.tiles_per_rank = g.tiles_per_rank;
     p.n_tiles = g.n_tiles;
+    p.align = s.segment_align > 1 ? s.segment_align : 1;
+    p.allow_unrouted = (s.flags & STRATA_FLAG_ALLOW_UNROUTED) ? 1 : 0;
     layout_count_scan_kernel<<<g.n_tiles, kLayoutThreads, count_scan_smem(s.E), st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return STRATA_ERR_CUDA;
     layout_rank_kernel<<<g.n_tiles, kLayoutThreads, (size_t)32 * s.E * sizeof(int), st>>>(p);

@@ -292,7 +292,7 @@ def test_bad_expert_id_is_skipped_and_reported():
     whole, recv = guarded(N, cfg.H, torch.int16, -1)
     ctx.register(whole)
     ctx.dispatch(lay, to_dev(inp["x"]), recv)
-    assert ctx.device_status() == B.STRATA_ERR_BAD_ROW
+    assert ctx.device_status() == B.STRATA_OK               # the layout already reported; -1 rows are just skipped
     hw = whole.cpu().numpy()
     assert np.all(hw[:GUARD] == -1) and np.all(hw[GUARD + N - 2:] == -1)
     x2 = inp["x"].reshape(cfg.n_tok, cfg.H)
@@ -301,7 +301,15 @@ def test_bad_expert_id_is_skipped_and_reported():
     # combine ignores the skipped slots
     out = torch.zeros((cfg.n_tok, cfg.H), dtype=torch.int16, device=DEV)
     ctx.combine(lay, recv, to_dev(inp["w"]), out)
+    assert ctx.device_status() == B.STRATA_OK
+    # a destination row that is neither valid nor -1 is reported
+    lay.dst_row.view(-1)[5] = cfg.n_items + 100
+    ctx.dispatch(lay, to_dev(inp["x"]), recv)
     assert ctx.device_status() == B.STRATA_ERR_BAD_ROW
+    ctx.combine(lay, recv, to_dev(inp["w"]), out)
+    assert ctx.device_status() == B.STRATA_ERR_BAD_ROW
+    hw = whole.cpu().numpy()
+    assert np.all(hw[:GUARD] == -1) and np.all(hw[GUARD + N:] == -1)      # still nothing out of bounds
     ctx.close()
 
 
@@ -443,3 +451,72 @@ def test_random_shapes(seed):
                     routing="zipf" if seed % 3 == 0 else "uniform",
                     expert=["identity", "scale", "affine"][seed % 3])
     run_full_case(cfg, threads=8)
+
+
+# ---- production layout variants: aligned segments and the "not routed" sentinel -----------------
+
+@pytest.mark.parametrize("kw,align,frac", [
+    (dict(R=4, T=128, H=1024, E=16, K=2), 128, 0.0),
+    (dict(R=4, T=128, H=1024, E=16, K=2), 1, 0.25),
+    (dict(R=8, T=300, H=512, E=64, K=6), 16, 0.2),            # cluster layout
+    (dict(R=16, T=128, H=7168, E=256, K=8), 128, 0.1),        # decode shape
+    (dict(R=8, T=2000, H=256, E=32, K=4), 64, 0.3),           # tiled layout (64,000 items)
+    (dict(R=2, T=50, H=128, E=4, K=2), 7, 1.0),               # nothing routed at all, odd alignment
+], ids=lambda v: str(v).replace(" ", "") if not isinstance(v, dict) else "R{R}T{T}H{H}E{E}K{K}".format(**v))
+def test_aligned_segments_and_unrouted_slots(kw, align, frac):
+    cfg = wl.shrink(wl.CONFIGS["tiny"], seed=4321, **kw)
+    inp = wl.generate(cfg)
+    ids = inp["ids"].copy()
+    rng = np.random.default_rng(11)
+    ids[rng.random(ids.shape) < frac] = -1
+    ref = oracle.layout(ids, cfg.E, segment_align=align, allow_unrouted=True)
+    ctx = B.MoEContext(cfg.R, cfg.T, cfg.H, cfg.E, cfg.K, segment_align=align, allow_unrouted=True)
+    n_rows = ctx.recv_rows
+    assert n_rows == cfg.n_items + cfg.E * (max(align, 1) - 1)
+    lay = ctx.layout(to_dev(ids))
+    torch.cuda.synchronize()
+    assert ctx.device_status() == B.STRATA_OK
+    total = int(ref["expert_offset"][cfg.E])
+    for key in ("expert_count", "expert_offset", "rank_count", "rank_offset", "src_expert_count", "dst_row"):
+        assert np.array_equal(getattr(lay, key).cpu().numpy(), ref[key]), key
+    assert np.array_equal(lay.src_of_row.cpu().numpy()[:total], ref["src_of_row"])
+
+    whole, recv = guarded(n_rows, cfg.H, torch.int16, SENTINEL16)
+    ctx.register(whole)
+    x_d, w_d = to_dev(inp["x"]), to_dev(inp["w"])
+    ctx.dispatch(lay, x_d, recv)
+    want = oracle.dispatch_bf16(ref["dst_row"], inp["x"], nthreads=4, n_rows=n_rows)
+    got = u16(recv)
+    written = np.zeros(n_rows, bool)
+    written[ref["dst_row"][ref["dst_row"] >= 0]] = True
+    assert np.array_equal(got[written], want[written])
+    assert np.all(got[~written] == SENTINEL16)                       # padding rows are never touched
+    hw = u16(whole)
+    assert np.all(hw[:GUARD] == SENTINEL16) and np.all(hw[GUARD + n_rows:] == SENTINEL16)
+
+    out = torch.empty((cfg.n_tok, cfg.H), dtype=torch.int16, device=DEV)
+    ctx.combine(lay, recv, w_d, out)
+    want_out = oracle.combine(ref["dst_row"], want, inp["w"], nthreads=4)
+    assert np.array_equal(u16(out), want_out)
+    assert ctx.device_status() == B.STRATA_OK
+
+    # the allocation-free layout entry honours the same two options
+    got2 = ctx.new_layout()
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    rc = B.strata_moe_layout_noalloc(ctx.shape, to_dev(ids).data_ptr(), got2.c, status.data_ptr(),
+                                     torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert rc == 0 and status.item() == 0
+    assert torch.equal(got2.dst_row, lay.dst_row) and torch.equal(got2.expert_offset, lay.expert_offset)
+    assert torch.equal(got2.src_of_row[:total], lay.src_of_row[:total])
+    ctx.close()
+
+
+def test_minus_one_is_an_error_without_the_flag():
+    cfg = wl.shrink(wl.CONFIGS["tiny"], H=64)
+    ids = wl.gen_topk_ids(cfg)
+    ids[0, 3, 1] = -1
+    ctx = make_ctx(cfg)
+    ctx.layout(to_dev(ids))
+    assert ctx.device_status() == B.STRATA_ERR_BAD_EXPERT_ID
+    ctx.close()
