@@ -17,6 +17,11 @@
  *    receive buffer, a bounded wait that ran out) set a device status word
  *    (first error wins), the offending item is skipped, nothing is accessed
  *    out of bounds, and the error is reported by strata_device_status().
+ *  - One context serves one stream of work: its calls must reach the GPU in the order they were
+ *    made (issue them to one stream, or order the streams yourself).  The workspace holds state
+ *    that consecutive launches hand to each other (work-claim counters, the layout ticket, the
+ *    status word); two calls on the same context whose kernels could overlap would corrupt it.
+ *    Use one context per concurrent stream.
  *  - Index convention: rank r in [0,R), token t in [0,T), slot k in [0,K);
  *    flat item i = (r*T + t)*K + k; token n = r*T + t; N = R*T*K.
  *    Expert e belongs to rank e / (E/R).  All R ranks are partitions of one
