@@ -28,7 +28,6 @@ struct strata_ctx {
     size_t ws_bytes;
     uint64_t next_region;
     uint64_t launches;
-    uint64_t n_dispatch, n_combine;      // launches so far: their parity selects the work-claim counter
     strata::TraceBuf trace;
     // host round trip only: copy streams and events, created on first use (no device memory)
     cudaStream_t s_in = nullptr, s_out = nullptr;
@@ -70,21 +69,8 @@ size_t workspace_bytes(const strata_moe_shape& s)
     return (b + 255) & ~(size_t)255;
 }
 
-// Counter pair of a kernel type; consecutive successful launches alternate (see WorkQueue).  The
-// parity only advances when a launch succeeded, so the counter a launch claims from is always the
-// one that the launch before it has zeroed.
-WorkQueue dispatch_queue(const strata_ctx* c)
-{
-    unsigned int* w = reinterpret_cast<unsigned int*>(c->ws) + 2;
-    const unsigned int k = (unsigned int)(c->n_dispatch & 1);
-    return WorkQueue{w + k, w + (k ^ 1)};
-}
-WorkQueue combine_queue(const strata_ctx* c)
-{
-    unsigned int* w = reinterpret_cast<unsigned int*>(c->ws) + 4;
-    const unsigned int k = (unsigned int)(c->n_combine & 1);
-    return WorkQueue{w + k, w + (k ^ 1)};
-}
+WorkQueue dispatch_queue(const strata_ctx* c) { return WorkQueue{reinterpret_cast<unsigned int*>(c->ws) + 2}; }
+WorkQueue combine_queue(const strata_ctx* c) { return WorkQueue{reinterpret_cast<unsigned int*>(c->ws) + 4}; }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -174,7 +160,6 @@ strata_status strata_ctx_create(strata_ctx** out, const strata_moe_shape* shape,
     c->ws_bytes = 0;
     c->next_region = 1;
     c->launches = 0;
-    c->n_dispatch = c->n_combine = 0;
     c->trace = strata::TraceBuf{nullptr, 0};
     *out = c;
     return STRATA_OK;
@@ -375,7 +360,6 @@ strata_status strata_moe_dispatch(strata_ctx* ctx, const strata_moe_layout_t* la
     {
         std::lock_guard<std::mutex> lk(ctx->mu);
         ctx->launches += 1;
-        if (err == cudaSuccess) ctx->n_dispatch += 1;
     }
     return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
 }
@@ -396,7 +380,6 @@ strata_status strata_moe_combine(strata_ctx* ctx, const strata_moe_layout_t* lay
     {
         std::lock_guard<std::mutex> lk(ctx->mu);
         ctx->launches += 1;
-        if (err == cudaSuccess) ctx->n_combine += 1;
     }
     return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
 }
@@ -518,7 +501,9 @@ strata_status strata_device_status(strata_ctx* ctx, void* stream, strata_status*
         return STRATA_ERR_CUDA;
     }
     if (word != 0) {
-        if (cudaMemsetAsync(ctx->ws, 0, sizeof(int), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) {
+        // clear the status word; after an error also the ticket and the work-claim counters, which a
+        // kernel that gave up may have left non-zero (header words 0..5)
+        if (cudaMemsetAsync(ctx->ws, 0, 6 * sizeof(int), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) {
             cudaGetLastError();
             return STRATA_ERR_CUDA;
         }
@@ -607,10 +592,6 @@ strata_status strata_moe_roundtrip_host(strata_ctx* ctx, const strata_moe_device
         {
             std::lock_guard<std::mutex> lk(ctx->mu);
             ctx->launches += 2;
-            if (err == cudaSuccess) {
-                ctx->n_dispatch += 1;
-                ctx->n_combine += 1;
-            }
         }
         if (err != cudaSuccess) {
             cudaGetLastError();

@@ -71,13 +71,13 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
     const unsigned int n_units = (unsigned int)(p.n_tok * p.parts);
     __shared__ unsigned int s_next[2];             // the claim made during unit j is read for unit j+1
     griddep_wait();
-    arm_next_queue(p.wq);
     if (tid == 0) trace_begin(p.trace);
 
     unsigned int u = blockIdx.x < n_units ? blockIdx.x : kNoUnit;
+    bool exhausted = false;                        // thread 0's view of the queue
     for (int j = 0; u != kNoUnit; ++j) {
         if (tid == 0) {
-            const unsigned int nx = claim_unit(p.wq, n_units, gridDim.x);
+            const unsigned int nx = claim_unit(p.wq, n_units, gridDim.x, exhausted);
             s_next[j & 1] = nx;
             if (nx == kNoUnit) griddep_launch_dependents();   // last unit of this CTA: let the next kernel in
         }
@@ -131,13 +131,13 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel<0>(CombinePara
     __shared__ float s_w[kMaxTopK];
     __shared__ unsigned int s_tok;
     griddep_wait();
-    arm_next_queue(p.wq);
     if (tid == 0) trace_begin(p.trace);
 
+    bool exhausted = false;
     for (int j = 0;; ++j) {
         __syncthreads();                           // everyone is done with the previous token's tables
         if (tid == 0) s_tok = j == 0 ? (blockIdx.x < n_units ? blockIdx.x : kNoUnit)
-                                     : claim_unit(p.wq, n_units, gridDim.x);
+                                     : claim_unit(p.wq, n_units, gridDim.x, exhausted);
         __syncthreads();
         const unsigned int n = s_tok;
         if (n == kNoUnit) break;

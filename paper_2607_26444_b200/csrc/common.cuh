@@ -11,8 +11,7 @@ namespace strata {
 // ---- workspace layout -----------------------------------------------------
 // word 0: device status (a strata_status, first error wins)
 // word 1: ticket of the layout kernel (returns to 0 after every call)
-// words 2,3: the two work-claim counters of dispatch (launches alternate between them)
-// words 4,5: the same for combine
+// word 2: work-claim counter of dispatch, word 4: of combine (both return to 0 inside the kernel)
 // bytes [256, ...): per-tile, per-expert counts, int32 [n_tiles, E]
 constexpr int kWsHeaderBytes = 256;
 constexpr int kLayoutThreads = 1024;   // threads per layout CTA
@@ -43,12 +42,11 @@ inline LayoutGeom layout_geom(const strata_moe_shape& s)
 // kernel time (the split is even in bytes, the memory system is not even in service), and claiming
 // lifts the dispatch pattern from 5.7 to 6.6 TB/s.  This is the SM-side answer to the core-level
 // long tails that the paper's workload-balanced partitioning removes (Sec. 6.2).
-// Each kernel type owns two counters and its launches alternate between them: a launch claims from
-// one and, once the launch before it has completed (after griddep_wait), zeroes the other for the
-// launch after it.  Nothing has to be reset at the end of a kernel.
+// Every CTA stops claiming at its first failed claim, so a launch makes exactly gridDim.x failed
+// claims; the CTA that draws the last of them puts the counter back to zero.  Nothing waits, nothing
+// is reset from the host, and a launch replayed from a CUDA graph finds the counter as it needs it.
 struct WorkQueue {
-    unsigned int* next;    // device: next unclaimed unit of this launch
-    unsigned int* other;   // device: the counter the next launch will use; zeroed by this launch
+    unsigned int* next;    // device: next unclaimed unit; zero between launches
 };
 constexpr unsigned int kNoUnit = 0xffffffffu;
 
@@ -187,20 +185,20 @@ __device__ __forceinline__ void trace_end(const TraceBuf& t)
     if (t.slots && (int)blockIdx.x < t.capacity) t.slots[2 * blockIdx.x + 1] = global_timer_ns();
 }
 
-// One thread claims; returns kNoUnit when the queue is exhausted.  Units below `base` were dealt
-// statically (every CTA starts on units it knows without asking: same-address atomics complete at
-// roughly one per 3.5 ns, so a burst of one claim per CTA at launch would cost microseconds).
-__device__ __forceinline__ unsigned int claim_unit(const WorkQueue& q, unsigned int n_units, unsigned int base)
+// One thread per CTA claims; returns kNoUnit when the queue is exhausted.  Units below `base` were
+// dealt statically (every CTA starts on units it knows without asking: same-address atomics complete
+// at roughly one per 3.5 ns, so a burst of one claim per CTA at launch would cost microseconds).
+// `exhausted` is the caller's per-CTA flag: after the first failed claim the counter is left alone.
+__device__ __forceinline__ unsigned int claim_unit(const WorkQueue& q, unsigned int n_units, unsigned int base,
+                                                   bool& exhausted)
 {
-    if (base >= n_units) return kNoUnit;           // everything was dealt statically: no traffic at all
-    const unsigned int u = base + atomicAdd(q.next, 1u);
-    return u < n_units ? u : kNoUnit;
-}
-// Called by every thread right after griddep_wait(): one thread of the grid re-arms the counter
-// of the next launch (the launch that last used it has completed by now).
-__device__ __forceinline__ void arm_next_queue(const WorkQueue& q)
-{
-    if (blockIdx.x == 0 && threadIdx.x == 0) *q.other = 0;
+    if (base >= n_units || exhausted) return kNoUnit;        // all static, or already failed once
+    const unsigned int old = atomicAdd(q.next, 1u);
+    if (base + old < n_units) return base + old;
+    exhausted = true;
+    // failed claims are numbered n_units-base .. n_units-base+gridDim.x-1; the last one re-arms the queue
+    if (old == n_units - base + gridDim.x - 1) *q.next = 0;
+    return kNoUnit;
 }
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p)

@@ -81,7 +81,6 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
     __syncwarp();
     const uint64_t pol = policy_evict_first();
     griddep_wait();                       // x and dst_row belong to earlier kernels in the stream
-    arm_next_queue(p.wq);
     if (lane == 0) trace_begin(p.trace);
 
     auto decode = [&](unsigned int u, long long& tok, uint32_t& col0, uint32_t& bytes) {
@@ -90,7 +89,7 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
         col0 = ch * p.chunk_cols;
         bytes = min(p.chunk_cols, (uint32_t)p.H - col0) * 2u;
     };
-    bool triggered = false;
+    bool triggered = false, exhausted = false;
     // The first stages-1 units of a CTA are fixed (blockIdx + j*grid); the rest are claimed.
     const unsigned int n_static = (unsigned int)(kBf16Stages - 1) * gridDim.x;
     auto issue_load = [&](long long j) {   // lane 0 only: next unit into stage j % stages
@@ -100,7 +99,7 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
             u = blockIdx.x + (unsigned int)j * gridDim.x;
             if (u >= n_units) u = kNoUnit;
         } else {
-            u = claim_unit(p.wq, n_units, n_static);
+            u = claim_unit(p.wq, n_units, n_static, exhausted);
         }
         s_unit[s] = u;
         if (u == kNoUnit) {
@@ -201,7 +200,6 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
     __syncthreads();
     const uint64_t pol = policy_evict_first();
     griddep_wait();
-    arm_next_queue(p.wq);
     if (tid == 0) trace_begin(p.trace);
 
     auto decode = [&](unsigned int u, long long& tok, uint32_t& col0, uint32_t& cols) {
@@ -210,7 +208,7 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
         col0 = ch * p.chunk_cols;
         cols = min(p.chunk_cols, (uint32_t)p.H - col0);
     };
-    bool triggered = false;
+    bool triggered = false, exhausted = false;
     const unsigned int n_static = 2u * gridDim.x;   // the first two units of a CTA are fixed
     auto issue_load = [&](long long j) {   // thread 0 only
         const int s = (int)(j & 1);
@@ -219,7 +217,7 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
             u = blockIdx.x + (unsigned int)j * gridDim.x;
             if (u >= n_units) u = kNoUnit;
         } else {
-            u = claim_unit(p.wq, n_units, n_static);
+            u = claim_unit(p.wq, n_units, n_static, exhausted);
         }
         s_unit[s] = u;
         if (u == kNoUnit) {

@@ -520,3 +520,50 @@ def test_minus_one_is_an_error_without_the_flag():
     ctx.layout(to_dev(ids))
     assert ctx.device_status() == B.STRATA_ERR_BAD_EXPERT_ID
     ctx.close()
+
+
+@pytest.mark.parametrize("kw", [dict(R=4, T=300, H=512, E=16, K=4),          # cluster layout, claimed units
+                                dict(R=8, T=1200, H=256, E=32, K=4)],         # tiled layout (38,400 items)
+                         ids=lambda kw: "R{R}T{T}H{H}E{E}K{K}".format(**kw))
+def test_cuda_graph_replay(kw):
+    """layout -> dispatch -> combine captured once in a CUDA graph and replayed on new inputs: every
+    piece of state the kernels hand from one launch to the next (ticket, work-claim counters) is
+    restored by the kernels themselves, so a replay computes the same as a fresh call."""
+    cfg = wl.shrink(wl.CONFIGS["decode"], seed=1, **kw)
+    ctx = make_ctx(cfg)
+    first = wl.generate(cfg)
+    ids_d, x_d, w_d = to_dev(first["ids"]), to_dev(first["x"]), to_dev(first["w"])
+    lay = ctx.new_layout()
+    recv = torch.empty((cfg.n_items, cfg.H), dtype=torch.int16, device=DEV)
+    out = torch.empty((cfg.n_tok, cfg.H), dtype=torch.int16, device=DEV)
+    ctx.register(recv)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for _ in range(2):                         # warm-up outside the capture
+            ctx.layout(ids_d, lay)
+            ctx.dispatch(lay, x_d, recv)
+            ctx.combine(lay, recv, w_d, out)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        ctx.layout(ids_d, lay)
+        ctx.dispatch(lay, x_d, recv)
+        ctx.combine(lay, recv, w_d, out)
+    for rep in range(4):
+        inp = wl.generate(wl.shrink(cfg, seed=100 + rep))
+        ids_d.copy_(to_dev(inp["ids"]))
+        x_d.copy_(to_dev(inp["x"]))
+        w_d.copy_(to_dev(inp["w"]))
+        recv.fill_(SENTINEL16)
+        out.fill_(SENTINEL16)
+        g.replay()
+        torch.cuda.synchronize()
+        ref = oracle.layout(inp["ids"], cfg.E)
+        assert np.array_equal(lay.dst_row.cpu().numpy(), ref["dst_row"]), rep
+        ref_recv = oracle.dispatch_bf16(ref["dst_row"], inp["x"], nthreads=4)
+        assert np.array_equal(u16(recv), ref_recv), rep
+        assert np.array_equal(u16(out), oracle.combine(ref["dst_row"], ref_recv, inp["w"], nthreads=4)), rep
+    assert ctx.device_status() == B.STRATA_OK
+    ctx.close()
