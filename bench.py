@@ -294,6 +294,28 @@ def per_call_us(case: DeviceCase, iters: int = 30, warmup: int = 3):
         torch.cuda.synchronize()
         ts = sorted(ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(iters))
         out[name] = {"median_us": ts[len(ts) // 2], "min_us": ts[0], "p95_us": ts[int(0.95 * (len(ts) - 1))]}
+    # the same three calls captured once in a CUDA graph and replayed (launch overhead paid once)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        case.step()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        case.step()
+    for _ in range(warmup):
+        graph.replay()
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+    torch.cuda._sleep(10_000_000)
+    ev[0].record()
+    for i in range(iters):
+        graph.replay()
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    ts = sorted(ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(iters))
+    out["step_graph"] = {"median_us": ts[len(ts) // 2], "min_us": ts[0], "p95_us": ts[int(0.95 * (len(ts) - 1))]}
     return out
 
 
@@ -523,6 +545,7 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
                 "combine_us": round(us["combine"]["median_us"], 2),
                 "layout+dispatch_us": round(us["layout+dispatch"]["median_us"], 2),
                 "step_us": round(us["step"]["median_us"], 2),
+                "step_cuda_graph_us": round(us["step_graph"]["median_us"], 2),
                 "dispatch_GBs": round(db / us["dispatch"]["median_us"] / 1e3, 1),
                 "combine_GBs": round(cb / us["combine"]["median_us"] / 1e3, 1),
             }
