@@ -326,16 +326,18 @@ def cta_finish_spread(case: DeviceCase):
     tr = case.ctx.trace(8192)
     out = {}
     for name, fn in (("dispatch", case.dispatch), ("combine", case.combine)):
-        vals = []
+        vals, stages = [], None
         for _ in range(5):
             tr.zero_()
             fn()
             torch.cuda.synchronize()
-            rec = tr.cpu().numpy()
-            used = rec[rec[:, 0] != 0]
-            total = float(used[:, 1].max() - used[:, 0].min())
-            vals.append(float(used[:, 1].max() - used[:, 1].min()) / total)
+            summ = case.ctx.trace_summary(tr)
+            vals.append(summ["finish_spread"])
+            stages = summ
         out[name] = round(float(np.median(vals)), 4)
+        if name == "dispatch":
+            out["dispatch_issue_thread"] = {"waiting_for_rows_in": round(stages["wait_in_share"], 3),
+                                            "waiting_for_rows_out": round(stages["wait_out_share"], 3)}
     case.ctx.trace_off()
     return out
 

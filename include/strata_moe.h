@@ -122,11 +122,13 @@ strata_status strata_ctx_launch_count(strata_ctx *ctx, uint64_t *count);
 
 /* Per-CTA stage probes (after the paper's in-kernel profiler, Sec. 6.4: probes at stage boundaries
  * writing a cycle counter into a per-core slice of a trace buffer).  dptr: device array of
- * 2*capacity_ctas uint64, owned by the caller; while set, CTA b (b < capacity_ctas) of every
- * dispatch and combine launch stores the GPU's global nanosecond timer at its start in dptr[2b] and
- * at its end in dptr[2b+1] (each launch overwrites the previous one's records).  dptr = NULL turns
- * tracing off (the default).  The spread of the end times is the load-balance evidence the paper
- * reports per core (Sec. 8.5). */
+ * 4*capacity_ctas uint64, owned by the caller; while set, CTA b (b < capacity_ctas) of every
+ * dispatch and combine launch stores in dptr[4b .. 4b+3]: the GPU's global nanosecond timer at its
+ * start, the timer at its end, the nanoseconds its issuing thread was blocked waiting for incoming
+ * rows, and the nanoseconds it was blocked waiting for outgoing rows to leave shared memory (the
+ * last two are filled by the bf16 dispatch kernel, zero elsewhere).  Each launch overwrites the
+ * previous one's records.  dptr = NULL turns tracing off (the default).  The spread of the end
+ * times is the load-balance evidence the paper reports per core (Sec. 8.5). */
 strata_status strata_ctx_set_trace(strata_ctx *ctx, uint64_t *dptr, size_t capacity_ctas);
 
 /* ---- pool: registration at allocation time ------------------------------

@@ -399,12 +399,28 @@ class MoEContext:
                                   self._stream()), "strata_moe_combine")
 
     def trace(self, capacity_ctas: int = 4096):
-        """Turns per-CTA probes on; returns the uint64 tensor [capacity, 2] = (start_ns, end_ns)."""
+        """Turns per-CTA probes on; returns the tensor [capacity, 4] = (start_ns, end_ns, wait_in_ns, wait_out_ns)."""
         import torch
-        t = torch.zeros((capacity_ctas, 2), dtype=torch.int64, device=self.device)
+        t = torch.zeros((capacity_ctas, 4), dtype=torch.int64, device=self.device)
         _check(strata_ctx_set_trace(self.h, t.data_ptr(), capacity_ctas), "strata_ctx_set_trace")
         self._trace = t
         return t
+
+    @staticmethod
+    def trace_summary(trace) -> dict:
+        """Decodes a trace tensor after a launch: kernel time, finish-time spread and stage shares."""
+        import numpy as np
+        rec = trace.cpu().numpy()
+        used = rec[rec[:, 0] != 0]
+        if used.shape[0] == 0:
+            return {"ctas": 0}
+        start, end = used[:, 0], used[:, 1]
+        total = float(end.max() - start.min())
+        busy = (end - start).astype(np.float64)
+        return {"ctas": int(used.shape[0]), "kernel_us": total / 1e3,
+                "finish_spread": float(end.max() - end.min()) / total,
+                "wait_in_share": float((used[:, 2] / busy).mean()),
+                "wait_out_share": float((used[:, 3] / busy).mean())}
 
     def trace_off(self) -> None:
         _check(strata_ctx_set_trace(self.h, None, 0), "strata_ctx_set_trace")

@@ -54,7 +54,7 @@ constexpr unsigned int kNoUnit = 0xffffffffu;
 // trace buffer): when a trace buffer is set on the context, every CTA of dispatch and combine
 // records the global timer at its start and end into its own slot.
 struct TraceBuf {
-    unsigned long long* slots;   // device, [capacity][2] = {start_ns, end_ns}; nullptr = tracing off
+    unsigned long long* slots;   // device, [capacity][4] = {start_ns, end_ns, wait_in_ns, wait_out_ns}; nullptr = off
     int capacity;
 };
 
@@ -178,12 +178,27 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
 // One thread per CTA calls these; slot = blockIdx.x.
 __device__ __forceinline__ void trace_begin(const TraceBuf& t)
 {
-    if (t.slots && (int)blockIdx.x < t.capacity) t.slots[2 * blockIdx.x] = global_timer_ns();
+    if (t.slots && (int)blockIdx.x < t.capacity) t.slots[4 * blockIdx.x] = global_timer_ns();
 }
-__device__ __forceinline__ void trace_end(const TraceBuf& t)
+// wait_in / wait_out: nanoseconds the CTA's issuing thread spent blocked on incoming data and on the
+// drain of outgoing data (0 where a kernel has no such stage)
+__device__ __forceinline__ void trace_end(const TraceBuf& t, unsigned long long wait_in = 0,
+                                          unsigned long long wait_out = 0)
 {
-    if (t.slots && (int)blockIdx.x < t.capacity) t.slots[2 * blockIdx.x + 1] = global_timer_ns();
+    if (t.slots && (int)blockIdx.x < t.capacity) {
+        t.slots[4 * blockIdx.x + 1] = global_timer_ns();
+        t.slots[4 * blockIdx.x + 2] = wait_in;
+        t.slots[4 * blockIdx.x + 3] = wait_out;
+    }
 }
+// Stage stopwatch: costs two timer reads per use, and only while a trace buffer is set.
+struct StageClock {
+    bool on;
+    unsigned long long t0, total;
+    __device__ explicit StageClock(const TraceBuf& t) : on(t.slots != nullptr), t0(0), total(0) {}
+    __device__ __forceinline__ void begin() { if (on) t0 = global_timer_ns(); }
+    __device__ __forceinline__ void end() { if (on) total += global_timer_ns() - t0; }
+};
 
 // One thread per CTA claims; returns kNoUnit when the queue is exhausted.  Units below `base` were
 // dealt statically (every CTA starts on units it knows without asking: same-address atomics complete

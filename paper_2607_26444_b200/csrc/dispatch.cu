@@ -120,6 +120,7 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
     __syncwarp();
 
     bool ok = true;
+    StageClock wait_in(p.trace), wait_out(p.trace);
     for (long long j = 0;; ++j) {
         const int s = (int)(j % kBf16Stages);
         const uint32_t parity = (uint32_t)((j / kBf16Stages) & 1);
@@ -133,7 +134,9 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
         const bool row_ok = (lane >= p.K) || (my_row >= 0 && my_row < p.capacity_rows);
         if (!row_ok && my_row != -1) report_status(p.status, STRATA_ERR_BAD_ROW);
 
+        wait_in.begin();
         ok = mbar_wait_bounded(&bars[s], parity);
+        wait_in.end();
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
 
@@ -151,15 +154,19 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
         if (lane == 0) {
             bulk_commit();
             // The stage that unit j-1 used is refilled next; its stores must have left shared memory.
+            wait_out.begin();
             bulk_wait_read<1>();
+            wait_out.end();
             issue_load(j + kBf16Stages - 1);
         }
         __syncwarp();
     }
     if (lane == 0) {
         if (!ok) report_status(p.status, STRATA_ERR_TIMEOUT);
+        wait_out.begin();
         bulk_wait_read<0>();
-        trace_end(p.trace);
+        wait_out.end();
+        trace_end(p.trace, wait_in.total, wait_out.total);
     }
 }
 

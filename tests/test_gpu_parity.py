@@ -425,6 +425,13 @@ def test_per_cta_trace_probes():
         total = used[:, 1].max() - used[:, 0].min()
         spread = (used[:, 1].max() - used[:, 1].min()) / total
         assert total > 0 and 0 <= spread < 0.5, (name, spread)
+        summ = ctx.trace_summary(tr)
+        assert summ["ctas"] == len(used) and abs(summ["finish_spread"] - spread) < 1e-9
+        if name == "dispatch":                   # the issuing thread's blocked time is part of its lifetime
+            assert np.all(used[:, 2] + used[:, 3] <= (used[:, 1] - used[:, 0]))
+            assert 0 < summ["wait_in_share"] + summ["wait_out_share"] <= 1.0
+        else:
+            assert np.all(used[:, 2] == 0) and np.all(used[:, 3] == 0)
     ctx.trace_off()
     tr.zero_()
     ctx.dispatch(lay, x_d, recv)
