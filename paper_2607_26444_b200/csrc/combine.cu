@@ -24,6 +24,9 @@ namespace {
 #ifndef STRATA_COMBINE_MAX_CTAS_PER_SM
 #define STRATA_COMBINE_MAX_CTAS_PER_SM 0     // 0: as many as fit
 #endif
+#ifndef STRATA_COMBINE_UNITS_PER_CTA
+#define STRATA_COMBINE_UNITS_PER_CTA 24      // rows are split into column parts until a CTA can expect this many units
+#endif
 constexpr int kCombineThreads = STRATA_COMBINE_THREADS;
 
 struct CombineParams {
@@ -194,7 +197,7 @@ cudaError_t launch_k(const CombineParams& p, int n_sm, cudaStream_t st)
         // vector per thread per unit)
         const int m_full = q.vec_per_part / kCombineThreads;
         int parts = 1;
-        while (parts < m_full && p.n_tok * parts < 6 * max_grid) ++parts;
+        while (parts < m_full && p.n_tok * parts < STRATA_COMBINE_UNITS_PER_CTA * max_grid) ++parts;
         q.vec_per_part = (m_full + parts - 1) / parts * kCombineThreads;
         q.parts = (p.H / 8 + q.vec_per_part - 1) / q.vec_per_part;
     }
