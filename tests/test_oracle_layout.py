@@ -242,3 +242,23 @@ def test_dispatch_and_combine_skip_unrouted_and_leave_padding():
     exact = ((rows >= 0) * w).sum(axis=1, keepdims=True) * xv
     got = wl.bf16_bits_to_f32(out).astype(np.float64)
     assert np.all(np.abs(got - exact) <= np.abs(exact) * 2.0 ** -8 + 1e-30)
+
+
+def test_ragged_ranks_are_padding_with_the_unrouted_sentinel():
+    """Ranks with different token counts: pad every rank to T tokens whose ids are all -1.  Because the
+    order is the flat (rank, token, slot) order, the rows of the real items are exactly those of the
+    compacted ragged batch."""
+    rng = np.random.default_rng(21)
+    R, T, K, E = 4, 30, 3, 8
+    tokens = [30, 7, 0, 19]                                   # per-rank token counts
+    ids = np.full((R, T, K), -1, np.int32)
+    for r, n in enumerate(tokens):
+        ids[r, :n] = rng.integers(0, E, size=(n, K))
+    lay = oracle.layout(ids, E, allow_unrouted=True)
+    compact = np.concatenate([ids[r, :n].reshape(-1, K) for r, n in enumerate(tokens)])
+    ref = oracle.layout(compact.reshape(1, -1, K), E)         # one "rank": same flat order
+    valid = ids.ravel() >= 0
+    assert np.array_equal(lay["dst_row"].ravel()[valid], ref["dst_row"].ravel())
+    assert np.array_equal(lay["expert_count"], ref["expert_count"])
+    assert np.array_equal(lay["expert_offset"], ref["expert_offset"])
+    assert lay["src_expert_count"].sum(axis=1).tolist() == [n * K for n in tokens]
