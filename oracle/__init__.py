@@ -35,7 +35,7 @@ def lib() -> ctypes.CDLL:
         L = ctypes.CDLL(build())
         i32, i64, vp = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p
         L.oracle_layout.restype = i64
-        L.oracle_layout.argtypes = [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.oracle_layout.argtypes = [i32, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.oracle_dispatch_bf16.restype = None
         L.oracle_dispatch_bf16.argtypes = [i64, i32, i32, vp, vp, vp, i32]
         L.oracle_dispatch_fp8.restype = None
@@ -73,9 +73,12 @@ class BadExpertId(ValueError):
         self.item = item
 
 
-def layout(ids: np.ndarray, E: int, segment_align: int = 1, allow_unrouted: bool = False) -> Dict[str, np.ndarray]:
+def layout(ids: np.ndarray, E: int, segment_align: int = 1, allow_unrouted: bool = False,
+           slot_capacity: int = 0) -> Dict[str, np.ndarray]:
     """Routing layout of ids int32 [R,T,K]; raises BadExpertId for an id outside [0,E) (-1 is accepted
-    as "not routed" with allow_unrouted).  segment_align > 1 pads every expert segment to that many rows."""
+    as "not routed" with allow_unrouted).  segment_align > 1 pads every expert segment to that many rows.
+    slot_capacity > 0 selects the fixed-capacity layout [E][R][capacity]; out["dropped"] counts the items
+    that did not fit."""
     ids = _c(ids, np.int32)
     R, T, K = ids.shape
     N = R * T * K
@@ -87,9 +90,10 @@ def layout(ids: np.ndarray, E: int, segment_align: int = 1, allow_unrouted: bool
         "rank_offset": np.zeros(R + 1, np.int32),
         "src_expert_count": np.zeros((R, E), np.int32),
         "dst_row": np.full((R, T, K), -1, np.int32),
-        "src_of_row": np.full(N + E * (A - 1), -1, np.int32),
+        "src_of_row": np.full(E * R * slot_capacity if slot_capacity > 0 else N + E * (A - 1), -1, np.int32),
     }
-    rc = lib().oracle_layout(R, T, K, E, A, int(bool(allow_unrouted)), _p(ids), _p(out["expert_count"]),
+    rc = lib().oracle_layout(R, T, K, E, A, int(bool(allow_unrouted)), int(slot_capacity), _p(ids),
+                             _p(out["expert_count"]),
                              _p(out["expert_offset"]), _p(out["rank_count"]), _p(out["rank_offset"]),
                              _p(out["src_expert_count"]), _p(out["dst_row"]), _p(out["src_of_row"]))
     if rc < 0:
@@ -97,6 +101,7 @@ def layout(ids: np.ndarray, E: int, segment_align: int = 1, allow_unrouted: bool
             raise ValueError("invalid shape (need R,K,E > 0 and E % R == 0)")
         raise BadExpertId(int(-rc - 1))
     out["src_of_row"] = out["src_of_row"][:int(out["expert_offset"][E])]
+    out["dropped"] = int(rc) if slot_capacity > 0 else 0
     return out
 
 

@@ -62,9 +62,74 @@
 /*  allow_unrouted: an id of -1 means "not routed": the item gets      */
 /*    dst_row = -1, is not counted, and is skipped by dispatch and     */
 /*    combine.  Without the flag -1 is rejected like any bad id.       */
+/*  slot_capacity C > 0 (fixed-capacity layout, for static shapes in   */
+/*    the low-latency mode; excludes segment_align): the receive       */
+/*    buffer is [E][R][C] rows; the j-th item (in (token, slot) order) */
+/*    that source rank r sends to expert e lands in row                */
+/*    (e*R + r)*C + j if j < C and is dropped otherwise (dst_row = -1; */
+/*    the return value is then the number of dropped items).  Counts   */
+/*    are the rows actually present: src_expert_count[r][e] =          */
+/*    min(count, C); expert_count[e] their sum over r; expert_offset[e]*/
+/*    = e*R*C; rank_offset[d] = d*(E/R)*R*C.  src_of_row has E*R*C     */
+/*    entries, -1 on empty rows.                                       */
 /* ------------------------------------------------------------------ */
+static int64_t oracle_layout_fixed(int32_t R, int32_t T, int32_t K, int32_t E, int32_t C, int32_t allow_unrouted,
+                                   const int32_t *ids, int32_t *expert_count, int32_t *expert_offset,
+                                   int32_t *rank_count, int32_t *rank_offset, int32_t *src_expert_count,
+                                   int32_t *dst_row, int32_t *src_of_row)
+{
+    const int64_t N = (int64_t)R * T * K, per_rank = (int64_t)T * K;
+    const int32_t E_loc = E / R;
+    int64_t dropped = 0;
+    int32_t *cnt = (int32_t *)calloc((size_t)R * E, sizeof(int32_t));     /* items seen per (r,e) */
+    if (!cnt) return INT64_MIN / 2;
+    if (src_of_row)
+        for (int64_t j = 0; j < (int64_t)E * R * C; ++j) src_of_row[j] = -1;
+    for (int64_t i = 0; i < N; ++i) {
+        const int32_t e = ids[i];
+        if (allow_unrouted && e == -1) {
+            dst_row[i] = -1;
+            continue;
+        }
+        if (e < 0 || e >= E) {
+            free(cnt);
+            return -(i + 1);
+        }
+        const int32_t r = (int32_t)(i / per_rank);
+        const int32_t j = cnt[r * E + e]++;
+        if (j < C) {
+            const int32_t row = (e * R + r) * C + j;
+            dst_row[i] = row;
+            if (src_of_row) src_of_row[row] = (int32_t)i;
+        } else {
+            dst_row[i] = -1;
+            ++dropped;
+        }
+    }
+    for (int32_t e = 0; e < E; ++e) {
+        int32_t sum = 0;
+        for (int32_t r = 0; r < R; ++r) {
+            const int32_t kept = cnt[r * E + e] < C ? cnt[r * E + e] : C;
+            if (src_expert_count) src_expert_count[r * E + e] = kept;
+            sum += kept;
+        }
+        expert_count[e] = sum;
+        expert_offset[e] = e * R * C;
+    }
+    expert_offset[E] = E * R * C;
+    for (int32_t d = 0; d < R; ++d) {
+        int32_t sum = 0;
+        for (int32_t e = d * E_loc; e < (d + 1) * E_loc; ++e) sum += expert_count[e];
+        rank_count[d] = sum;
+        rank_offset[d] = expert_offset[d * E_loc];
+    }
+    rank_offset[R] = expert_offset[E];
+    free(cnt);
+    return dropped;
+}
+
 int64_t oracle_layout(int32_t R, int32_t T, int32_t K, int32_t E,
-                      int32_t segment_align, int32_t allow_unrouted,
+                      int32_t segment_align, int32_t allow_unrouted, int32_t slot_capacity,
                       const int32_t *ids,           /* [R,T,K] */
                       int32_t *expert_count,        /* [E]     */
                       int32_t *expert_offset,       /* [E+1]   */
@@ -75,6 +140,11 @@ int64_t oracle_layout(int32_t R, int32_t T, int32_t K, int32_t E,
                       int32_t *src_of_row)          /* [offset[E]] or NULL */
 {
     if (R <= 0 || T < 0 || K <= 0 || E <= 0 || E % R != 0) return INT64_MIN / 2;
+    if (slot_capacity > 0) {
+        if (segment_align > 1) return INT64_MIN / 2;
+        return oracle_layout_fixed(R, T, K, E, slot_capacity, allow_unrouted, ids, expert_count, expert_offset,
+                                   rank_count, rank_offset, src_expert_count, dst_row, src_of_row);
+    }
     const int64_t N = (int64_t)R * T * K;
     const int64_t per_rank = (int64_t)T * K;
     const int32_t E_loc = E / R;

@@ -262,3 +262,56 @@ def test_ragged_ranks_are_padding_with_the_unrouted_sentinel():
     assert np.array_equal(lay["expert_count"], ref["expert_count"])
     assert np.array_equal(lay["expert_offset"], ref["expert_offset"])
     assert lay["src_expert_count"].sum(axis=1).tolist() == [n * K for n in tokens]
+
+
+# ---- fixed-capacity layout -----------------------------------------------------------------------
+
+def test_worked_example_fixed_capacity():
+    rows = {}
+    with open(os.path.join(GOLDEN, "layout_fixed_capacity_example.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].split()
+            if line:
+                rows[line[0]] = np.array(line[1:], dtype=np.int64)
+    R, T, K, E = rows["shape"]
+    lay = oracle.layout(rows["ids"].astype(np.int32).reshape(R, T, K), int(E), slot_capacity=int(rows["capacity"][0]))
+    for key in ("expert_count", "expert_offset", "rank_count", "rank_offset", "src_expert_count", "dst_row",
+                "src_of_row"):
+        assert np.array_equal(lay[key].ravel(), rows[key]), key
+    assert lay["dropped"] == rows["dropped"][0]
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_fixed_capacity_matches_brute_force(seed):
+    rng = np.random.default_rng(300 + seed)
+    R = int(rng.choice([1, 2, 4]))
+    E = R * int(rng.integers(1, 4))
+    T, K, C = int(rng.integers(1, 30)), int(rng.integers(1, 4)), int(rng.integers(1, 9))
+    ids = rng.integers(-1, E, size=(R, T, K)).astype(np.int32)
+    lay = oracle.layout(ids, E, allow_unrouted=True, slot_capacity=C)
+    # independent formulation: group the routed items by (expert, rank) with a comparison sort
+    tuples = sorted((int(ids[r, t, k]), r, t, k) for r in range(R) for t in range(T) for k in range(K) if ids[r, t, k] >= 0)
+    dst = np.full((R, T, K), -1, np.int32)
+    seen, dropped = {}, 0
+    for e, r, t, k in tuples:
+        j = seen.get((e, r), 0)
+        seen[(e, r)] = j + 1
+        if j < C:
+            dst[r, t, k] = (e * R + r) * C + j
+        else:
+            dropped += 1
+    assert np.array_equal(lay["dst_row"], dst) and lay["dropped"] == dropped
+    kept = np.array([[min(seen.get((e, r), 0), C) for e in range(E)] for r in range(R)])
+    assert np.array_equal(lay["src_expert_count"], kept)
+    assert np.array_equal(lay["expert_count"], kept.sum(axis=0))
+    assert np.array_equal(lay["expert_offset"], np.arange(E + 1) * R * C)
+    assert lay["rank_offset"][R] == E * R * C
+    src = lay["src_of_row"]
+    assert src.size == E * R * C and (src >= 0).sum() == (dst >= 0).sum()
+    assert np.array_equal(lay["dst_row"].ravel()[src[src >= 0]], np.flatnonzero(src >= 0))
+    # a capacity nobody reaches: same slots, nothing dropped, counts are the plain counts
+    big = oracle.layout(ids, E, allow_unrouted=True, slot_capacity=T * K + 1)
+    assert big["dropped"] == 0
+    assert np.array_equal(big["expert_count"], oracle.layout(ids, E, allow_unrouted=True)["expert_count"])
+    with pytest.raises(ValueError):
+        oracle.layout(ids, E, allow_unrouted=True, slot_capacity=C, segment_align=4)
