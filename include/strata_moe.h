@@ -68,13 +68,21 @@ typedef enum {
  *    src_of_row is -1 there.  rank_offset follows the padded offsets, rank_count and expert_count
  *    stay the numbers of real rows.  The receive buffer needs strata_moe_recv_rows() rows.
  *  STRATA_FLAG_ALLOW_UNROUTED: an id of -1 means "not routed" (dropped token slot): dst_row = -1,
- *    counted nowhere, skipped by dispatch, contributes nothing in combine, and is not an error. */
+ *    counted nowhere, skipped by dispatch, contributes nothing in combine, and is not an error.
+ *  slot_capacity C > 0: fixed-capacity layout, a receive buffer of static shape [E][R][C] rows for the
+ *    low-latency mode (pairs with CUDA-graph replay; excludes segment_align).  The j-th item, in
+ *    (token, slot) order, that source rank r sends to expert e lands in row (e*R + r)*C + j if j < C;
+ *    otherwise it is dropped (dst_row = -1) and STRATA_ERR_CAPACITY is raised on the device status.
+ *    Counts are the rows present: src_expert_count[r][e] = min(count, C), expert_count[e] their sum,
+ *    expert_offset[e] = e*R*C, rank_offset[d] = d*(E/R)*R*C; src_of_row is -1 on empty rows.  The
+ *    window-partitioning calls do not support this layout. */
 #define STRATA_FLAG_ALLOW_UNROUTED 1
 typedef struct {
     int32_t R, T, H, E, K;
     int32_t dispatch_dtype;        /* a strata_dtype */
     int32_t segment_align;         /* rows; 0 or 1 = packed segments; at most 65536 */
     int32_t flags;                 /* STRATA_FLAG_* */
+    int32_t slot_capacity;         /* rows per (expert, source rank) slot; 0 = packed/aligned segments */
 } strata_moe_shape;
 
 typedef struct strata_ctx strata_ctx;   /* opaque, host side */
@@ -113,7 +121,8 @@ strata_status strata_ctx_destroy(strata_ctx *ctx);
  * valid and unshared while calls on this context are in flight. */
 strata_status strata_moe_workspace_bytes(const strata_moe_shape *shape, size_t *bytes);
 /* Rows the receive buffer (and src_of_row) must hold: R*T*K + E*(segment_align-1), the worst case of
- * the padded layout (R*T*K for packed segments).  Host arithmetic only. */
+ * the padded layout (R*T*K for packed segments), or E*R*slot_capacity for the fixed-capacity layout.
+ * Host arithmetic only. */
 strata_status strata_moe_recv_rows(const strata_moe_shape *shape, size_t *rows);
 strata_status strata_ctx_set_workspace(strata_ctx *ctx, void *dptr, size_t bytes);
 

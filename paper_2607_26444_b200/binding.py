@@ -45,7 +45,7 @@ EXPORTS = [
 class strata_moe_shape(ctypes.Structure):
     _fields_ = [("R", ctypes.c_int32), ("T", ctypes.c_int32), ("H", ctypes.c_int32),
                 ("E", ctypes.c_int32), ("K", ctypes.c_int32), ("dispatch_dtype", ctypes.c_int32),
-                ("segment_align", ctypes.c_int32), ("flags", ctypes.c_int32)]
+                ("segment_align", ctypes.c_int32), ("flags", ctypes.c_int32), ("slot_capacity", ctypes.c_int32)]
 
 
 class strata_moe_layout_t(ctypes.Structure):
@@ -319,12 +319,13 @@ class MoEContext:
     """One shape on one GPU.  Owns a strata_ctx and its workspace tensor."""
 
     def __init__(self, R: int, T: int, H: int, E: int, K: int, dispatch_dtype: int = STRATA_BF16,
-                 device: int = 0, segment_align: int = 0, allow_unrouted: bool = False):
+                 device: int = 0, segment_align: int = 0, allow_unrouted: bool = False,
+                 slot_capacity: int = 0):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("MoEContext needs a CUDA device (there is no CPU fallback)")
         self.shape = strata_moe_shape(R, T, H, E, K, dispatch_dtype, segment_align,
-                                      STRATA_FLAG_ALLOW_UNROUTED if allow_unrouted else 0)
+                                      STRATA_FLAG_ALLOW_UNROUTED if allow_unrouted else 0, slot_capacity)
         self.R, self.T, self.H, self.E, self.K = R, T, H, E, K
         self.fp8 = dispatch_dtype == STRATA_FP8_E4M3_B128
         self.n_tok, self.n_items = R * T, R * T * K

@@ -44,6 +44,7 @@ using namespace strata;
 // rows of the receive buffer: all items plus the worst-case padding of aligned segments
 long long recv_rows(const strata_moe_shape& s)
 {
+    if (s.slot_capacity > 0) return (long long)s.E * s.R * s.slot_capacity;
     const long long pad = s.segment_align > 1 ? s.segment_align - 1 : 0;
     return (long long)s.R * s.T * s.K + (long long)s.E * pad;
 }
@@ -58,6 +59,7 @@ strata_status check_shape(const strata_moe_shape* s)
     if (s->dispatch_dtype == STRATA_FP8_E4M3_B128 && s->H % 128 != 0) return STRATA_ERR_SHAPE;
     if (s->segment_align < 0 || s->segment_align > 65536) return STRATA_ERR_SHAPE;
     if ((s->flags & ~STRATA_FLAG_ALLOW_UNROUTED) != 0) return STRATA_ERR_SHAPE;
+    if (s->slot_capacity < 0 || (s->slot_capacity > 0 && s->segment_align > 1)) return STRATA_ERR_SHAPE;
     if (recv_rows(*s) >= (1ll << 31)) return STRATA_ERR_SHAPE;
     return STRATA_OK;
 }
@@ -426,6 +428,7 @@ strata_status strata_moe_partition(strata_ctx* ctx, const strata_moe_layout_t* l
         return STRATA_ERR_INVALID_ARG;
     strata_status st = check_policy(ctx->shape, policy);
     if (st != STRATA_OK) return st;
+    if (ctx->shape.slot_capacity > 0) return STRATA_ERR_SHAPE;      // windows assume packed/aligned segments
     if (n_cores < 1 || n_cores > partition_max_cores_supported()) return STRATA_ERR_SHAPE;
     if (max_units < 1 || max_units > (size_t)1 << 20) return STRATA_ERR_CAPACITY;
     if (!ctx->ws) return STRATA_ERR_WORKSPACE;
@@ -450,7 +453,8 @@ strata_status strata_moe_dispatch_windows(strata_ctx* ctx, const strata_moe_layo
     if (!partition->win_base || !partition->unit_desc || !partition->task_offset || !partition->task_unit)
         return STRATA_ERR_INVALID_ARG;
     const strata_moe_shape& s = ctx->shape;
-    if (s.dispatch_dtype != STRATA_BF16 || (uint32_t)s.H * 2u > windows_max_row_bytes()) return STRATA_ERR_SHAPE;
+    if (s.dispatch_dtype != STRATA_BF16 || (uint32_t)s.H * 2u > windows_max_row_bytes() || s.slot_capacity > 0)
+        return STRATA_ERR_SHAPE;
     if (n_cores < 1 || n_cores > partition_max_cores_supported()) return STRATA_ERR_SHAPE;
     if (!aligned16(x) || !aligned16(recv)) return STRATA_ERR_ALIGNMENT;
     if (!ctx->ws) return STRATA_ERR_WORKSPACE;

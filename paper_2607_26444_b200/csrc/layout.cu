@@ -38,6 +38,7 @@ struct LayoutParams {
     int items_per_rank, tiles_per_rank, n_tiles;
     int align;            // >= 1: rows every expert segment is padded to
     int allow_unrouted;   // id -1 is legal and means "not routed"
+    int capacity;         // > 0: fixed-capacity layout [E][R][capacity]
 };
 
 __device__ __forceinline__ int round_up_rows(int n, int a) { return (n + a - 1) / a * a; }
@@ -238,7 +239,41 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_count_scan_kernel(Layou
                 }
         }
     }
-    if (p.src_expert_count) {
+    if (p.capacity > 0) {
+        // Fixed-capacity layout: rows are [E][R][capacity]; counts are clamped to the capacity, the
+        // offsets are constants, and every row starts empty.
+        __syncthreads();                  // the prefixes written above, by this CTA, are read below
+        const int C = p.capacity;
+        if (tid < E) {
+            int kept_sum = 0;
+            bool over = false;
+            for (int rr = 0; rr < p.R; ++rr) {
+                const int lo = p.tile_cnt[(size_t)(rr * p.tiles_per_rank) * E + tid];
+                const int hi = (rr + 1 < p.R) ? p.tile_cnt[(size_t)((rr + 1) * p.tiles_per_rank) * E + tid] : count_e;
+                const int kept = min(hi - lo, C);
+                over |= hi - lo > C;
+                if (p.src_expert_count) p.src_expert_count[(size_t)rr * E + tid] = kept;
+                kept_sum += kept;
+            }
+            if (over) report_status(p.status, STRATA_ERR_CAPACITY);
+            p.expert_count[tid] = kept_sum;
+            p.expert_offset[tid] = tid * p.R * C;
+            offs[tid] = kept_sum;         // reused below for the per-rank sums
+        }
+        if (tid == 0) {
+            p.expert_offset[E] = E * p.R * C;
+            p.rank_offset[p.R] = E * p.R * C;
+        }
+        __syncthreads();
+        for (int d = tid; d < p.R; d += kLayoutThreads) {
+            int real = 0;
+            for (int e2 = d * p.e_loc; e2 < (d + 1) * p.e_loc; ++e2) real += offs[e2];
+            p.rank_count[d] = real;
+            p.rank_offset[d] = d * p.e_loc * p.R * C;
+        }
+        if (p.src_of_row)
+            for (long long x = tid; x < (long long)E * p.R * C; x += kLayoutThreads) p.src_of_row[x] = -1;
+    } else if (p.src_expert_count) {
         __syncthreads();                  // the prefixes written above, by this CTA, are read below
         for (int x = tid; x < p.R * E; x += kLayoutThreads) {
             const int rr = x / E, e2 = x - rr * E;
@@ -315,9 +350,16 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_rank_kernel(LayoutParam
         const long long item = rank_base + in_rank;
         const int e = ids[q];
         if ((unsigned)e < (unsigned)E) {
-            const int row = p.expert_offset[e] + p.tile_cnt[(size_t)tile * E + e] + mine[e] + in_warp[q];
+            int row;
+            if (p.capacity > 0) {         // index inside the (expert, source rank) slot; dropped beyond the capacity
+                const int idx = p.tile_cnt[(size_t)tile * E + e] - p.tile_cnt[(size_t)(r * p.tiles_per_rank) * E + e] +
+                                mine[e] + in_warp[q];
+                row = idx < p.capacity ? (e * p.R + r) * p.capacity + idx : -1;
+            } else {
+                row = p.expert_offset[e] + p.tile_cnt[(size_t)tile * E + e] + mine[e] + in_warp[q];
+            }
             p.dst_row[item] = row;
-            if (p.src_of_row) p.src_of_row[row] = (int32_t)item;
+            if (p.src_of_row && row >= 0) p.src_of_row[row] = (int32_t)item;
         } else {
             p.dst_row[item] = -1;
         }
@@ -551,10 +593,12 @@ cudaError_t launch_layout(const strata_moe_shape& s, const int32_t* ids, const s
     p.n_tiles = g.n_tiles;
     p.align = s.segment_align > 1 ? s.segment_align : 1;
     p.allow_unrouted = (s.flags & STRATA_FLAG_ALLOW_UNROUTED) ? 1 : 0;
+    p.capacity = s.slot_capacity > 0 ? s.slot_capacity : 0;
 
     const long long n_items = (long long)s.R * s.T * s.K;
     const size_t small_bytes = small_smem(s.E, s.R, L.src_expert_count != nullptr);
-    if (n_items <= (long long)kSmallItems * kLayoutCluster && small_bytes <= kSmallSmemLimit) {
+    // the fixed-capacity layout needs per-source-rank prefixes, which only the tiled path keeps
+    if (p.capacity == 0 && n_items <= (long long)kSmallItems * kLayoutCluster && small_bytes <= kSmallSmemLimit) {
         const unsigned n_cta = n_items <= kSmallItems ? 1u : (unsigned)kLayoutCluster;
         *n_launches = 1;
         return launch_pdl_cluster(layout_cluster_kernel, n_cta, kLayoutThreads, small_bytes, n_cta, st, p,
@@ -636,6 +680,8 @@ extern "C" strata_status strata_moe_layout_noalloc(const strata_moe_shape* shape
     if (s.R <= 0 || s.T <= 0 || s.E <= 0 || s.K <= 0) return STRATA_ERR_SHAPE;
     if (s.E % s.R != 0 || s.E > kMaxExperts || s.K > kMaxTopK) return STRATA_ERR_SHAPE;
     if (s.segment_align < 0 || s.segment_align > 65536) return STRATA_ERR_SHAPE;
+    if (s.slot_capacity < 0 || (s.slot_capacity > 0 && s.segment_align > 1)) return STRATA_ERR_SHAPE;
+    if ((long long)s.E * s.R * s.slot_capacity >= (1ll << 31)) return STRATA_ERR_SHAPE;
     if ((long long)s.R * s.T * s.K + (long long)s.E * (s.segment_align > 1 ? s.segment_align - 1 : 0) >= (1ll << 31))
         return STRATA_ERR_SHAPE;
     const LayoutGeom g = layout_geom(s);
@@ -671,6 +717,7 @@ extern "C" strata_status strata_moe_layout_noalloc(const strata_moe_shape* shape
     p.n_tiles = g.n_tiles;
     p.align = s.segment_align > 1 ? s.segment_align : 1;
     p.allow_unrouted = (s.flags & STRATA_FLAG_ALLOW_UNROUTED) ? 1 : 0;
+    p.capacity = s.slot_capacity > 0 ? s.slot_capacity : 0;
     layout_count_scan_kernel<<<g.n_tiles, kLayoutThreads, count_scan_smem(s.E), st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return STRATA_ERR_CUDA;
     layout_rank_kernel<<<g.n_tiles, kLayoutThreads, (size_t)32 * s.E * sizeof(int), st>>>(p);

@@ -574,3 +574,46 @@ def test_cuda_graph_replay(kw):
         assert np.array_equal(u16(out), oracle.combine(ref["dst_row"], ref_recv, inp["w"], nthreads=4)), rep
     assert ctx.device_status() == B.STRATA_OK
     ctx.close()
+
+
+@pytest.mark.parametrize("kw,cap,frac", [
+    (dict(R=4, T=128, H=1024, E=16, K=2), 24, 0.0),               # some slots overflow
+    (dict(R=16, T=128, H=7168, E=256, K=8), 16, 0.0),             # decode shape, static [256][16][16] buffer
+    (dict(R=8, T=1500, H=128, E=32, K=4), 200, 0.2),              # several tiles per rank, unrouted slots
+    (dict(R=2, T=60, H=64, E=4, K=3), 1000, 0.0),                 # capacity nobody reaches
+], ids=lambda v: str(v) if not isinstance(v, dict) else "R{R}T{T}H{H}E{E}K{K}".format(**v))
+def test_fixed_capacity_layout(kw, cap, frac):
+    cfg = wl.shrink(wl.CONFIGS["tiny"], seed=555, **kw)
+    inp = wl.generate(cfg)
+    ids = inp["ids"].copy()
+    if frac:
+        ids[np.random.default_rng(2).random(ids.shape) < frac] = -1
+    ref = oracle.layout(ids, cfg.E, allow_unrouted=True, slot_capacity=cap)
+    ctx = B.MoEContext(cfg.R, cfg.T, cfg.H, cfg.E, cfg.K, allow_unrouted=True, slot_capacity=cap)
+    n_rows = ctx.recv_rows
+    assert n_rows == cfg.E * cfg.R * cap
+    lay = ctx.layout(to_dev(ids))
+    torch.cuda.synchronize()
+    assert ctx.device_status() == (B.STRATA_ERR_CAPACITY if ref["dropped"] else B.STRATA_OK)
+    for key in ("expert_count", "expert_offset", "rank_count", "rank_offset", "src_expert_count", "dst_row",
+                "src_of_row"):
+        assert np.array_equal(getattr(lay, key).cpu().numpy(), ref[key]), key
+    whole, recv = guarded(n_rows, cfg.H, torch.int16, SENTINEL16)
+    ctx.register(whole)
+    ctx.dispatch(lay, to_dev(inp["x"]), recv)
+    want = oracle.dispatch_bf16(ref["dst_row"], inp["x"], nthreads=4, n_rows=n_rows)
+    got = u16(recv)
+    used = ref["src_of_row"] >= 0
+    assert np.array_equal(got[used], want[used]) and np.all(got[~used] == SENTINEL16)
+    out = torch.empty((cfg.n_tok, cfg.H), dtype=torch.int16, device=DEV)
+    ctx.combine(lay, recv, to_dev(inp["w"]), out)
+    assert np.array_equal(u16(out), oracle.combine(ref["dst_row"], want, inp["w"], nthreads=4))
+    assert ctx.device_status() == B.STRATA_OK                    # dropped items are -1 rows: skipped silently
+    hw = u16(whole)
+    assert np.all(hw[:GUARD] == SENTINEL16) and np.all(hw[GUARD + n_rows:] == SENTINEL16)
+    # the window-partitioning variant declines this layout
+    pol = B.make_policy([(10, 64, 16, 2)])
+    part = B.Partition(cfg.R, cfg.E, 8, 64, ctx.device)
+    assert B.strata_moe_partition(ctx.h, lay.c, pol, 8, part.c, 64, torch.cuda.current_stream().cuda_stream) \
+        == B.STRATA_ERR_SHAPE
+    ctx.close()
