@@ -227,8 +227,11 @@ cudaError_t launch_combine(const strata_moe_shape& s, const int32_t* dst_row, co
     switch (s.K) {
         case 1: return launch_k<1>(p, n_sm, st);
         case 2: return launch_k<2>(p, n_sm, st);
+        case 3: return launch_k<3>(p, n_sm, st);
         case 4: return launch_k<4>(p, n_sm, st);
+        case 5: return launch_k<5>(p, n_sm, st);
         case 6: return launch_k<6>(p, n_sm, st);
+        case 7: return launch_k<7>(p, n_sm, st);
         case 8: return launch_k<8>(p, n_sm, st);
         default: return launch_k<0>(p, n_sm, st);
     }
