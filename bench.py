@@ -550,6 +550,8 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
                 "step_cuda_graph_us": round(us["step_graph"]["median_us"], 2),
                 "dispatch_GBs": round(db / us["dispatch"]["median_us"] / 1e3, 1),
                 "combine_GBs": round(cb / us["combine"]["median_us"] / 1e3, 1),
+                "min_p95_us": {k: [round(v["min_us"], 2), round(v["p95_us"], 2)] for k, v in us.items()},
+                "iters": 30,
             }
             if name == "skew":
                 # load balance under Zipf routing: per-CTA finish-time spread, and the same shape with
