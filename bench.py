@@ -265,9 +265,23 @@ class DeviceCase:
         self.combine()
 
     def check(self):
+        """Device status clean, and (bf16, identity experts) the timed buffers hold the right answer:
+        every receive row equals its source row, and combine returned x (gate weights sum to 1)."""
+        torch = self.torch
         st = self.ctx.device_status()
         if st != 0:
             raise RuntimeError(f"device status {st}: {self.B.strata_status_string(st)}")
+        if self.y is self.recv:
+            cfg = self.cfg
+            x2 = self.x.view(cfg.n_tok, cfg.H)
+            if not bool((self.out.view(torch.bfloat16) == x2.view(torch.bfloat16)).all()):
+                raise RuntimeError("combine output differs from x")
+            dst = self.lay.dst_row.view(cfg.n_tok, cfg.K)
+            sample = torch.arange(0, cfg.n_tok, max(1, cfg.n_tok // 4096), device=self.dev)
+            for k in range(cfg.K):
+                if not torch.equal(self.recv[dst[sample, k].long()], x2[sample]):
+                    raise RuntimeError("a receive row differs from its source row")
+        return True
 
 
 def per_call_us(case: DeviceCase, iters: int = 30, warmup: int = 3):
@@ -596,6 +610,7 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
                    "bytes_per_step": step_bytes, "l2": "inputs larger than L2 (8.4 GB working set), no flush",
                    "parallelism": "replicas only" if world > 1 else "1 GPU, 16 ranks emulated in HBM"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(n1 - n0), "roofline": roofline,
+        "verified": "after the timed steps: device status clean, out == x, sampled receive rows == source rows",
         "pct_of_8TBs": {"dispatch": round(100 * kernels[disp_name]["frac_of_nominal_8TBs"], 2),
                         "combine": round(100 * kernels["combine_kernel"]["frac_of_nominal_8TBs"], 2)},
         "other_configs": other, "cpu_baseline": cpu,
