@@ -166,7 +166,8 @@ strata_status strata_pool_reset(strata_ctx *ctx, uint64_t region_id);
  * Duplicate ids inside a token are legal.  An id outside [0,E) is skipped
  * (dst_row = -1, not counted) and raises BAD_EXPERT_ID on the device status
  * (except -1 under STRATA_FLAG_ALLOW_UNROUTED, which is legal).
- * Needs a workspace.  One kernel launch for up to 32,768 items, two beyond. */
+ * Needs a workspace.  One kernel launch for up to 32,768 items, two beyond
+ * (and always two for the fixed-capacity layout). */
 strata_status strata_moe_layout(strata_ctx *ctx, const int32_t *topk_ids,
                                 const strata_moe_layout_t *layout, void *stream);
 
