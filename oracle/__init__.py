@@ -48,6 +48,11 @@ def lib() -> ctypes.CDLL:
         L.oracle_partition.argtypes = [i32, i32, i64, i32, vp, vp, vp, i32, i32, i32, i64, vp, vp, vp, vp, vp, vp]
         L.oracle_dispatch_windows.restype = None
         L.oracle_dispatch_windows.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        for name in ("oracle_allgather", "oracle_alltoall", "oracle_reducescatter", "oracle_allreduce"):
+            getattr(L, name).restype = None
+            getattr(L, name).argtypes = [i32, i64, vp, vp]
+        L.oracle_broadcast.restype = None
+        L.oracle_broadcast.argtypes = [i32, i32, i64, vp, vp]
         L.oracle_max_threads.restype = i32
         L.oracle_max_threads.argtypes = []
         _lib = L
@@ -210,3 +215,53 @@ def dispatch_windows(lay: Dict[str, np.ndarray], part: Dict[str, np.ndarray], x:
                                   _p(_c(part["task_unit"], np.int32)), _p(_c(lay["src_of_row"], np.int32)),
                                   _p(x2), _p(recv))
     return recv
+
+
+# ---- full-mesh collectives over emulated ranks (paper Sec. 6.1) ----------------------------------
+
+def allgather(x: np.ndarray) -> np.ndarray:
+    """x uint8 [R, M] -> out uint8 [R, R, M], out[r, p] = x[p]."""
+    x = _c(x, np.uint8)
+    R, M = x.shape
+    out = np.empty((R, R, M), np.uint8)
+    lib().oracle_allgather(R, M, _p(x), _p(out))
+    return out
+
+
+def alltoall(x: np.ndarray) -> np.ndarray:
+    """x uint8 [R, R, S] -> out uint8 [R, R, S], out[r, p] = x[p, r]."""
+    x = _c(x, np.uint8)
+    R, R2, S = x.shape
+    assert R == R2
+    out = np.empty((R, R, S), np.uint8)
+    lib().oracle_alltoall(R, S, _p(x), _p(out))
+    return out
+
+
+def broadcast(x: np.ndarray, root: int) -> np.ndarray:
+    """x uint8 [R, M] -> out uint8 [R, M], out[r] = x[root]."""
+    x = _c(x, np.uint8)
+    R, M = x.shape
+    assert 0 <= root < R
+    out = np.empty((R, M), np.uint8)
+    lib().oracle_broadcast(R, root, M, _p(x), _p(out))
+    return out
+
+
+def reducescatter(x: np.ndarray) -> np.ndarray:
+    """x bf16 bits uint16 [R, R, S] -> out uint16 [R, S], out[r] = sum over p (rank order, fp32) of x[p, r]."""
+    x = _c(x, np.uint16)
+    R, R2, S = x.shape
+    assert R == R2
+    out = np.empty((R, S), np.uint16)
+    lib().oracle_reducescatter(R, S, _p(x), _p(out))
+    return out
+
+
+def allreduce(x: np.ndarray) -> np.ndarray:
+    """x bf16 bits uint16 [R, M] -> out uint16 [R, M], out[r] = sum over p (rank order, fp32) of x[p]."""
+    x = _c(x, np.uint16)
+    R, M = x.shape
+    out = np.empty((R, M), np.uint16)
+    lib().oracle_allreduce(R, M, _p(x), _p(out))
+    return out

@@ -17,6 +17,8 @@
  *    into the user buffer (no staging copy).
  *  - Combine (paper Sec. 6.1, reduction-bearing operators): the top-k expert
  *    outputs of a token are accumulated into the token's local destination.
+ *  - Full-mesh collectives over emulated ranks (paper Sec. 6.1): pull-mode
+ *    data movement and rank-ordered accumulation.
  * The paper prints no pseudo-code, layout, dtype or worked example for this
  * path; the concrete conventions below (segment order expert -> source rank ->
  * token -> slot, packed segments, contiguous expert->rank blocks, fp32 FMA in
@@ -30,6 +32,10 @@
  * for the partitioning: exact cover of the receive rows, Graham's tight LPT
  * example, the 4/3 - 1/(3C) bound against a brute-force optimum, the fan-out
  * cap, and equality of window-major with token-major dispatch.
+ * For the full-mesh collectives (tests/test_oracle_collectives.py): counter
+ * patterns with closed-form results, the involution of all-to-all, exact
+ * integer sums, a hand-worked order-sensitive sum, all-reduce = reduce-scatter
+ * followed by all-gather, and an fp64 bound.
  * No function here is "parity unpinned".
  *
  * Index convention: rank r in [0,R), token t in [0,T), slot k in [0,K),
@@ -527,6 +533,67 @@ void oracle_dispatch_windows(int32_t R, int32_t E, int32_t K, int32_t H, int32_t
                 rows -= take;
                 first = 0;
             }
+        }
+}
+
+/* ------------------------------------------------------------------ */
+/* O6: full-mesh collectives over R emulated ranks (paper Sec. 6.1).    */
+/* Every rank's buffer is one partition of a slab: rank r's input is    */
+/* in[r], its output out[r].  Data-movement operators follow the pull   */
+/* mode: rank r reads the peers' slices and writes them into its own    */
+/* output.  Reduction-bearing operators accumulate the peers' operands  */
+/* into the local destination; this build's reading of the arithmetic   */
+/* (the paper names none): bf16 operands, one binary32 addition per     */
+/* peer in rank order 0..R-1 starting from +0, one rounding to bf16     */
+/* (RNE) at the end.                                                    */
+/*   all-gather      in [R][M] bytes      out[r][p][j] = in[p][j]       */
+/*   all-to-all      in [R][R][S] bytes   out[r][p][j] = in[p][r][j]    */
+/*   broadcast       in [R][M] bytes      out[r][j]    = in[root][j]    */
+/*   reduce-scatter  in [R][R][S] bf16    out[r][j] = sum_p in[p][r][j] */
+/*   all-reduce      in [R][M] bf16       out[r][j] = sum_p in[p][j]    */
+/* ------------------------------------------------------------------ */
+void oracle_allgather(int32_t R, int64_t M, const uint8_t *in, uint8_t *out)
+{
+    for (int32_t r = 0; r < R; ++r)
+        for (int32_t p = 0; p < R; ++p)
+            for (int64_t j = 0; j < M; ++j)
+                out[((size_t)r * R + p) * M + j] = in[(size_t)p * M + j];
+}
+
+void oracle_alltoall(int32_t R, int64_t S, const uint8_t *in, uint8_t *out)
+{
+    for (int32_t r = 0; r < R; ++r)
+        for (int32_t p = 0; p < R; ++p)
+            for (int64_t j = 0; j < S; ++j)
+                out[((size_t)r * R + p) * S + j] = in[((size_t)p * R + r) * S + j];
+}
+
+void oracle_broadcast(int32_t R, int32_t root, int64_t M, const uint8_t *in, uint8_t *out)
+{
+    for (int32_t r = 0; r < R; ++r)
+        for (int64_t j = 0; j < M; ++j)
+            out[(size_t)r * M + j] = in[(size_t)root * M + j];
+}
+
+void oracle_reducescatter(int32_t R, int64_t S, const uint16_t *in, uint16_t *out)
+{
+    for (int32_t r = 0; r < R; ++r)
+        for (int64_t j = 0; j < S; ++j) {
+            float acc = 0.0f;
+            for (int32_t p = 0; p < R; ++p)
+                acc = acc + bf16_to_f32(in[((size_t)p * R + r) * S + j]);
+            out[(size_t)r * S + j] = f32_to_bf16_rne(acc);
+        }
+}
+
+void oracle_allreduce(int32_t R, int64_t M, const uint16_t *in, uint16_t *out)
+{
+    for (int32_t r = 0; r < R; ++r)
+        for (int64_t j = 0; j < M; ++j) {
+            float acc = 0.0f;
+            for (int32_t p = 0; p < R; ++p)
+                acc = acc + bf16_to_f32(in[(size_t)p * M + j]);
+            out[(size_t)r * M + j] = f32_to_bf16_rne(acc);
         }
 }
 

@@ -178,6 +178,18 @@ def gen_gate_weights(cfg: MoEConfig) -> np.ndarray:
     return np.ascontiguousarray(p.reshape(cfg.R, cfg.T, cfg.K), dtype=np.float32)
 
 
+def gen_payload(R: int, elems_per_rank: int, seed: int) -> np.ndarray:
+    """uint16 [R, elems_per_rank]: every emulated rank's collective payload, bf16 bits of N(0, 1).
+
+    The data-movement collectives treat the same array as raw bytes.
+    """
+    rng = _rng(seed, 7)
+    out = np.empty((R, elems_per_rank), dtype=np.uint16)
+    for r in range(R):
+        out[r] = f32_to_bf16_bits(rng.standard_normal(elems_per_rank, dtype=np.float32))
+    return out
+
+
 def generate(cfg: MoEConfig) -> Dict[str, np.ndarray]:
     return {"ids": gen_topk_ids(cfg), "x": gen_x(cfg), "w": gen_gate_weights(cfg)}
 
