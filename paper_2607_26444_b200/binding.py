@@ -39,6 +39,7 @@ EXPORTS = [
     "strata_moe_roundtrip_host", "strata_moe_layout_noalloc", "strata_ctx_set_trace",
     "strata_moe_partition_max_units", "strata_moe_partition", "strata_moe_dispatch_windows",
     "strata_moe_recv_rows",
+    "strata_allgather", "strata_alltoall", "strata_broadcast", "strata_reducescatter", "strata_allreduce",
 ]
 
 
@@ -131,6 +132,11 @@ def lib() -> ctypes.CDLL:
         "strata_moe_partition": [vp, P(strata_moe_layout_t), P(strata_partition_policy), i32,
                                  P(strata_partition_t), sz, vp],
         "strata_moe_dispatch_windows": [vp, P(strata_moe_layout_t), P(strata_partition_t), i32, vp, vp, sz, vp],
+        "strata_allgather": [vp, i32, vp, vp, sz, vp],
+        "strata_alltoall": [vp, i32, vp, vp, sz, vp],
+        "strata_broadcast": [vp, i32, i32, vp, vp, sz, vp],
+        "strata_reducescatter": [vp, i32, vp, vp, sz, vp],
+        "strata_allreduce": [vp, i32, vp, vp, sz, vp],
     }
     for name, args in sigs.items():
         fn = getattr(L, name)
@@ -263,6 +269,26 @@ def strata_moe_dispatch_windows(ctx, layout: strata_moe_layout_t, partition: str
                                 x: int, recv: int, capacity_rows: int, stream: int) -> int:
     return lib().strata_moe_dispatch_windows(ctx, ctypes.byref(layout), ctypes.byref(partition), n_cores, x, recv,
                                              capacity_rows, stream)
+
+
+def strata_allgather(ctx, R: int, src: int, dst: int, bytes_per_rank: int, stream: int) -> int:
+    return lib().strata_allgather(ctx, R, src, dst, bytes_per_rank, stream)
+
+
+def strata_alltoall(ctx, R: int, src: int, dst: int, bytes_per_slice: int, stream: int) -> int:
+    return lib().strata_alltoall(ctx, R, src, dst, bytes_per_slice, stream)
+
+
+def strata_broadcast(ctx, R: int, root: int, src: int, dst: int, nbytes: int, stream: int) -> int:
+    return lib().strata_broadcast(ctx, R, root, src, dst, nbytes, stream)
+
+
+def strata_reducescatter(ctx, R: int, src: int, dst: int, elems_per_slice: int, stream: int) -> int:
+    return lib().strata_reducescatter(ctx, R, src, dst, elems_per_slice, stream)
+
+
+def strata_allreduce(ctx, R: int, src: int, dst: int, elems: int, stream: int) -> int:
+    return lib().strata_allreduce(ctx, R, src, dst, elems, stream)
 
 
 # ---- convenience wrapper over torch tensors (memory + streams only) ---------
@@ -441,6 +467,37 @@ class MoEContext:
     def dispatch_windows(self, layout: Layout, part: Partition, x, recv) -> None:
         _check(strata_moe_dispatch_windows(self.h, layout.c, part.c, part.n_cores, x.data_ptr(), recv.data_ptr(),
                                            recv.shape[0], self._stream()), "strata_moe_dispatch_windows")
+
+    # full-mesh collectives over emulated ranks: tensors are [R, ...] slabs, one part per rank ------
+    def allgather(self, src, dst) -> None:
+        """src [R, n] -> dst [R, R, n] (any dtype; moved as bytes)."""
+        R = src.shape[0]
+        _check(strata_allgather(self.h, R, src.data_ptr(), dst.data_ptr(), src[0].numel() * src.element_size(),
+                                self._stream()), "strata_allgather")
+
+    def alltoall(self, src, dst) -> None:
+        """src [R, R, n] -> dst [R, R, n], dst[r, p] = src[p, r]."""
+        R = src.shape[0]
+        _check(strata_alltoall(self.h, R, src.data_ptr(), dst.data_ptr(), src[0, 0].numel() * src.element_size(),
+                               self._stream()), "strata_alltoall")
+
+    def broadcast(self, src, dst, root: int) -> None:
+        """src [R, n] -> dst [R, n], dst[r] = src[root]."""
+        R = src.shape[0]
+        _check(strata_broadcast(self.h, R, root, src.data_ptr(), dst.data_ptr(),
+                                src[0].numel() * src.element_size(), self._stream()), "strata_broadcast")
+
+    def reducescatter(self, src, dst) -> None:
+        """src bf16 [R, R, n] -> dst bf16 [R, n], dst[r] = sum over p of src[p, r] (rank order, fp32)."""
+        R = src.shape[0]
+        _check(strata_reducescatter(self.h, R, src.data_ptr(), dst.data_ptr(), src[0, 0].numel(), self._stream()),
+               "strata_reducescatter")
+
+    def allreduce(self, src, dst) -> None:
+        """src bf16 [R, n] -> dst bf16 [R, n], dst[r] = sum over p of src[p] (rank order, fp32)."""
+        R = src.shape[0]
+        _check(strata_allreduce(self.h, R, src.data_ptr(), dst.data_ptr(), src[0].numel(), self._stream()),
+               "strata_allreduce")
 
     def device_status(self) -> int:
         rc, st = strata_device_status(self.h, self._stream())

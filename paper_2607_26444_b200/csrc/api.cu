@@ -11,6 +11,7 @@ namespace strata {
 cudaError_t configure_layout_kernels();
 cudaError_t configure_dispatch_kernels();
 cudaError_t configure_partition_kernels();
+cudaError_t configure_collective_kernels();
 }  // namespace strata
 
 struct strata_region {
@@ -73,6 +74,7 @@ size_t workspace_bytes(const strata_moe_shape& s)
 
 WorkQueue dispatch_queue(const strata_ctx* c) { return WorkQueue{reinterpret_cast<unsigned int*>(c->ws) + 2}; }
 WorkQueue combine_queue(const strata_ctx* c) { return WorkQueue{reinterpret_cast<unsigned int*>(c->ws) + 4}; }
+WorkQueue collective_queue(const strata_ctx* c) { return WorkQueue{reinterpret_cast<unsigned int*>(c->ws) + 6}; }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -148,7 +150,7 @@ strata_status strata_ctx_create(strata_ctx** out, const strata_moe_shape* shape,
         if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
             return STRATA_ERR_CUDA;
         if (configure_layout_kernels() != cudaSuccess || configure_dispatch_kernels() != cudaSuccess ||
-            configure_partition_kernels() != cudaSuccess) {
+            configure_partition_kernels() != cudaSuccess || configure_collective_kernels() != cudaSuccess) {
             cudaGetLastError();
             return STRATA_ERR_CUDA;
         }
@@ -476,6 +478,110 @@ strata_status strata_moe_dispatch_windows(strata_ctx* ctx, const strata_moe_layo
     return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
 }
 
+// ---- full-mesh collectives over emulated ranks ------------------------------------------------
+
+namespace {
+constexpr int kMaxCollectiveRanks = 1024;
+
+// checks shared by the five operators
+strata_status collective_prologue(strata_ctx* ctx, int32_t R, const void* in, void* out)
+{
+    if (!ctx || !in || !out) return STRATA_ERR_INVALID_ARG;
+    if (R < 1 || R > kMaxCollectiveRanks) return STRATA_ERR_INVALID_ARG;
+    if (!aligned16(in) || !aligned16(out)) return STRATA_ERR_ALIGNMENT;
+    if (!ctx->ws) return STRATA_ERR_WORKSPACE;
+    return STRATA_OK;
+}
+
+strata_status run_copy(strata_ctx* ctx, const void* in, void* out, unsigned long long n_slices,
+                       unsigned long long slice_bytes, unsigned int inner, unsigned long long stride_a,
+                       unsigned long long stride_b, int fan, unsigned long long fan_stride, void* stream)
+{
+    if (slice_bytes % 16 != 0) return STRATA_ERR_SHAPE;
+    if (slice_bytes == 0) return STRATA_OK;
+    const unsigned long long chunk = collective_chunk_bytes();
+    const unsigned long long cps = (slice_bytes + chunk - 1) / chunk;
+    if (cps > 0xfffffffeull / n_slices) return STRATA_ERR_SHAPE;
+    if (ctx->device < 0) return STRATA_ERR_CUDA;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return STRATA_ERR_CUDA;
+    cudaError_t err = launch_slice_copy(in, out, n_slices, slice_bytes, inner, stride_a, stride_b, fan, fan_stride,
+                                        ctx->ws, collective_queue(ctx), ctx->n_sm, ctx->trace,
+                                        static_cast<cudaStream_t>(stream));
+    {
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        ctx->launches += 1;
+    }
+    return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
+}
+
+strata_status run_reduce(strata_ctx* ctx, const void* in, void* out, unsigned long long elems, int R, int fan,
+                         void* stream)
+{
+    if (elems % 8 != 0) return STRATA_ERR_SHAPE;
+    if (elems == 0) return STRATA_OK;
+    const unsigned long long n_vec = elems / 8;
+    if (n_vec / 128 >= 0xfffffffeull) return STRATA_ERR_SHAPE;
+    if (ctx->device < 0) return STRATA_ERR_CUDA;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return STRATA_ERR_CUDA;
+    cudaError_t err = launch_slice_reduce(in, out, n_vec, R, fan, collective_queue(ctx), ctx->n_sm, ctx->trace,
+                                          static_cast<cudaStream_t>(stream));
+    {
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        ctx->launches += 1;
+    }
+    return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
+}
+}  // namespace
+
+strata_status strata_allgather(strata_ctx* ctx, int32_t R, const void* in, void* out, size_t bytes_per_rank,
+                               void* stream)
+{
+    strata_status st = collective_prologue(ctx, R, in, out);
+    if (st != STRATA_OK) return st;
+    // slice p = rank p's input; copy f lands in rank f's output at offset p*M
+    return run_copy(ctx, in, out, (unsigned long long)R, bytes_per_rank, 1u, bytes_per_rank, 0ull, R,
+                    (unsigned long long)R * bytes_per_rank, stream);
+}
+
+strata_status strata_alltoall(strata_ctx* ctx, int32_t R, const void* in, void* out, size_t bytes_per_slice,
+                              void* stream)
+{
+    strata_status st = collective_prologue(ctx, R, in, out);
+    if (st != STRATA_OK) return st;
+    // slice s = p*R + r (sender p, receiver r) lands at (r*R + p)*S
+    return run_copy(ctx, in, out, (unsigned long long)R * R, bytes_per_slice, (unsigned int)R, bytes_per_slice,
+                    (unsigned long long)R * bytes_per_slice, 1, 0ull, stream);
+}
+
+strata_status strata_broadcast(strata_ctx* ctx, int32_t R, int32_t root, const void* in, void* out, size_t bytes,
+                               void* stream)
+{
+    strata_status st = collective_prologue(ctx, R, in, out);
+    if (st != STRATA_OK) return st;
+    if (root < 0 || root >= R) return STRATA_ERR_INVALID_ARG;
+    return run_copy(ctx, static_cast<const unsigned char*>(in) + (size_t)root * bytes, out, 1ull, bytes, 1u, 0ull, 0ull,
+                    R, bytes, stream);
+}
+
+strata_status strata_reducescatter(strata_ctx* ctx, int32_t R, const void* in, void* out, size_t elems_per_slice,
+                                   void* stream)
+{
+    strata_status st = collective_prologue(ctx, R, in, out);
+    if (st != STRATA_OK) return st;
+    if (elems_per_slice % 8 != 0) return STRATA_ERR_SHAPE;
+    // out, flat over [R][S], is the sum over the peers of their flat [R][S] inputs
+    return run_reduce(ctx, in, out, (unsigned long long)R * elems_per_slice, R, 1, stream);
+}
+
+strata_status strata_allreduce(strata_ctx* ctx, int32_t R, const void* in, void* out, size_t elems, void* stream)
+{
+    strata_status st = collective_prologue(ctx, R, in, out);
+    if (st != STRATA_OK) return st;
+    return run_reduce(ctx, in, out, elems, R, R, stream);
+}
+
 strata_status strata_moe_recv_view(strata_ctx* ctx, const int32_t* h_rank_offset, int rank, void* recv,
                                    void** rank_base, int64_t* rows)
 {
@@ -506,8 +612,8 @@ strata_status strata_device_status(strata_ctx* ctx, void* stream, strata_status*
     }
     if (word != 0) {
         // clear the status word; after an error also the ticket and the work-claim counters, which a
-        // kernel that gave up may have left non-zero (header words 0..5)
-        if (cudaMemsetAsync(ctx->ws, 0, 6 * sizeof(int), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) {
+        // kernel that gave up may have left non-zero (header words 0..7)
+        if (cudaMemsetAsync(ctx->ws, 0, 8 * sizeof(int), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) {
             cudaGetLastError();
             return STRATA_ERR_CUDA;
         }

@@ -1,0 +1,276 @@
+// Full-mesh collectives over emulated ranks (paper Sec. 6.1): an operator is a slice map (which
+// byte ranges go where) plus a memory action (copy, or accumulate).  Two kernels execute every
+// operator of the family; the frontends in the C-ABI layer only fill in the slice map.
+//
+// slice_copy_kernel   all-gather, all-to-all, broadcast.  A slice is cut into chunks of at most one
+//     stage; a unit is one chunk: one bulk load global->shared, then `fan` bulk stores shared->global
+//     (fan = R for all-gather and broadcast: the R pulls of one slice collapse into one read, since
+//     every emulated rank lives in the same memory; fan = 1 for all-to-all).  Single-warp CTAs run
+//     the SM's bulk-copy engine as a DMA program, exactly like the bf16 token dispatch; units are
+//     claimed in order from a counter in the workspace.
+// slice_reduce_kernel reduce-scatter, all-reduce.  A thread owns one 16-byte vector (8 bf16) of the
+//     output at a time: it issues up to 8 independent streaming loads (one per peer), adds them in
+//     binary32 in rank order, repeats for the next 8 peers, rounds once to bf16 and writes `fan`
+//     copies (fan = R for all-reduce).  The operands are accumulated on chip and each destination is
+//     written by exactly one thread, so the paper's atomic write-back (needed when several cores
+//     update the same memory) has nothing to protect here.
+#include "common.cuh"
+
+namespace strata {
+
+namespace {
+
+constexpr int kCopyStages = 3;
+constexpr uint32_t kCopyChunkBytes = 16384;
+constexpr int kCopyCtasPerSm = 2;
+constexpr int kReduceThreads = 128;
+constexpr int kReduceUnitsPerCta = 24;    // vectors per unit shrink until a CTA can expect this many units
+
+struct CopyParams {
+    const unsigned char* in;
+    unsigned char* out;
+    unsigned long long slice_bytes;
+    unsigned int chunks_per_slice;
+    unsigned int n_units;                 // n_slices * chunks_per_slice
+    // destination of slice s, copy f:  out + f*fan_stride + (s / inner)*stride_a + (s % inner)*stride_b
+    unsigned int inner;
+    unsigned long long stride_a, stride_b;
+    int fan;
+    unsigned long long fan_stride;
+    int* status;
+    WorkQueue wq;
+    TraceBuf trace;
+};
+
+__global__ void __launch_bounds__(32) slice_copy_kernel(CopyParams p)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kCopyStages * kCopyChunkBytes);
+    unsigned int* s_unit = reinterpret_cast<unsigned int*>(bars + kCopyStages);
+    const int lane = threadIdx.x;
+    const unsigned int n_units = p.n_units;
+
+    if (lane == 0) {
+        for (int s = 0; s < kCopyStages; ++s) {
+            mbar_init(&bars[s], 1);
+            s_unit[s] = kNoUnit;
+        }
+        mbar_fence_init();
+    }
+    __syncwarp();
+    const uint64_t pol = policy_evict_first();
+    griddep_wait();
+    if (lane == 0) trace_begin(p.trace);
+
+    auto decode = [&](unsigned int u, unsigned int& slice, unsigned long long& off, uint32_t& bytes) {
+        slice = u / p.chunks_per_slice;
+        off = (unsigned long long)(u - slice * p.chunks_per_slice) * kCopyChunkBytes;
+        const unsigned long long left = p.slice_bytes - off;
+        bytes = left < kCopyChunkBytes ? (uint32_t)left : kCopyChunkBytes;
+    };
+    bool triggered = false, exhausted = false;
+    const unsigned int n_static = (unsigned int)(kCopyStages - 1) * gridDim.x;
+    auto issue_load = [&](long long j) {   // lane 0 only
+        const int s = (int)(j % kCopyStages);
+        unsigned int u;
+        if (j < kCopyStages - 1) {
+            u = blockIdx.x + (unsigned int)j * gridDim.x;
+            if (u >= n_units) u = kNoUnit;
+        } else {
+            u = claim_unit(p.wq, n_units, n_static, exhausted);
+        }
+        s_unit[s] = u;
+        if (u == kNoUnit) {
+            if (!triggered) griddep_launch_dependents();
+            triggered = true;
+            return;
+        }
+        unsigned int slice;
+        unsigned long long off;
+        uint32_t bytes;
+        decode(u, slice, off, bytes);
+        mbar_expect_tx(&bars[s], bytes);
+        bulk_g2s(smem + (size_t)s * kCopyChunkBytes, p.in + (size_t)slice * p.slice_bytes + off, bytes, &bars[s], pol);
+    };
+
+    if (lane == 0)
+        for (long long j = 0; j < kCopyStages - 1; ++j) issue_load(j);
+    __syncwarp();
+
+    bool ok = true;
+    StageClock wait_in(p.trace), wait_out(p.trace);
+    for (long long j = 0;; ++j) {
+        const int s = (int)(j % kCopyStages);
+        const uint32_t parity = (uint32_t)((j / kCopyStages) & 1);
+        const unsigned int u = s_unit[s];
+        if (u == kNoUnit) break;
+        wait_in.begin();
+        ok = mbar_wait_bounded(&bars[s], parity);
+        wait_in.end();
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (lane == 0) {
+            unsigned int slice;
+            unsigned long long off;
+            uint32_t bytes;
+            decode(u, slice, off, bytes);
+            unsigned char* dst = p.out + (size_t)(slice / p.inner) * p.stride_a + (size_t)(slice % p.inner) * p.stride_b + off;
+            for (int f = 0; f < p.fan; ++f) bulk_s2g(dst + (size_t)f * p.fan_stride, smem + (size_t)s * kCopyChunkBytes, bytes);
+            bulk_commit();
+            wait_out.begin();
+            bulk_wait_read<1>();           // the stage refilled next held unit j-1: its stores have left shared memory
+            wait_out.end();
+            issue_load(j + kCopyStages - 1);
+        }
+        __syncwarp();
+    }
+    if (lane == 0) {
+        if (!ok) report_status(p.status, STRATA_ERR_TIMEOUT);
+        wait_out.begin();
+        bulk_wait_read<0>();
+        wait_out.end();
+        trace_end(p.trace, wait_in.total, wait_out.total);
+    }
+}
+
+struct ReduceParams {
+    const unsigned char* in;
+    unsigned char* out;
+    unsigned long long n_vec;             // 16-byte vectors of one reduced image
+    unsigned long long rank_stride;       // bytes between two peers' operands
+    int R;
+    int fan;                              // copies of the result
+    unsigned long long fan_stride;
+    unsigned int n_units;
+    unsigned int vec_per_unit;            // a multiple of the CTA size
+    WorkQueue wq;
+    TraceBuf trace;
+};
+
+__device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi)
+{
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+__device__ __forceinline__ void add8(float (&a)[8], const uint4& d)
+{
+    a[0] = __fadd_rn(a[0], __uint_as_float(d.x << 16));
+    a[1] = __fadd_rn(a[1], __uint_as_float(d.x & 0xffff0000u));
+    a[2] = __fadd_rn(a[2], __uint_as_float(d.y << 16));
+    a[3] = __fadd_rn(a[3], __uint_as_float(d.y & 0xffff0000u));
+    a[4] = __fadd_rn(a[4], __uint_as_float(d.z << 16));
+    a[5] = __fadd_rn(a[5], __uint_as_float(d.z & 0xffff0000u));
+    a[6] = __fadd_rn(a[6], __uint_as_float(d.w << 16));
+    a[7] = __fadd_rn(a[7], __uint_as_float(d.w & 0xffff0000u));
+}
+
+__global__ void __launch_bounds__(kReduceThreads) slice_reduce_kernel(ReduceParams p)
+{
+    const int tid = threadIdx.x;
+    __shared__ unsigned int s_next[2];
+    griddep_wait();
+    if (tid == 0) trace_begin(p.trace);
+
+    unsigned int u = blockIdx.x < p.n_units ? blockIdx.x : kNoUnit;
+    bool exhausted = false;
+    for (int j = 0; u != kNoUnit; ++j) {
+        if (tid == 0) {
+            const unsigned int nx = claim_unit(p.wq, p.n_units, gridDim.x, exhausted);
+            s_next[j & 1] = nx;
+            if (nx == kNoUnit) griddep_launch_dependents();
+        }
+        const unsigned long long v_begin = (unsigned long long)u * p.vec_per_unit;
+        const unsigned long long v_end = min(v_begin + p.vec_per_unit, p.n_vec);
+        for (unsigned long long v = v_begin + tid; v < v_end; v += kReduceThreads) {
+            const unsigned char* src = p.in + (size_t)v * 16;
+            float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            for (int p0 = 0; p0 < p.R; p0 += 8) {
+                uint4 d[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    d[k] = (p0 + k < p.R) ? ld_stream16(src + (size_t)(p0 + k) * p.rank_stride) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (p0 + k < p.R) add8(a, d[k]);
+            }
+            uint4 o;
+            o.x = pack2_bf16(a[0], a[1]);
+            o.y = pack2_bf16(a[2], a[3]);
+            o.z = pack2_bf16(a[4], a[5]);
+            o.w = pack2_bf16(a[6], a[7]);
+            unsigned char* dst = p.out + (size_t)v * 16;
+            for (int f = 0; f < p.fan; ++f) st_stream16(dst + (size_t)f * p.fan_stride, o);
+        }
+        __syncthreads();
+        u = s_next[j & 1];
+    }
+    if (tid == 0) trace_end(p.trace);
+}
+
+constexpr size_t kCopySmem = (size_t)kCopyStages * kCopyChunkBytes + kCopyStages * sizeof(uint64_t) + kCopyStages * sizeof(unsigned int) + 16;
+
+}  // namespace
+
+cudaError_t configure_collective_kernels()
+{
+    return cudaFuncSetAttribute(slice_copy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCopySmem);
+}
+
+uint32_t collective_chunk_bytes() { return kCopyChunkBytes; }
+
+cudaError_t launch_slice_copy(const void* in, void* out, unsigned long long n_slices, unsigned long long slice_bytes,
+                              unsigned int inner, unsigned long long stride_a, unsigned long long stride_b, int fan,
+                              unsigned long long fan_stride, int* status, WorkQueue wq, int n_sm, TraceBuf trace,
+                              cudaStream_t st)
+{
+    CopyParams p{};
+    p.in = static_cast<const unsigned char*>(in);
+    p.out = static_cast<unsigned char*>(out);
+    p.slice_bytes = slice_bytes;
+    p.chunks_per_slice = (unsigned int)((slice_bytes + kCopyChunkBytes - 1) / kCopyChunkBytes);
+    p.n_units = (unsigned int)(n_slices * p.chunks_per_slice);
+    p.inner = inner;
+    p.stride_a = stride_a;
+    p.stride_b = stride_b;
+    p.fan = fan;
+    p.fan_stride = fan_stride;
+    p.status = status;
+    p.wq = wq;
+    p.trace = trace;
+    const unsigned grid = (unsigned)max(1ll, min((long long)n_sm * kCopyCtasPerSm, (long long)p.n_units));
+    const bool small = (long long)(n_slices * slice_bytes) * (fan + 1) < kPdlMaxBytes;
+    return STRATA_LAUNCH_LONG(small, slice_copy_kernel, grid, 32, kCopySmem, st, p);
+}
+
+cudaError_t launch_slice_reduce(const void* in, void* out, unsigned long long n_vec, int R, int fan,
+                                WorkQueue wq, int n_sm, TraceBuf trace, cudaStream_t st)
+{
+    ReduceParams p{};
+    p.in = static_cast<const unsigned char*>(in);
+    p.out = static_cast<unsigned char*>(out);
+    p.n_vec = n_vec;
+    p.rank_stride = n_vec * 16ull;
+    p.R = R;
+    p.fan = fan;
+    p.fan_stride = n_vec * 16ull;
+    p.wq = wq;
+    p.trace = trace;
+    int per_sm = 0;
+    cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, slice_reduce_kernel, kReduceThreads, 0);
+    if (err != cudaSuccess) return err;
+    if (per_sm < 1) per_sm = 1;
+    const long long max_grid = (long long)n_sm * per_sm;
+    unsigned int m = 4;                   // vectors per thread per unit
+    while (m > 1 && (long long)((n_vec + (unsigned long long)m * kReduceThreads - 1) / ((unsigned long long)m * kReduceThreads)) <
+                        kReduceUnitsPerCta * max_grid)
+        m >>= 1;
+    p.vec_per_unit = m * kReduceThreads;
+    p.n_units = (unsigned int)((n_vec + p.vec_per_unit - 1) / p.vec_per_unit);
+    const unsigned grid = (unsigned)max(1ll, min(max_grid, (long long)p.n_units));
+    const bool small = (long long)(n_vec * 16ull) * (R + fan) < kPdlMaxBytes;
+    return STRATA_LAUNCH_LONG(small, slice_reduce_kernel, grid, kReduceThreads, 0, st, p);
+}
+
+}  // namespace strata

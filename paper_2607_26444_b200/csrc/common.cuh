@@ -5,13 +5,15 @@
 #include <stdint.h>
 
 #include "strata_moe.h"
+#include "strata_collective.h"
 
 namespace strata {
 
 // ---- workspace layout -----------------------------------------------------
 // word 0: device status (a strata_status, first error wins)
 // word 1: ticket of the layout kernel (returns to 0 after every call)
-// word 2: work-claim counter of dispatch, word 4: of combine (both return to 0 inside the kernel)
+// word 2: work-claim counter of dispatch, word 4: of combine, word 6: of the collectives (each returns
+//         to 0 inside the kernel)
 // bytes [256, ...): per-tile, per-expert counts, int32 [n_tiles, E]
 constexpr int kWsHeaderBytes = 256;
 constexpr int kLayoutThreads = 1024;   // threads per layout CTA
@@ -76,6 +78,13 @@ cudaError_t launch_partition(const strata_moe_shape& s, const strata_moe_layout_
 cudaError_t launch_dispatch_windows(const strata_moe_shape& s, const strata_moe_layout_t& L,
                                     const strata_partition_t& part, int n_cores, const void* x, void* recv,
                                     size_t capacity_rows, int* status, TraceBuf trace, cudaStream_t st);
+cudaError_t launch_slice_copy(const void* in, void* out, unsigned long long n_slices, unsigned long long slice_bytes,
+                              unsigned int inner, unsigned long long stride_a, unsigned long long stride_b, int fan,
+                              unsigned long long fan_stride, int* status, WorkQueue wq, int n_sm, TraceBuf trace,
+                              cudaStream_t st);
+cudaError_t launch_slice_reduce(const void* in, void* out, unsigned long long n_vec, int R, int fan, WorkQueue wq,
+                                int n_sm, TraceBuf trace, cudaStream_t st);
+uint32_t collective_chunk_bytes();
 int partition_max_units_supported();
 int partition_max_cores_supported();
 uint32_t windows_max_row_bytes();

@@ -20,7 +20,8 @@ def built():
 
 
 def declared_functions():
-    text = open(os.path.join(ROOT, "include", "strata_moe.h")).read()
+    inc = os.path.join(ROOT, "include")
+    text = "".join(open(os.path.join(inc, f)).read() for f in sorted(os.listdir(inc)) if f.endswith(".h"))
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(strata_[a-z_0-9]+)\s*\(", text)))
 
@@ -188,3 +189,35 @@ def test_null_context_everywhere():
     assert B.strata_moe_layout(None, 16, _fake_layout(), None) == B.STRATA_ERR_INVALID_ARG
     rc, _ = B.strata_device_status(None, None)
     assert rc == B.STRATA_ERR_INVALID_ARG
+
+
+def test_collectives_reject_bad_arguments_before_any_launch():
+    rc, h = B.strata_ctx_create(shape(), -1)
+    assert rc == B.STRATA_OK
+    try:
+        fake = 1 << 20
+        # no workspace yet
+        assert B.strata_allgather(h, 4, fake, 2 * fake, 64, None) == B.STRATA_ERR_WORKSPACE
+        assert B.strata_ctx_set_workspace(h, 256 << 10, 1 << 30) == B.STRATA_OK
+        assert B.strata_allgather(h, 0, fake, 2 * fake, 64, None) == B.STRATA_ERR_INVALID_ARG
+        assert B.strata_allgather(h, 2000, fake, 2 * fake, 64, None) == B.STRATA_ERR_INVALID_ARG
+        assert B.strata_allgather(h, 4, None, 2 * fake, 64, None) == B.STRATA_ERR_INVALID_ARG
+        assert B.strata_allgather(h, 4, fake + 8, 2 * fake, 64, None) == B.STRATA_ERR_ALIGNMENT
+        assert B.strata_alltoall(h, 4, fake, 2 * fake + 4, 64, None) == B.STRATA_ERR_ALIGNMENT
+        assert B.strata_broadcast(h, 4, 4, fake, 2 * fake, 64, None) == B.STRATA_ERR_INVALID_ARG
+        assert B.strata_broadcast(h, 4, -1, fake, 2 * fake, 64, None) == B.STRATA_ERR_INVALID_ARG
+        assert B.strata_allgather(h, 4, fake, 2 * fake, 40, None) == B.STRATA_ERR_SHAPE
+        assert B.strata_allreduce(h, 4, fake, 2 * fake, 12, None) == B.STRATA_ERR_SHAPE
+        assert B.strata_reducescatter(h, 4, fake, 2 * fake, 4, None) == B.STRATA_ERR_SHAPE
+        assert B.strata_allgather(h, 4, fake, 2 * fake, 0, None) == B.STRATA_OK        # nothing to move
+        # a host-only context never launches
+        for rc in (B.strata_allgather(h, 4, fake, 2 * fake, 64, None),
+                   B.strata_alltoall(h, 4, fake, 2 * fake, 64, None),
+                   B.strata_broadcast(h, 4, 1, fake, 2 * fake, 64, None),
+                   B.strata_reducescatter(h, 4, fake, 2 * fake, 64, None),
+                   B.strata_allreduce(h, 4, fake, 2 * fake, 64, None)):
+            assert rc == B.STRATA_ERR_CUDA
+        rc, n = B.strata_ctx_launch_count(h)
+        assert rc == B.STRATA_OK and n == 0
+    finally:
+        B.strata_ctx_destroy(h)
