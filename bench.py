@@ -413,7 +413,11 @@ def window_partitioning_report(cfg: wl.MoEConfig, dev_index: int, unit_rows: int
     return out
 
 
-def collectives_report(dev_index: int, R: int = 32, per_rank_mib=(1, 16), iters: int = 10, warmup: int = 3):
+COLLECTIVE_OPS = ("allgather", "alltoall", "broadcast", "reducescatter", "allreduce")
+
+
+def collectives_report(dev_index: int, R: int = 32, per_rank_kib=(64, 1024, 16384), iters: int = 10,
+                       warmup: int = 3, only=COLLECTIVE_OPS):
     """Full-mesh collectives over R emulated ranks (paper Sec. 6.1 / 7.1: 32 ranks, payloads from 1 MiB
     per rank): median microseconds and effective HBM GB/s of each operator.  Algorithmic bytes: the
     operator's input read once plus its output written once.  A working set below the 126 MB L2 is
@@ -424,13 +428,13 @@ def collectives_report(dev_index: int, R: int = 32, per_rank_mib=(1, 16), iters:
     ctx = B.MoEContext(4, 128, 1024, 16, 2, device=dev_index)
     peak, _ = measured_peak()
     rep = {"R": R, "iters": iters, "bytes": "input read once + output written once", "sizes": {}}
-    for mib in per_rank_mib:
-        M = mib << 20                                   # bytes per rank
+    for kib in per_rank_kib:
+        M = kib << 10                                   # bytes per rank
         E = M // 2                                      # bf16 elements per rank
         x = torch.empty((R, E), dtype=torch.int16, device=dev)
         x.view(torch.uint8).random_(0, 256)
         x &= 0x3FFF | -32768                            # finite bf16 patterns of magnitude < 2
-        big = torch.empty((R, R, E), dtype=torch.int16, device=dev)
+        big = torch.empty((R, R, E), dtype=torch.int16, device=dev) if "allgather" in only else None
         same = torch.empty((R, E), dtype=torch.int16, device=dev)
         small = torch.empty((E,), dtype=torch.int16, device=dev)
         ops = {
@@ -442,6 +446,8 @@ def collectives_report(dev_index: int, R: int = 32, per_rank_mib=(1, 16), iters:
         }
         entry = {}
         for name, (fn, nbytes) in ops.items():
+            if name not in only:
+                continue
             for _ in range(warmup):
                 fn()
             torch.cuda.synchronize()
@@ -459,11 +465,13 @@ def collectives_report(dev_index: int, R: int = 32, per_rank_mib=(1, 16), iters:
                            "l2_resident": nbytes < 126_000_000}
         # the timed buffers hold what the operators define (checked with torch views; parity with the
         # oracle is the tests' job)
-        ok = bool(torch.equal(big[R - 1], x)) and bool(torch.equal(same, same[0].expand(R, E)))
+        ok = big is None or bool(torch.equal(big[R - 1], x))
+        if "allreduce" in only or "broadcast" in only:
+            ok = ok and bool(torch.equal(same, same[0].expand(R, E)))
         ctx.alltoall(x.view(R, R, E // R), same.view(R, R, E // R))
         ok = ok and bool(torch.equal(same.view(R, R, E // R), x.view(R, R, E // R).transpose(0, 1)))
         entry["verified"] = ok and ctx.device_status() == B.STRATA_OK
-        rep["sizes"][f"{mib}MiB_per_rank"] = entry
+        rep["sizes"][f"{kib}KiB_per_rank"] = entry
         del x, big, same, small
         torch.cuda.empty_cache()
     ctx.close()
@@ -690,6 +698,11 @@ def main():
     ap.add_argument("--workload", default="prefill", choices=wl.CONFIG_ORDER,
                     help="configuration to step through (the bench line is quoted on the default)")
     ap.add_argument("--tokens-per-rank", type=int, default=0, help="shrink T (profiling captures only)")
+    ap.add_argument("--collectives", action="store_true",
+                    help="print only the report on the full-mesh collectives (one JSON object; not the bench line)")
+    ap.add_argument("--collective-kib", type=int, nargs="+", default=[64, 1024, 16384], help="payload per rank, KiB")
+    ap.add_argument("--collective-iters", type=int, default=10)
+    ap.add_argument("--collective-ops", nargs="+", default=list(COLLECTIVE_OPS), choices=COLLECTIVE_OPS)
     ap.add_argument("--profile", action="store_true",
                     help="for runs under a profiler: no e2e/cpu/other legs, warm-up not clamped")
     args = ap.parse_args()
@@ -702,6 +715,12 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.collectives:
+        if rank == 0:
+            print(json.dumps(collectives_report(local_rank, per_rank_kib=tuple(args.collective_kib),
+                                                iters=args.collective_iters, warmup=min(args.warmup, 3),
+                                                only=tuple(args.collective_ops))), flush=True)
         return
     run_gpu(args, rank, local_rank, world)
 
