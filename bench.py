@@ -460,7 +460,16 @@ def collectives_report(dev_index: int, R: int = 32, per_rank_kib=(64, 1024, 1638
             torch.cuda.synchronize()
             ts = sorted(ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(iters))
             med = ts[len(ts) // 2]
-            entry[name] = {"median_us": round(med, 2), "min_us": round(ts[0], 2), "bytes": nbytes,
+            # the same calls with no event between them: what a stream of such calls costs per call (an
+            # event record between two short kernels adds to both, and events tick in ~2 us steps)
+            torch.cuda._sleep(10_000_000)
+            ev[0].record()
+            for i in range(4 * iters):
+                fn()
+            ev[1].record()
+            torch.cuda.synchronize()
+            entry[name] = {"median_us": round(med, 2), "min_us": round(ts[0], 2),
+                           "back_to_back_us": round(ev[0].elapsed_time(ev[1]) * 1e3 / (4 * iters), 2), "bytes": nbytes,
                            "GBs": round(nbytes / med / 1e3, 1), "frac_of_measured_peak": round(nbytes / med / 1e3 / peak, 4),
                            "l2_resident": nbytes < 126_000_000}
         # the timed buffers hold what the operators define (checked with torch views; parity with the

@@ -7,13 +7,15 @@
 //     (fan = R for all-gather and broadcast: the R pulls of one slice collapse into one read, since
 //     every emulated rank lives in the same memory; fan = 1 for all-to-all).  Single-warp CTAs run
 //     the SM's bulk-copy engine as a DMA program, exactly like the bf16 token dispatch; units are
-//     claimed in order from a counter in the workspace.
+//     claimed in order from a counter in the workspace.  Payloads too small to give every CTA two units
+//     are latency bound: the fan copies of a chunk are then dealt to several units and the chunks shrink.
 // slice_reduce_kernel reduce-scatter, all-reduce.  A thread owns one 16-byte vector (8 bf16) of the
 //     output at a time: it issues up to 8 independent streaming loads (one per peer), adds them in
 //     binary32 in rank order, repeats for the next 8 peers, rounds once to bf16 and writes `fan`
 //     copies (fan = R for all-reduce).  The operands are accumulated on chip and each destination is
 //     written by exactly one thread, so the paper's atomic write-back (needed when several cores
-//     update the same memory) has nothing to protect here.
+//     update the same memory) has nothing to protect here.  Payloads that do not fill the GPU run as
+//     one-warp CTAs with up to 32 peers' loads in flight per thread (one round trip to memory).
 #include "common.cuh"
 
 namespace strata {
@@ -30,8 +32,11 @@ struct CopyParams {
     const unsigned char* in;
     unsigned char* out;
     unsigned long long slice_bytes;
+    unsigned int chunk_bytes;             // <= kCopyChunkBytes, a multiple of 16
     unsigned int chunks_per_slice;
-    unsigned int n_units;                 // n_slices * chunks_per_slice
+    unsigned int fan_groups;              // the fan copies of a chunk are dealt to this many units
+    unsigned int fan_per_group;
+    unsigned int n_units;                 // n_slices * chunks_per_slice * fan_groups
     // destination of slice s, copy f:  out + f*fan_stride + (s / inner)*stride_a + (s % inner)*stride_b
     unsigned int inner;
     unsigned long long stride_a, stride_b;
@@ -62,11 +67,13 @@ __global__ void __launch_bounds__(32) slice_copy_kernel(CopyParams p)
     griddep_wait();
     if (lane == 0) trace_begin(p.trace);
 
-    auto decode = [&](unsigned int u, unsigned int& slice, unsigned long long& off, uint32_t& bytes) {
-        slice = u / p.chunks_per_slice;
-        off = (unsigned long long)(u - slice * p.chunks_per_slice) * kCopyChunkBytes;
+    auto decode = [&](unsigned int u, unsigned int& slice, unsigned long long& off, uint32_t& bytes, int& f0) {
+        const unsigned int c = u / p.fan_groups;               // chunk index over all slices
+        f0 = (int)((u - c * p.fan_groups) * p.fan_per_group);
+        slice = c / p.chunks_per_slice;
+        off = (unsigned long long)(c - slice * p.chunks_per_slice) * p.chunk_bytes;
         const unsigned long long left = p.slice_bytes - off;
-        bytes = left < kCopyChunkBytes ? (uint32_t)left : kCopyChunkBytes;
+        bytes = left < p.chunk_bytes ? (uint32_t)left : p.chunk_bytes;
     };
     bool triggered = false, exhausted = false;
     const unsigned int n_static = (unsigned int)(kCopyStages - 1) * gridDim.x;
@@ -88,7 +95,8 @@ __global__ void __launch_bounds__(32) slice_copy_kernel(CopyParams p)
         unsigned int slice;
         unsigned long long off;
         uint32_t bytes;
-        decode(u, slice, off, bytes);
+        int f0;
+        decode(u, slice, off, bytes, f0);
         mbar_expect_tx(&bars[s], bytes);
         bulk_g2s(smem + (size_t)s * kCopyChunkBytes, p.in + (size_t)slice * p.slice_bytes + off, bytes, &bars[s], pol);
     };
@@ -113,9 +121,11 @@ __global__ void __launch_bounds__(32) slice_copy_kernel(CopyParams p)
             unsigned int slice;
             unsigned long long off;
             uint32_t bytes;
-            decode(u, slice, off, bytes);
+            int f0;
+            decode(u, slice, off, bytes, f0);
             unsigned char* dst = p.out + (size_t)(slice / p.inner) * p.stride_a + (size_t)(slice % p.inner) * p.stride_b + off;
-            for (int f = 0; f < p.fan; ++f) bulk_s2g(dst + (size_t)f * p.fan_stride, smem + (size_t)s * kCopyChunkBytes, bytes);
+            const int f1 = min(p.fan, f0 + (int)p.fan_per_group);
+            for (int f = f0; f < f1; ++f) bulk_s2g(dst + (size_t)f * p.fan_stride, smem + (size_t)s * kCopyChunkBytes, bytes);
             bulk_commit();
             wait_out.begin();
             bulk_wait_read<1>();           // the stage refilled next held unit j-1: its stores have left shared memory
@@ -142,7 +152,7 @@ struct ReduceParams {
     int fan;                              // copies of the result
     unsigned long long fan_stride;
     unsigned int n_units;
-    unsigned int vec_per_unit;            // a multiple of the CTA size
+    unsigned int vec_per_unit;            // a multiple of the CTA size (128 threads; 32 for latency-bound sizes)
     WorkQueue wq;
     TraceBuf trace;
 };
@@ -166,6 +176,10 @@ __device__ __forceinline__ void add8(float (&a)[8], const uint4& d)
     a[7] = __fadd_rn(a[7], __uint_as_float(d.w & 0xffff0000u));
 }
 
+// B = peers whose operands a thread has in flight at once.  8 keeps 9 CTAs per SM for payloads that are
+// bandwidth bound; 32 serves a whole 32-rank reduction with one round trip to memory, for payloads so small
+// that the grid does not fill the GPU and the time is the latency of dependent loads.
+template <int B>
 __global__ void __launch_bounds__(kReduceThreads) slice_reduce_kernel(ReduceParams p)
 {
     const int tid = threadIdx.x;
@@ -183,16 +197,16 @@ __global__ void __launch_bounds__(kReduceThreads) slice_reduce_kernel(ReducePara
         }
         const unsigned long long v_begin = (unsigned long long)u * p.vec_per_unit;
         const unsigned long long v_end = min(v_begin + p.vec_per_unit, p.n_vec);
-        for (unsigned long long v = v_begin + tid; v < v_end; v += kReduceThreads) {
+        for (unsigned long long v = v_begin + tid; v < v_end; v += blockDim.x) {
             const unsigned char* src = p.in + (size_t)v * 16;
             float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            for (int p0 = 0; p0 < p.R; p0 += 8) {
-                uint4 d[8];
+            for (int p0 = 0; p0 < p.R; p0 += B) {
+                uint4 d[B];
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
+                for (int k = 0; k < B; ++k)
                     d[k] = (p0 + k < p.R) ? ld_stream16(src + (size_t)(p0 + k) * p.rank_stride) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
+                for (int k = 0; k < B; ++k)
                     if (p0 + k < p.R) add8(a, d[k]);
             }
             uint4 o;
@@ -229,8 +243,25 @@ cudaError_t launch_slice_copy(const void* in, void* out, unsigned long long n_sl
     p.in = static_cast<const unsigned char*>(in);
     p.out = static_cast<unsigned char*>(out);
     p.slice_bytes = slice_bytes;
-    p.chunks_per_slice = (unsigned int)((slice_bytes + kCopyChunkBytes - 1) / kCopyChunkBytes);
-    p.n_units = (unsigned int)(n_slices * p.chunks_per_slice);
+    // Large payloads: 16 KB chunks, all fan copies of a chunk from one load.  When that leaves the grid
+    // short of units (small payloads are latency bound: a unit's stores are issued by one thread), first the
+    // fan copies of a chunk are dealt to several units (each re-reads the chunk, an L2 hit), then the chunks
+    // shrink, down to 2 KB.
+    const unsigned long long want = 2ull * (unsigned long long)n_sm * kCopyCtasPerSm;
+    unsigned long long chunk = kCopyChunkBytes, fpg = (unsigned long long)fan;
+    auto units = [&]() {
+        return n_slices * ((slice_bytes + chunk - 1) / chunk) * (((unsigned long long)fan + fpg - 1) / fpg);
+    };
+    while (units() < want) {
+        if (fpg > 1) fpg = (fpg + 1) / 2;
+        else if (chunk > 2048) chunk /= 2;
+        else break;
+    }
+    p.chunk_bytes = (unsigned int)chunk;
+    p.chunks_per_slice = (unsigned int)((slice_bytes + chunk - 1) / chunk);
+    p.fan_per_group = (unsigned int)fpg;
+    p.fan_groups = (unsigned int)(((unsigned long long)fan + fpg - 1) / fpg);
+    p.n_units = (unsigned int)units();
     p.inner = inner;
     p.stride_a = stride_a;
     p.stride_b = stride_b;
@@ -257,8 +288,15 @@ cudaError_t launch_slice_reduce(const void* in, void* out, unsigned long long n_
     p.fan_stride = n_vec * 16ull;
     p.wq = wq;
     p.trace = trace;
+    const bool small = (long long)(n_vec * 16ull) * (R + fan) < kPdlMaxBytes;
+    if (R > 8 && n_vec <= (unsigned long long)n_sm * 2u * kReduceThreads) {
+        // latency bound: one-warp CTAs so that more SMs take part, the deepest batch of loads
+        p.vec_per_unit = 32;
+        p.n_units = (unsigned int)((n_vec + 31) / 32);
+        return STRATA_LAUNCH_LONG(small, slice_reduce_kernel<32>, p.n_units, 32, 0, st, p);
+    }
     int per_sm = 0;
-    cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, slice_reduce_kernel, kReduceThreads, 0);
+    cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, slice_reduce_kernel<8>, kReduceThreads, 0);
     if (err != cudaSuccess) return err;
     if (per_sm < 1) per_sm = 1;
     const long long max_grid = (long long)n_sm * per_sm;
@@ -269,8 +307,7 @@ cudaError_t launch_slice_reduce(const void* in, void* out, unsigned long long n_
     p.vec_per_unit = m * kReduceThreads;
     p.n_units = (unsigned int)((n_vec + p.vec_per_unit - 1) / p.vec_per_unit);
     const unsigned grid = (unsigned)max(1ll, min(max_grid, (long long)p.n_units));
-    const bool small = (long long)(n_vec * 16ull) * (R + fan) < kPdlMaxBytes;
-    return STRATA_LAUNCH_LONG(small, slice_reduce_kernel, grid, kReduceThreads, 0, st, p);
+    return STRATA_LAUNCH_LONG(small, slice_reduce_kernel<8>, grid, kReduceThreads, 0, st, p);
 }
 
 }  // namespace strata
