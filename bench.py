@@ -418,7 +418,7 @@ COLLECTIVE_OPS = ("allgather", "alltoall", "broadcast", "reducescatter", "allred
 
 def collectives_report(dev_index: int, R: int = 32, per_rank_kib=(64, 1024, 16384), iters: int = 10,
                        warmup: int = 3, only=COLLECTIVE_OPS):
-    """Full-mesh collectives over R emulated ranks (paper Sec. 6.1 / 7.1: 32 ranks, payloads from 1 MiB
+    """Full-mesh collectives over R emulated ranks (paper Sec. 6.1 / 8.1: 32 ranks, payloads from 1 MiB
     per rank): median microseconds and effective HBM GB/s of each operator.  Algorithmic bytes: the
     operator's input read once plus its output written once.  A working set below the 126 MB L2 is
     marked, its GB/s is not an HBM figure."""

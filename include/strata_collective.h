@@ -5,7 +5,7 @@
  * transfers that complete in one logical step.  Data-movement operators run in pull mode (a rank
  * reads the peers' slices and writes them into its own output, no producer-consumer handshake);
  * reduction-bearing operators load the peers' operands on chip and accumulate them into the local
- * destination.  The paper measures them at 32 ranks with 1 MiB .. 1 GiB per rank (Sec. 7.1).
+ * destination.  The paper measures them at 32 ranks with 1 MiB .. 1 GiB per rank (Sec. 8.1).
  *
  * Here all R ranks are partitions of ONE GPU's memory, as for the MoE path: rank r's input is the
  * r-th equal part of `in`, its output the r-th equal part of `out`.  Nothing crosses a link, so what

@@ -87,7 +87,7 @@ typedef struct {
 
 typedef struct strata_ctx strata_ctx;   /* opaque, host side */
 
-/* Routing metadata (paper App. C, "token placement": destination expert,
+/* Routing metadata (paper App. D, "token placement": destination expert,
  * per-expert counts, prefix-sum offsets, token-local offsets), produced by
  * strata_moe_layout and consumed by dispatch and combine.  All members are
  * device pointers to int32 arrays owned by the caller. */
@@ -137,7 +137,7 @@ strata_status strata_ctx_launch_count(strata_ctx *ctx, uint64_t *count);
  * rows, and the nanoseconds it was blocked waiting for outgoing rows to leave shared memory (the
  * last two are filled by the bf16 dispatch kernel, zero elsewhere).  Each launch overwrites the
  * previous one's records.  dptr = NULL turns tracing off (the default).  The spread of the end
- * times is the load-balance evidence the paper reports per core (Sec. 8.5). */
+ * times is the load-balance evidence the paper reports per core (Sec. 9.6). */
 strata_status strata_ctx_set_trace(strata_ctx *ctx, uint64_t *dptr, size_t capacity_ctas);
 
 /* ---- pool: registration at allocation time ------------------------------
@@ -146,7 +146,7 @@ strata_status strata_ctx_set_trace(strata_ctx *ctx, uint64_t *dptr, size_t capac
  * only performs a cheap local readiness check (phase 2).  Here the caller
  * allocates (e.g. a torch tensor), the library records [base, base+bytes) and
  * can sub-allocate from it, so the receive buffer handed to dispatch is the
- * very tensor the expert GEMM reads: no staging copy exists (Sec. 2.2 / 7.1
+ * very tensor the expert GEMM reads: no staging copy exists (Sec. 2.2 / 8.1
  * describe the staging copies this removes).  Rank partitions are disjoint
  * sub-ranges of one address space (Sec. 5.2). */
 strata_status strata_pool_register(strata_ctx *ctx, void *dbase, size_t bytes, uint64_t *region_id);
@@ -159,7 +159,7 @@ strata_status strata_pool_reset(strata_ctx *ctx, uint64_t region_id);
 
 /* ---- the hot path --------------------------------------------------------- */
 
-/* Routing layout (paper App. C, level 1).  topk_ids: device int32 [R,T,K].
+/* Routing layout (paper App. D, level 1).  topk_ids: device int32 [R,T,K].
  * Computes a stable counting sort of the items by expert id: dst_row[i] =
  * expert_offset[e_i] + #{j < i : e_j = e_i}, i.e. segments ordered by expert,
  * then source rank, then token, then slot, packed without padding.
@@ -198,7 +198,7 @@ strata_status strata_moe_layout_noalloc(const strata_moe_shape *shape, const int
                                         const strata_moe_layout_t *layout, int32_t *device_status,
                                         void *stream);
 
-/* Dispatch (paper Sec. 6.2 / 7.1).  x: device bf16 [R,T,H].
+/* Dispatch (paper Sec. 6.2 / 8.1).  x: device bf16 [R,T,H].
  * BF16:  recv is device bf16 [capacity_rows, H]; recv[dst_row[i], :] = x[n(i), :] bit for bit;
  *        recv_scale must be NULL.
  * FP8:   recv is device uint8 [capacity_rows, H], recv_scale device float [capacity_rows, H/128];
@@ -222,7 +222,7 @@ strata_status strata_moe_dispatch(strata_ctx *ctx, const strata_moe_layout_t *la
 strata_status strata_moe_combine(strata_ctx *ctx, const strata_moe_layout_t *layout, const void *y,
                                  size_t y_rows, const float *topk_w, void *out, void *stream);
 
-/* ---- optional: the paper's hierarchical workload partitioning (Sec. 6.2, App. B and C) -----------
+/* ---- optional: the paper's hierarchical workload partitioning (Sec. 6.2, App. B to D) -----------
  * The default dispatch balances at run time by ordered work claiming.  These two calls build and run
  * the paper's own static scheme instead, so that it can be compared on this hardware:
  *   expert windows  (source rank r, expert e): src_expert_count[r][e] contiguous receive rows starting

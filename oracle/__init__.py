@@ -178,7 +178,7 @@ def make_tiers(tiers) -> np.ndarray:
 
 def partition(lay: Dict[str, np.ndarray], row_bytes: int, n_cores: int, tiers, g0: int = 1, g1: int = 1,
               max_units: int = 1 << 16) -> Dict[str, np.ndarray]:
-    """Window partitioning + LPT-style list scheduling of dispatch (paper Sec. 6.2, App. B, C)."""
+    """Window partitioning + LPT-style list scheduling of dispatch (paper Sec. 6.2, App. B to D)."""
     sec = _c(lay["src_expert_count"], np.int32)
     R, E = sec.shape
     off = _c(lay["expert_offset"], np.int32)

@@ -9,10 +9,10 @@
  * the benchmark may call it.
  *
  * What it follows:
- *  - Routing metadata (paper App. C, "token placement"): destination expert,
+ *  - Routing metadata (paper App. D, "token placement"): destination expert,
  *    per-expert counts, prefix-sum offsets and token-local offsets, which
  *    dispatch and combine both reuse.
- *  - Dispatch (paper Sec. 6.2 / 7.1): each routed token's hidden vector is
+ *  - Dispatch (paper Sec. 6.2 / 8.1): each routed token's hidden vector is
  *    moved to the receive segment of the rank that owns its expert, directly
  *    into the user buffer (no staging copy).
  *  - Combine (paper Sec. 6.1, reduction-bearing operators): the top-k expert
@@ -383,7 +383,7 @@ void oracle_combine(int64_t n_tok, int32_t K, int32_t H,
 
 /* ------------------------------------------------------------------ */
 /* O5: hierarchical workload partitioning for dispatch (paper Sec. 6.2, */
-/* App. B and C).                                                       */
+/* App. B to D).                                                        */
 /*  level 2, expert-window aggregation: the rows that source rank r     */
 /*    sends to expert e form one contiguous window of the receive       */
 /*    buffer, win_base[r][e] .. + src_expert_count[r][e].               */

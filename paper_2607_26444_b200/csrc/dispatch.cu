@@ -1,4 +1,4 @@
-// Token dispatch (paper Sec. 6.2 / 7.1): every token's hidden vector goes to the K receive rows
+// Token dispatch (paper Sec. 6.2 / 8.1): every token's hidden vector goes to the K receive rows
 // the layout assigned, straight into the caller's (registered) receive buffer.
 //
 // Work split: a unit is one token (or one column chunk of a token when a row is larger than

@@ -1,4 +1,4 @@
-// Routing layout (paper App. C, level 1 "token placement"): per-expert counts, prefix-sum
+// Routing layout (paper App. D, level 1 "token placement"): per-expert counts, prefix-sum
 // offsets and token-local offsets, as a stable counting sort of the items by expert id.
 //
 // Batches of up to 32,768 items take one launch of one thread-block cluster (layout_cluster_kernel).

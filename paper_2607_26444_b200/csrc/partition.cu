@@ -1,4 +1,4 @@
-// Hierarchical workload partitioning for dispatch, the paper's own scheme (Sec. 6.2, App. B and C), as
+// Hierarchical workload partitioning for dispatch, the paper's own scheme (Sec. 6.2, App. B to D), as
 // an optional work-assignment variant next to the default ordered work claiming:
 //   level 2  expert-window aggregation: rows that source rank r sends to expert e are one contiguous
 //            window of the receive buffer (win_base[r][e], src_expert_count[r][e] rows);

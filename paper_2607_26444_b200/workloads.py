@@ -7,7 +7,7 @@ method's arithmetic (no layout, no scatter, no quantisation, no combine) and
 imports neither the CUDA binding nor the CPU oracle, so both sides can be fed
 the very same bytes.
 
-Shapes follow the paper's microbenchmark setting (Sec. 7.1: hidden 7168, top-8,
+Shapes follow the paper's microbenchmark setting (Sec. 8.1: hidden 7168, top-8,
 4096 tokens per batch) and its serving deployment (EP=16 decode); the expert
 counts and the FP8/skew variants are the build's own benchmark configurations.
 The paper's production routing traces are not available: uniform and Zipf

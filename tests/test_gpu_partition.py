@@ -1,4 +1,4 @@
-"""GPU-vs-oracle parity for the paper's window partitioning and LPT-style policy (Sec. 6.2, App. B, C),
+"""GPU-vs-oracle parity for the paper's window partitioning and LPT-style policy (Sec. 6.2, App. B to D),
 through the C ABI: every output array of the policy is integer work and must be bit-identical, and the
 window-major dispatch must write exactly what the oracle's (and the token-major) dispatch writes."""
 import numpy as np

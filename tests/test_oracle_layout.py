@@ -1,4 +1,4 @@
-"""Pins for the oracle's routing layout (paper App. C, token placement).
+"""Pins for the oracle's routing layout (paper App. D, token placement).
 
 None of these retype the oracle's counting sort: they use a comparison sort of
 (expert, rank, token, slot) tuples, a hand-worked example, closed forms and

@@ -1,4 +1,4 @@
-"""Pins for the oracle's hierarchical workload partitioning (paper Sec. 6.2, App. B and C):
+"""Pins for the oracle's hierarchical workload partitioning (paper Sec. 6.2, App. B to D):
 expert windows, peer windows, transfer units with cost alpha + s/beta, LPT-style list scheduling under
 a stripe-level fan-out cap.  None of these re-run the oracle's own greedy loop: they use hand-worked
 schedules (Graham's tight instances), a brute-force optimum, closed-form unit counts, and the
