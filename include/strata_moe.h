@@ -140,6 +140,52 @@ strata_status strata_ctx_launch_count(strata_ctx *ctx, uint64_t *count);
  * times is the load-balance evidence the paper reports per core (Sec. 9.6). */
 strata_status strata_ctx_set_trace(strata_ctx *ctx, uint64_t *dptr, size_t capacity_ctas);
 
+/* Per-CTA event timeline (the paper's in-kernel profiler, Sec. 6.4, manual mode: named begin/end probes
+ * at stage boundaries; every core appends time-stamped events to its own slice of a trace buffer, which
+ * is decoded into per-core timelines afterwards).
+ * buf: n_ctas slices of (1 + events_per_cta) uint64, owned by the caller, zeroed by the caller before
+ * use, and readable/writable by the GPU: device memory, or page-locked host memory (under unified
+ * addressing the kernels write it in place across PCIe, as the paper's cores write a host-pinned
+ * buffer).  Word 0 of slice b counts the events CTA b has recorded so far (events beyond
+ * events_per_cta are counted but not stored); the following words are events, appended by every launch
+ * on this context while the timeline is set, in stream order:
+ *   bits  0..47  GPU global timer, nanoseconds (low 48 bits)
+ *   bits 48..55  stage   (strata_stage)
+ *   bit  56      0 = begin, 1 = end
+ *   bits 57..63  kernel  (strata_kernel_id)
+ * One thread per CTA records; a probe costs one timer read and one 8-byte store, and nothing when the
+ * timeline is off (buf = NULL, the default).  CTAs with blockIdx >= n_ctas record nothing.
+ * Every probed kernel records its CTA lifetime (STRATA_STAGE_KERNEL).  Inside it, per unit of work: the
+ * bf16 dispatch and the collectives' copy kernel record WAIT_IN, WORK and WAIT_OUT; combine and the
+ * collectives' reduce kernel record WORK; the fp8 and the window-major dispatch record the lifetime only.
+ * The layout kernels are not probed. */
+typedef enum {
+    STRATA_STAGE_KERNEL = 0,     /* the CTA's lifetime inside one launch                        */
+    STRATA_STAGE_WAIT_IN = 1,    /* blocked until a unit's input has arrived in shared memory   */
+    STRATA_STAGE_WORK = 2,       /* issuing a unit's stores / computing a unit                  */
+    STRATA_STAGE_WAIT_OUT = 3    /* blocked until earlier stores have left shared memory        */
+} strata_stage;
+typedef enum {
+    STRATA_KERNEL_DISPATCH_BF16 = 1, STRATA_KERNEL_DISPATCH_FP8 = 2, STRATA_KERNEL_COMBINE = 3,
+    STRATA_KERNEL_DISPATCH_WINDOWS = 4, STRATA_KERNEL_SLICE_COPY = 5, STRATA_KERNEL_SLICE_REDUCE = 6
+} strata_kernel_id;
+strata_status strata_ctx_set_timeline(strata_ctx *ctx, uint64_t *buf, size_t n_ctas, size_t events_per_cta);
+
+/* One decoded interval of a timeline: CTA `cta` of kernel `kernel` spent [begin_ns, end_ns) in `stage`. */
+typedef struct {
+    uint32_t cta;
+    uint8_t kernel;              /* strata_kernel_id */
+    uint8_t stage;               /* strata_stage     */
+    uint16_t flags;              /* 1: a begin that was never closed; 2: an end without a begin (end_ns = begin_ns) */
+    uint64_t begin_ns, end_ns;   /* 48-bit timer values, made monotonic within the slice */
+} strata_span;
+/* Host-only: pairs the begin/end events of a timeline buffer (a HOST copy, same layout as above) into
+ * spans, slice by slice in event order; nested stages are allowed (a stack per slice).  Writes at most
+ * max_spans spans; *n_spans is the number found (> max_spans: call again with more room); *dropped is
+ * the number of events the kernels counted but could not store.  INVALID_ARG on NULL pointers. */
+strata_status strata_timeline_decode(const uint64_t *host_buf, size_t n_ctas, size_t events_per_cta,
+                                     strata_span *spans, size_t max_spans, size_t *n_spans, size_t *dropped);
+
 /* ---- pool: registration at allocation time ------------------------------
  * Analogue of the paper's registration-on-allocation (Sec. 5.1): a buffer is
  * registered once, when it is allocated (phase 1); every later operator call

@@ -39,6 +39,7 @@ EXPORTS = [
     "strata_moe_roundtrip_host", "strata_moe_layout_noalloc", "strata_ctx_set_trace",
     "strata_moe_partition_max_units", "strata_moe_partition", "strata_moe_dispatch_windows",
     "strata_moe_recv_rows",
+    "strata_ctx_set_timeline", "strata_timeline_decode",
     "strata_allgather", "strata_alltoall", "strata_broadcast", "strata_reducescatter", "strata_allreduce",
 ]
 
@@ -59,6 +60,16 @@ class strata_moe_layout_t(ctypes.Structure):
 class strata_moe_device_buffers(ctypes.Structure):
     _fields_ = [("ids", ctypes.c_void_p), ("x", ctypes.c_void_p), ("w", ctypes.c_void_p),
                 ("recv", ctypes.c_void_p), ("out", ctypes.c_void_p), ("layout", strata_moe_layout_t)]
+
+
+class strata_span(ctypes.Structure):
+    _fields_ = [("cta", ctypes.c_uint32), ("kernel", ctypes.c_uint8), ("stage", ctypes.c_uint8),
+                ("flags", ctypes.c_uint16), ("begin_ns", ctypes.c_uint64), ("end_ns", ctypes.c_uint64)]
+
+
+STAGE_NAMES = {0: "kernel", 1: "wait_in", 2: "work", 3: "wait_out"}
+KERNEL_NAMES = {1: "dispatch_bf16", 2: "dispatch_fp8", 3: "combine", 4: "dispatch_windows", 5: "slice_copy",
+                6: "slice_reduce"}
 
 
 class strata_tier(ctypes.Structure):
@@ -132,6 +143,8 @@ def lib() -> ctypes.CDLL:
         "strata_moe_partition": [vp, P(strata_moe_layout_t), P(strata_partition_policy), i32,
                                  P(strata_partition_t), sz, vp],
         "strata_moe_dispatch_windows": [vp, P(strata_moe_layout_t), P(strata_partition_t), i32, vp, vp, sz, vp],
+        "strata_ctx_set_timeline": [vp, vp, sz, sz],
+        "strata_timeline_decode": [vp, sz, sz, vp, sz, P(sz), P(sz)],
         "strata_allgather": [vp, i32, vp, vp, sz, vp],
         "strata_alltoall": [vp, i32, vp, vp, sz, vp],
         "strata_broadcast": [vp, i32, i32, vp, vp, sz, vp],
@@ -269,6 +282,84 @@ def strata_moe_dispatch_windows(ctx, layout: strata_moe_layout_t, partition: str
                                 x: int, recv: int, capacity_rows: int, stream: int) -> int:
     return lib().strata_moe_dispatch_windows(ctx, ctypes.byref(layout), ctypes.byref(partition), n_cores, x, recv,
                                              capacity_rows, stream)
+
+
+def strata_ctx_set_timeline(ctx, buf: Optional[int], n_ctas: int, events_per_cta: int) -> int:
+    return lib().strata_ctx_set_timeline(ctx, buf, n_ctas, events_per_cta)
+
+
+def strata_timeline_decode(host_buf: int, n_ctas: int, events_per_cta: int, spans: Optional[int],
+                           max_spans: int) -> Tuple[int, int, int]:
+    """Returns (status, spans found, events dropped); host_buf and spans are host addresses."""
+    n, lost = ctypes.c_size_t(), ctypes.c_size_t()
+    rc = lib().strata_timeline_decode(host_buf, n_ctas, events_per_cta, spans, max_spans, ctypes.byref(n),
+                                      ctypes.byref(lost))
+    return rc, n.value, lost.value
+
+
+def decode_timeline(buf):
+    """buf: numpy uint64 [n_ctas, 1 + events_per_cta] (a host copy of a timeline buffer).
+    Returns (spans, dropped): spans is a numpy structured array (cta, kernel, stage, flags, begin_ns, end_ns)."""
+    import numpy as np
+    buf = np.ascontiguousarray(buf, dtype=np.uint64)
+    n_ctas, width = buf.shape
+    dt = np.dtype([("cta", np.uint32), ("kernel", np.uint8), ("stage", np.uint8), ("flags", np.uint16),
+                   ("begin_ns", np.uint64), ("end_ns", np.uint64)], align=True)
+    assert dt.itemsize == ctypes.sizeof(strata_span)
+    rc, n, lost = strata_timeline_decode(buf.ctypes.data, n_ctas, width - 1, None, 0)
+    _check(rc, "strata_timeline_decode")
+    spans = np.zeros(n, dtype=dt)
+    rc, n2, lost = strata_timeline_decode(buf.ctypes.data, n_ctas, width - 1, spans.ctypes.data if n else None, n)
+    _check(rc, "strata_timeline_decode")
+    assert n2 == n
+    return spans, lost
+
+
+def timeline_summary(spans) -> dict:
+    """Per kernel: CTAs, wall time from the first begin to the last end, spread of the CTAs' finish times,
+    and per stage the number of intervals, their total time and its share of the CTAs' lifetimes."""
+    import numpy as np
+    out = {}
+    for k in np.unique(spans["kernel"]):
+        sk = spans[(spans["kernel"] == k) & (spans["flags"] == 0)]
+        life = sk[sk["stage"] == 0]
+        if life.size == 0:
+            continue
+        t0, t1 = int(life["begin_ns"].min()), int(life["end_ns"].max())
+        busy = float((life["end_ns"] - life["begin_ns"]).sum())
+        ent = {"ctas": int(np.unique(life["cta"]).size), "launches_per_cta": float(life.size) / np.unique(life["cta"]).size,
+               "wall_us": (t1 - t0) / 1e3,
+               "finish_spread": float(int(life["end_ns"].max()) - int(life["end_ns"].min())) / max(1, t1 - t0),
+               "stages": {}}
+        for st in np.unique(sk["stage"]):
+            if st == 0:
+                continue
+            ss = sk[sk["stage"] == st]
+            tot = float((ss["end_ns"] - ss["begin_ns"]).sum())
+            ent["stages"][STAGE_NAMES.get(int(st), str(int(st)))] = {
+                "intervals": int(ss.size), "total_us": tot / 1e3, "share_of_cta_time": tot / busy if busy else 0.0,
+                "mean_ns": tot / ss.size}
+        out[KERNEL_NAMES.get(int(k), str(int(k)))] = ent
+    return out
+
+
+def timeline_chrome_trace(spans, path: str, max_ctas: int = 64) -> int:
+    """Writes the spans of the first max_ctas CTAs as a Chrome trace-event JSON file (one process per
+    kernel, one thread per CTA, microseconds from the first event); returns the number of events written."""
+    import json
+    import numpy as np
+    sel = spans[(spans["cta"] < max_ctas) & (spans["flags"] == 0)]
+    if sel.size == 0:
+        with open(path, "w") as f:
+            json.dump({"traceEvents": []}, f)
+        return 0
+    t0 = int(sel["begin_ns"].min())
+    ev = [{"name": STAGE_NAMES.get(int(s["stage"]), str(int(s["stage"]))), "ph": "X",
+           "pid": KERNEL_NAMES.get(int(s["kernel"]), str(int(s["kernel"]))), "tid": int(s["cta"]),
+           "ts": (int(s["begin_ns"]) - t0) / 1e3, "dur": (int(s["end_ns"]) - int(s["begin_ns"])) / 1e3} for s in sel]
+    with open(path, "w") as f:
+        json.dump({"traceEvents": ev, "displayTimeUnit": "ns"}, f)
+    return len(ev)
 
 
 def strata_allgather(ctx, R: int, src: int, dst: int, bytes_per_rank: int, stream: int) -> int:
@@ -448,6 +539,30 @@ class MoEContext:
                 "finish_spread": float(end.max() - end.min()) / total,
                 "wait_in_share": float((used[:, 2] / busy).mean()),
                 "wait_out_share": float((used[:, 3] / busy).mean())}
+
+    def timeline(self, n_ctas: int = 2048, events_per_cta: int = 2048, pinned: bool = False):
+        """Turns the event timeline on; returns the zeroed buffer [n_ctas, 1 + events_per_cta] (int64), in
+        device memory or, with pinned=True, in page-locked host memory that the kernels write in place."""
+        import torch
+        if pinned:
+            t = torch.zeros((n_ctas, 1 + events_per_cta), dtype=torch.int64, pin_memory=True)
+        else:
+            t = torch.zeros((n_ctas, 1 + events_per_cta), dtype=torch.int64, device=self.device)
+        torch.cuda.synchronize(self.device)
+        _check(strata_ctx_set_timeline(self.h, t.data_ptr(), n_ctas, events_per_cta), "strata_ctx_set_timeline")
+        self._timeline = t
+        return t
+
+    def timeline_off(self) -> None:
+        _check(strata_ctx_set_timeline(self.h, None, 0, 0), "strata_ctx_set_timeline")
+        self._timeline = None
+
+    @staticmethod
+    def timeline_spans(t):
+        """Synchronises and decodes a timeline buffer; returns (spans, dropped)."""
+        import torch
+        torch.cuda.synchronize()
+        return decode_timeline(t.cpu().numpy().view("uint64"))
 
     def trace_off(self) -> None:
         _check(strata_ctx_set_trace(self.h, None, 0), "strata_ctx_set_trace")

@@ -164,7 +164,7 @@ strata_status strata_ctx_create(strata_ctx** out, const strata_moe_shape* shape,
     c->ws_bytes = 0;
     c->next_region = 1;
     c->launches = 0;
-    c->trace = strata::TraceBuf{nullptr, 0};
+    c->trace = strata::TraceBuf{nullptr, 0, nullptr, 0, 0};
     *out = c;
     return STRATA_OK;
 }
@@ -242,6 +242,65 @@ strata_status strata_ctx_set_trace(strata_ctx* ctx, uint64_t* dptr, size_t capac
     std::lock_guard<std::mutex> lk(ctx->mu);
     ctx->trace.slots = reinterpret_cast<unsigned long long*>(dptr);
     ctx->trace.capacity = dptr ? (int)capacity_ctas : 0;
+    return STRATA_OK;
+}
+
+strata_status strata_ctx_set_timeline(strata_ctx* ctx, uint64_t* buf, size_t n_ctas, size_t events_per_cta)
+{
+    if (!ctx) return STRATA_ERR_INVALID_ARG;
+    if (buf && (reinterpret_cast<uintptr_t>(buf) & 7u) != 0) return STRATA_ERR_ALIGNMENT;
+    if (buf && (n_ctas == 0 || n_ctas > (size_t)1 << 24 || events_per_cta == 0 || events_per_cta > (size_t)1 << 24))
+        return STRATA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(ctx->mu);
+    ctx->trace.tl = reinterpret_cast<unsigned long long*>(buf);
+    ctx->trace.tl_ctas = buf ? (int)n_ctas : 0;
+    ctx->trace.tl_cap = buf ? (int)events_per_cta : 0;
+    return STRATA_OK;
+}
+
+strata_status strata_timeline_decode(const uint64_t* host_buf, size_t n_ctas, size_t events_per_cta,
+                                     strata_span* spans, size_t max_spans, size_t* n_spans, size_t* dropped)
+{
+    if (!host_buf || !n_spans || !dropped || (!spans && max_spans > 0)) return STRATA_ERR_INVALID_ARG;
+    size_t found = 0, lost = 0;
+    struct Open { uint8_t kernel, stage; uint64_t t; };
+    std::vector<Open> stack;
+    auto emit = [&](uint32_t cta, uint8_t kernel, uint8_t stage, uint16_t flags, uint64_t b, uint64_t e) {
+        if (found < max_spans) spans[found] = strata_span{cta, kernel, stage, flags, b, e};
+        ++found;
+    };
+    for (size_t b = 0; b < n_ctas; ++b) {
+        const uint64_t* slice = host_buf + b * (events_per_cta + 1);
+        const uint64_t counted = slice[0];
+        const size_t n = counted < events_per_cta ? (size_t)counted : events_per_cta;
+        lost += (size_t)(counted - n);
+        stack.clear();
+        uint64_t wraps = 0, prev = 0;
+        for (size_t i = 0; i < n; ++i) {
+            const uint64_t ev = slice[1 + i];
+            uint64_t t = ev & 0xffffffffffffull;
+            if (i > 0 && t + wraps < prev && prev - (t + wraps) > (1ull << 47)) wraps += 1ull << 48;   // timer wrapped
+            t += wraps;
+            prev = t;
+            const uint8_t stage = (uint8_t)((ev >> 48) & 0xff), kernel = (uint8_t)(ev >> 57);
+            if (((ev >> 56) & 1) == 0) {
+                stack.push_back(Open{kernel, stage, t});
+                continue;
+            }
+            // an end closes the innermost open begin of the same kernel and stage
+            size_t k = stack.size();
+            while (k > 0 && !(stack[k - 1].kernel == kernel && stack[k - 1].stage == stage)) --k;
+            if (k == 0) {
+                emit((uint32_t)b, kernel, stage, 2, t, t);           // an end without a begin
+                continue;
+            }
+            emit((uint32_t)b, kernel, stage, 0, stack[k - 1].t, t);
+            stack.erase(stack.begin() + (long)(k - 1));
+        }
+        for (const Open& o : stack) emit((uint32_t)b, o.kernel, o.stage, 1, o.t, o.t);   // never closed
+    }
+    *n_spans = found;
+    *dropped = lost;
     return STRATA_OK;
 }
 
@@ -695,10 +754,10 @@ strata_status strata_moe_roundtrip_host(strata_ctx* ctx, const strata_moe_device
             cq = combine_queue(ctx);
         }
         cudaError_t err = launch_dispatch_bf16(sub, dev->layout.dst_row + a * s.K, dx + a * row_bytes, dev->recv, n_recv,
-                                               ctx->ws, dq, ctx->n_sm, TraceBuf{nullptr, 0}, st);
+                                               ctx->ws, dq, ctx->n_sm, TraceBuf{nullptr, 0, nullptr, 0, 0}, st);
         if (err == cudaSuccess)
             err = launch_combine(sub, dev->layout.dst_row + a * s.K, dev->recv, n_recv, dev->w + a * s.K,
-                                 dout + a * row_bytes, ctx->ws, cq, ctx->n_sm, TraceBuf{nullptr, 0}, st);
+                                 dout + a * row_bytes, ctx->ws, cq, ctx->n_sm, TraceBuf{nullptr, 0, nullptr, 0, 0}, st);
         {
             std::lock_guard<std::mutex> lk(ctx->mu);
             ctx->launches += 2;

@@ -66,6 +66,8 @@ __global__ void __launch_bounds__(32) slice_copy_kernel(CopyParams p)
     const uint64_t pol = policy_evict_first();
     griddep_wait();
     if (lane == 0) trace_begin(p.trace);
+    Timeline tl(p.trace, STRATA_KERNEL_SLICE_COPY, lane == 0);
+    tl.begin(STRATA_STAGE_KERNEL);
 
     auto decode = [&](unsigned int u, unsigned int& slice, unsigned long long& off, uint32_t& bytes, int& f0) {
         const unsigned int c = u / p.fan_groups;               // chunk index over all slices
@@ -113,7 +115,9 @@ __global__ void __launch_bounds__(32) slice_copy_kernel(CopyParams p)
         const unsigned int u = s_unit[s];
         if (u == kNoUnit) break;
         wait_in.begin();
+        tl.begin(STRATA_STAGE_WAIT_IN);
         ok = mbar_wait_bounded(&bars[s], parity);
+        tl.end(STRATA_STAGE_WAIT_IN);
         wait_in.end();
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -123,12 +127,16 @@ __global__ void __launch_bounds__(32) slice_copy_kernel(CopyParams p)
             uint32_t bytes;
             int f0;
             decode(u, slice, off, bytes, f0);
+            tl.begin(STRATA_STAGE_WORK);
             unsigned char* dst = p.out + (size_t)(slice / p.inner) * p.stride_a + (size_t)(slice % p.inner) * p.stride_b + off;
             const int f1 = min(p.fan, f0 + (int)p.fan_per_group);
             for (int f = f0; f < f1; ++f) bulk_s2g(dst + (size_t)f * p.fan_stride, smem + (size_t)s * kCopyChunkBytes, bytes);
             bulk_commit();
+            tl.end(STRATA_STAGE_WORK);
             wait_out.begin();
+            tl.begin(STRATA_STAGE_WAIT_OUT);
             bulk_wait_read<1>();           // the stage refilled next held unit j-1: its stores have left shared memory
+            tl.end(STRATA_STAGE_WAIT_OUT);
             wait_out.end();
             issue_load(j + kCopyStages - 1);
         }
@@ -137,9 +145,13 @@ __global__ void __launch_bounds__(32) slice_copy_kernel(CopyParams p)
     if (lane == 0) {
         if (!ok) report_status(p.status, STRATA_ERR_TIMEOUT);
         wait_out.begin();
+        tl.begin(STRATA_STAGE_WAIT_OUT);
         bulk_wait_read<0>();
+        tl.end(STRATA_STAGE_WAIT_OUT);
         wait_out.end();
         trace_end(p.trace, wait_in.total, wait_out.total);
+        tl.end(STRATA_STAGE_KERNEL);
+        tl.finish();
     }
 }
 
@@ -186,10 +198,13 @@ __global__ void __launch_bounds__(kReduceThreads) slice_reduce_kernel(ReducePara
     __shared__ unsigned int s_next[2];
     griddep_wait();
     if (tid == 0) trace_begin(p.trace);
+    Timeline tl(p.trace, STRATA_KERNEL_SLICE_REDUCE, tid == 0);
+    tl.begin(STRATA_STAGE_KERNEL);
 
     unsigned int u = blockIdx.x < p.n_units ? blockIdx.x : kNoUnit;
     bool exhausted = false;
     for (int j = 0; u != kNoUnit; ++j) {
+        tl.begin(STRATA_STAGE_WORK);
         if (tid == 0) {
             const unsigned int nx = claim_unit(p.wq, p.n_units, gridDim.x, exhausted);
             s_next[j & 1] = nx;
@@ -218,9 +233,14 @@ __global__ void __launch_bounds__(kReduceThreads) slice_reduce_kernel(ReducePara
             for (int f = 0; f < p.fan; ++f) st_stream16(dst + (size_t)f * p.fan_stride, o);
         }
         __syncthreads();
+        tl.end(STRATA_STAGE_WORK);
         u = s_next[j & 1];
     }
-    if (tid == 0) trace_end(p.trace);
+    if (tid == 0) {
+        trace_end(p.trace);
+        tl.end(STRATA_STAGE_KERNEL);
+        tl.finish();
+    }
 }
 
 constexpr size_t kCopySmem = (size_t)kCopyStages * kCopyChunkBytes + kCopyStages * sizeof(uint64_t) + kCopyStages * sizeof(unsigned int) + 16;

@@ -75,10 +75,13 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
     __shared__ unsigned int s_next[2];             // the claim made during unit j is read for unit j+1
     griddep_wait();
     if (tid == 0) trace_begin(p.trace);
+    Timeline tl(p.trace, STRATA_KERNEL_COMBINE, tid == 0);
+    tl.begin(STRATA_STAGE_KERNEL);
 
     unsigned int u = blockIdx.x < n_units ? blockIdx.x : kNoUnit;
     bool exhausted = false;                        // thread 0's view of the queue
     for (int j = 0; u != kNoUnit; ++j) {
+        tl.begin(STRATA_STAGE_WORK);
         if (tid == 0) {
             const unsigned int nx = claim_unit(p.wq, n_units, gridDim.x, exhausted);
             s_next[j & 1] = nx;
@@ -115,10 +118,13 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
             st_stream16(dst + (size_t)v * 16, o);
         }
         __syncthreads();                           // one barrier per unit: publishes the next claim
+        tl.end(STRATA_STAGE_WORK);
         u = s_next[j & 1];
     }
     if (tid == 0) {
         trace_end(p.trace);
+        tl.end(STRATA_STAGE_KERNEL);
+        tl.finish();
     }
 }
 
@@ -135,6 +141,8 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel<0>(CombinePara
     __shared__ unsigned int s_tok;
     griddep_wait();
     if (tid == 0) trace_begin(p.trace);
+    Timeline tl(p.trace, STRATA_KERNEL_COMBINE, tid == 0);
+    tl.begin(STRATA_STAGE_KERNEL);
 
     bool exhausted = false;
     for (int j = 0;; ++j) {
@@ -144,6 +152,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel<0>(CombinePara
         __syncthreads();
         const unsigned int n = s_tok;
         if (n == kNoUnit) break;
+        tl.begin(STRATA_STAGE_WORK);
         if (tid < K) {
             const int row = p.dst_row[(long long)n * K + tid];
             const bool row_ok = row >= 0 && row < p.y_rows;
@@ -173,9 +182,12 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel<0>(CombinePara
             o.w = pack_bf16x2(a[6], a[7]);
             st_stream16(dst + (size_t)v * 16, o);
         }
+        tl.end(STRATA_STAGE_WORK);
     }
     if (tid == 0) {
         trace_end(p.trace);
+        tl.end(STRATA_STAGE_KERNEL);
+        tl.finish();
     }
 }
 

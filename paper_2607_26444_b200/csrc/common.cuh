@@ -58,6 +58,10 @@ constexpr unsigned int kNoUnit = 0xffffffffu;
 struct TraceBuf {
     unsigned long long* slots;   // device, [capacity][4] = {start_ns, end_ns, wait_in_ns, wait_out_ns}; nullptr = off
     int capacity;
+    // event timeline: tl_ctas slices of (1 + tl_cap) words, word 0 = events recorded so far; nullptr = off
+    unsigned long long* tl;
+    int tl_ctas;
+    int tl_cap;
 };
 
 // ---- launchers (defined next to their kernels) -----------------------------
@@ -207,6 +211,36 @@ struct StageClock {
     __device__ explicit StageClock(const TraceBuf& t) : on(t.slots != nullptr), t0(0), total(0) {}
     __device__ __forceinline__ void begin() { if (on) t0 = global_timer_ns(); }
     __device__ __forceinline__ void end() { if (on) total += global_timer_ns() - t0; }
+};
+
+// Event timeline (paper Sec. 6.4, manual probes).  One thread per CTA owns the writer; construct it
+// after griddep_wait(), so that the event count left by the previous launch is visible.
+struct Timeline {
+    unsigned long long* slice;
+    unsigned int n, cap, kernel;
+    __device__ Timeline(const TraceBuf& t, unsigned int kernel_id, bool owner)
+        : slice(nullptr), n(0), cap(0), kernel(kernel_id)
+    {
+        if (owner && t.tl && (int)blockIdx.x < t.tl_ctas) {
+            slice = t.tl + (size_t)blockIdx.x * (size_t)(t.tl_cap + 1);
+            n = (unsigned int)*reinterpret_cast<volatile unsigned long long*>(slice);
+            cap = (unsigned int)t.tl_cap;
+        }
+    }
+    __device__ __forceinline__ void mark(unsigned int stage, unsigned int is_end)
+    {
+        if (!slice) return;
+        if (n < cap)
+            slice[1 + n] = (global_timer_ns() & 0xffffffffffffull) | ((unsigned long long)(stage & 0xffu) << 48) |
+                           ((unsigned long long)(is_end & 1u) << 56) | ((unsigned long long)(kernel & 0x7fu) << 57);
+        ++n;
+    }
+    __device__ __forceinline__ void begin(unsigned int stage) { mark(stage, 0); }
+    __device__ __forceinline__ void end(unsigned int stage) { mark(stage, 1); }
+    __device__ __forceinline__ void finish()
+    {
+        if (slice) slice[0] = n;
+    }
 };
 
 // One thread per CTA claims; returns kNoUnit when the queue is exhausted.  Units below `base` were

@@ -82,6 +82,8 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
     const uint64_t pol = policy_evict_first();
     griddep_wait();                       // x and dst_row belong to earlier kernels in the stream
     if (lane == 0) trace_begin(p.trace);
+    Timeline tl(p.trace, STRATA_KERNEL_DISPATCH_BF16, lane == 0);
+    tl.begin(STRATA_STAGE_KERNEL);
 
     auto decode = [&](unsigned int u, long long& tok, uint32_t& col0, uint32_t& bytes) {
         tok = u / (unsigned int)p.chunks_per_row;
@@ -135,11 +137,14 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
         if (!row_ok && my_row != -1) report_status(p.status, STRATA_ERR_BAD_ROW);
 
         wait_in.begin();
+        tl.begin(STRATA_STAGE_WAIT_IN);
         ok = mbar_wait_bounded(&bars[s], parity);
+        tl.end(STRATA_STAGE_WAIT_IN);
         wait_in.end();
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
 
+        tl.begin(STRATA_STAGE_WORK);
         for (int k = 0; k < p.K; ++k) {
             const int row = __shfl_sync(0xffffffffu, my_row, k);
             if (lane == 0 && row >= 0 && row < p.capacity_rows) {
@@ -153,9 +158,12 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
         }
         if (lane == 0) {
             bulk_commit();
+            tl.end(STRATA_STAGE_WORK);
             // The stage that unit j-1 used is refilled next; its stores must have left shared memory.
             wait_out.begin();
+            tl.begin(STRATA_STAGE_WAIT_OUT);
             bulk_wait_read<1>();
+            tl.end(STRATA_STAGE_WAIT_OUT);
             wait_out.end();
             issue_load(j + kBf16Stages - 1);
         }
@@ -164,9 +172,13 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
     if (lane == 0) {
         if (!ok) report_status(p.status, STRATA_ERR_TIMEOUT);
         wait_out.begin();
+        tl.begin(STRATA_STAGE_WAIT_OUT);
         bulk_wait_read<0>();
+        tl.end(STRATA_STAGE_WAIT_OUT);
         wait_out.end();
         trace_end(p.trace, wait_in.total, wait_out.total);
+        tl.end(STRATA_STAGE_KERNEL);
+        tl.finish();
     }
 }
 
@@ -208,6 +220,8 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
     const uint64_t pol = policy_evict_first();
     griddep_wait();
     if (tid == 0) trace_begin(p.trace);
+    Timeline tl(p.trace, STRATA_KERNEL_DISPATCH_FP8, tid == 0);
+    tl.begin(STRATA_STAGE_KERNEL);
 
     auto decode = [&](unsigned int u, long long& tok, uint32_t& col0, uint32_t& cols) {
         tok = u / (unsigned int)p.chunks_per_row;
@@ -316,6 +330,8 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
         if (!ok) report_status(p.status, STRATA_ERR_TIMEOUT);
         bulk_wait_read<0>();
         trace_end(p.trace);
+        tl.end(STRATA_STAGE_KERNEL);
+        tl.finish();
     }
 }
 

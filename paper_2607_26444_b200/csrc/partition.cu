@@ -373,6 +373,8 @@ __global__ void __launch_bounds__(32) dispatch_windows_kernel(WindowsParams p)
     griddep_wait();
     griddep_launch_dependents();
     if (lane == 0) trace_begin(p.trace);
+    Timeline tl(p.trace, STRATA_KERNEL_DISPATCH_WINDOWS, lane == 0);
+    tl.begin(STRATA_STAGE_KERNEL);
 
     // lane 0 only: store the oldest loaded row
     long long issued = 0, stored = 0;
@@ -460,6 +462,8 @@ __global__ void __launch_bounds__(32) dispatch_windows_kernel(WindowsParams p)
         if (!ok) report_status(p.status, STRATA_ERR_TIMEOUT);
         bulk_wait_read<0>();
         trace_end(p.trace);
+        tl.end(STRATA_STAGE_KERNEL);
+        tl.finish();
     }
 }
 
