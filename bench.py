@@ -413,6 +413,35 @@ def window_partitioning_report(cfg: wl.MoEConfig, dev_index: int, unit_rows: int
     return out
 
 
+def timeline_report(cfg: wl.MoEConfig, dev_index: int, trace_path: str = "", pinned: bool = False):
+    """One step with the in-kernel event timeline on (paper Sec. 6.4): per kernel the CTA count, wall time,
+    finish-time spread and the share of CTA time per stage.  Probes cost time: these are not bench numbers."""
+    case = DeviceCase(cfg, dev_index)
+    torch, B = case.torch, case.B
+    for _ in range(3):
+        case.step()
+    torch.cuda.synchronize()
+    units = cfg.n_tok * max(1, -(-cfg.H * 2 // 16384))
+    cap = 16 + 8 * (units // (2 * 148) + 64)                 # 6 events per dispatch unit, with room to spare
+    t = case.ctx.timeline(n_ctas=2048, events_per_cta=cap, pinned=pinned)
+    case.step()
+    spans, dropped = case.ctx.timeline_spans(t)
+    case.ctx.timeline_off()
+    case.check()
+    rep = {"workload": cfg.name, "buffer": "pinned host" if pinned else "device", "events_per_cta": cap,
+           "spans": int(spans.size), "events_dropped": int(dropped), "kernels": B.timeline_summary(spans)}
+    for k in rep["kernels"].values():
+        k["wall_us"] = round(k["wall_us"], 2)
+        k["finish_spread"] = round(k["finish_spread"], 4)
+        for st in k["stages"].values():
+            st["total_us"] = round(st["total_us"], 1)
+            st["share_of_cta_time"] = round(st["share_of_cta_time"], 4)
+            st["mean_ns"] = round(st["mean_ns"], 1)
+    if trace_path:
+        rep["chrome_trace_events"] = B.timeline_chrome_trace(spans, trace_path, max_ctas=32)
+    return rep
+
+
 COLLECTIVE_OPS = ("allgather", "alltoall", "broadcast", "reducescatter", "allreduce")
 
 
@@ -707,6 +736,10 @@ def main():
     ap.add_argument("--workload", default="prefill", choices=wl.CONFIG_ORDER,
                     help="configuration to step through (the bench line is quoted on the default)")
     ap.add_argument("--tokens-per-rank", type=int, default=0, help="shrink T (profiling captures only)")
+    ap.add_argument("--timeline", action="store_true",
+                    help="print only the in-kernel timeline summary of one step of --workload (not the bench line)")
+    ap.add_argument("--timeline-trace", default="", help="also write a Chrome trace-event file of the first 32 CTAs")
+    ap.add_argument("--timeline-pinned", action="store_true", help="kernels write the events into pinned host memory")
     ap.add_argument("--collectives", action="store_true",
                     help="print only the report on the full-mesh collectives (one JSON object; not the bench line)")
     ap.add_argument("--collective-kib", type=int, nargs="+", default=[64, 1024, 16384], help="payload per rank, KiB")
@@ -724,6 +757,13 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.timeline:
+        if rank == 0:
+            cfg = wl.CONFIGS[args.workload]
+            if args.tokens_per_rank:
+                cfg = wl.shrink(cfg, T=args.tokens_per_rank)
+            print(json.dumps(timeline_report(cfg, local_rank, args.timeline_trace, args.timeline_pinned)), flush=True)
         return
     if args.collectives:
         if rank == 0:
