@@ -53,6 +53,10 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).argtypes = [i32, i64, vp, vp]
         L.oracle_broadcast.restype = None
         L.oracle_broadcast.argtypes = [i32, i32, i64, vp, vp]
+        L.oracle_alltoallv.restype = i64
+        L.oracle_alltoallv.argtypes = [i32, i64, i64, vp, vp, vp, vp, vp]
+        L.oracle_p2p.restype = None
+        L.oracle_p2p.argtypes = [i32, i32, i64, vp, vp]
         L.oracle_max_threads.restype = i32
         L.oracle_max_threads.argtypes = []
         _lib = L
@@ -265,3 +269,20 @@ def allreduce(x: np.ndarray) -> np.ndarray:
     out = np.empty((R, M), np.uint16)
     lib().oracle_allreduce(R, M, _p(x), _p(out))
     return out
+
+
+def alltoallv(x: np.ndarray, out: np.ndarray, send_bytes, send_off, recv_off) -> int:
+    """x uint8 [R, in_stride]; out uint8 [R, out_stride] is updated in place: rank p's send_bytes[p, r] bytes at
+    x[p, send_off[p, r]:] land at out[r, recv_off[r, p]:].  Returns the number of pairs skipped for not fitting."""
+    x = _c(x, np.uint8)
+    assert out.dtype == np.uint8 and out.flags.c_contiguous
+    R = x.shape[0]
+    sb, so, ro = (_c(a, np.int64).reshape(R, R) for a in (send_bytes, send_off, recv_off))
+    return int(lib().oracle_alltoallv(R, x.shape[1], out.shape[1], _p(x), _p(out), _p(sb), _p(so), _p(ro)))
+
+
+def p2p(x: np.ndarray, out: np.ndarray, src: int, dst: int) -> None:
+    """x, out uint8 [R, M]: out[dst] = x[src]; the other parts of out are left alone."""
+    x = _c(x, np.uint8)
+    assert out.dtype == np.uint8 and out.flags.c_contiguous and out.shape == x.shape
+    lib().oracle_p2p(src, dst, x.shape[1], _p(x), _p(out))

@@ -35,7 +35,9 @@
  * For the full-mesh collectives (tests/test_oracle_collectives.py): counter
  * patterns with closed-form results, the involution of all-to-all, exact
  * integer sums, a hand-worked order-sensitive sum, all-reduce = reduce-scatter
- * followed by all-gather, and an fp64 bound.
+ * followed by all-gather, and an fp64 bound; all-to-all-v: equal counts reduce
+ * to all-to-all, a hand-worked example, the reverse exchange restores the
+ * input, bytes nobody addresses stay untouched.
  * No function here is "parity unpinned".
  *
  * Index convention: rank r in [0,R), token t in [0,T), slot k in [0,K),
@@ -595,6 +597,36 @@ void oracle_allreduce(int32_t R, int64_t M, const uint16_t *in, uint16_t *out)
                 acc = acc + bf16_to_f32(in[(size_t)p * M + j]);
             out[(size_t)r * M + j] = f32_to_bf16_rne(acc);
         }
+}
+
+/* all-to-all-v and point-to-point (paper Sec. 6.1 names both; Sec. 6.2 names all-to-all-v as   */
+/* the operator whose peers exchange different volumes).  Byte counts and offsets per (sender,   */
+/* receiver) pair, MPI style:                                                                    */
+/*   rank p sends send_bytes[p][r] bytes, found at in[p] + send_off[p][r], to rank r, where     */
+/*   they land at out[r] + recv_off[r][p].  Bytes of out that no pair addresses are left alone.  */
+/* Returns the number of pairs that do not fit their buffers (those are skipped).               */
+int64_t oracle_alltoallv(int32_t R, int64_t in_stride, int64_t out_stride, const uint8_t *in, uint8_t *out,
+                         const int64_t *send_bytes, const int64_t *send_off, const int64_t *recv_off)
+{
+    int64_t bad = 0;
+    for (int32_t p = 0; p < R; ++p)
+        for (int32_t r = 0; r < R; ++r) {
+            const int64_t n = send_bytes[(size_t)p * R + r];
+            const int64_t so = send_off[(size_t)p * R + r], ro = recv_off[(size_t)r * R + p];
+            if (n == 0) continue;
+            if (n < 0 || so < 0 || ro < 0 || so + n > in_stride || ro + n > out_stride) {
+                ++bad;
+                continue;
+            }
+            for (int64_t j = 0; j < n; ++j)
+                out[(size_t)r * out_stride + ro + j] = in[(size_t)p * in_stride + so + j];
+        }
+    return bad;
+}
+
+void oracle_p2p(int32_t src, int32_t dst, int64_t M, const uint8_t *in, uint8_t *out)
+{
+    for (int64_t j = 0; j < M; ++j) out[(size_t)dst * M + j] = in[(size_t)src * M + j];
 }
 
 int32_t oracle_max_threads(void)

@@ -190,6 +190,30 @@ def gen_payload(R: int, elems_per_rank: int, seed: int) -> np.ndarray:
     return out
 
 
+def gen_pair_bytes(R: int, mean_bytes: int, seed: int, skew: float = 1.2, zero_frac: float = 0.1) -> np.ndarray:
+    """int64 [R, R]: bytes rank p sends to rank r in an uneven all-to-all, multiples of 16.
+
+    Receiver popularity follows a Zipf(skew) law over a seeded permutation (the shape of the MoE skew
+    workload), each pair is jittered by a uniform factor in [0.5, 1.5), and a fraction of the pairs is empty."""
+    rng = _rng(seed, 8)
+    pop = 1.0 / np.arange(1, R + 1, dtype=np.float64) ** skew
+    pop = pop[rng.permutation(R)] / pop.mean()
+    size = mean_bytes * pop[None, :] * rng.uniform(0.5, 1.5, size=(R, R))
+    size[rng.uniform(size=(R, R)) < zero_frac] = 0.0
+    return (np.floor(size / 16.0).astype(np.int64)) * 16
+
+
+def packed_offsets(pair_bytes: np.ndarray):
+    """(send_off [R, R], recv_off [R, R], in_stride, out_stride) for back-to-back packing: rank p's slices lie in
+    receiver order in its input, rank r's in sender order in its output."""
+    send_off = np.cumsum(pair_bytes, axis=1) - pair_bytes
+    recv = pair_bytes.T                                   # recv[r, p] = bytes r gets from p
+    recv_off = np.cumsum(recv, axis=1) - recv
+    in_stride = int(max(16, pair_bytes.sum(axis=1).max()))
+    out_stride = int(max(16, recv.sum(axis=1).max()))
+    return send_off.astype(np.int64), recv_off.astype(np.int64), in_stride, out_stride
+
+
 def generate(cfg: MoEConfig) -> Dict[str, np.ndarray]:
     return {"ids": gen_topk_ids(cfg), "x": gen_x(cfg), "w": gen_gate_weights(cfg)}
 

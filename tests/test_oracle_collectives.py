@@ -135,3 +135,91 @@ def test_single_rank_reduction_returns_the_input_as_values():
     x[0, 0] = 0x8000                                           # +0 + (-0) = +0
     out = oracle.allreduce(x)
     assert out[0, 0] == 0 and np.array_equal(out[0, 1:], x[0, 1:])
+
+
+# ---- all-to-all-v and point-to-point -----------------------------------------------------------
+
+def _v_golden():
+    path = os.path.join(os.path.dirname(__file__), "golden", "alltoallv_worked_example.txt")
+    d = {}
+    for line in open(path):
+        t = line.split()
+        if t and not t[0].startswith("#"):
+            d[t[0]] = [int(v) for v in t[1:]]
+    return d
+
+
+def test_alltoallv_worked_example():
+    d = _v_golden()
+    R, si, so = d["R"][0], d["in_stride"][0], d["out_stride"][0]
+    x = (np.arange(R)[:, None] * 16 + np.arange(si)[None, :]).astype(np.uint8)
+    out = np.full((R, so), 255, np.uint8)
+    bad = oracle.alltoallv(x, out, d["send_bytes"], d["send_off"], d["recv_off"])
+    assert bad == 0
+    for r in range(R):
+        assert out[r].tolist() == d[f"out{r}"], r
+
+
+def test_alltoallv_with_equal_counts_is_alltoall():
+    R, S = 5, 48
+    x = _bytes(R, R * S, 31)
+    sb = np.full((R, R), S, np.int64)
+    off = np.tile(np.arange(R) * S, (R, 1)).astype(np.int64)
+    out = np.zeros((R, R * S), np.uint8)
+    assert oracle.alltoallv(x, out, sb, off, off) == 0
+    assert np.array_equal(out.reshape(R, R, S), oracle.alltoall(x.reshape(R, R, S)))
+
+
+def test_alltoallv_reverse_exchange_restores_the_input_and_leaves_gaps_alone():
+    R = 6
+    sb = wl.gen_pair_bytes(R, 160, seed=4)
+    so, ro, si, st = wl.packed_offsets(sb)
+    so += 16                                                   # a 16-byte gap in front of every rank's data
+    ro += 32
+    si, st = si + 48, st + 64
+    x = _bytes(R, si, 32)
+    out = np.full((R, st), 0xEE, np.uint8)
+    assert oracle.alltoallv(x, out, sb, so, ro) == 0
+    # conservation: every rank received exactly the bytes addressed to it, the rest is untouched
+    touched = np.zeros((R, st), bool)
+    for r in range(R):
+        for p in range(R):
+            touched[r, ro[r, p]:ro[r, p] + sb[p, r]] = True
+    assert touched.sum() == sb.sum() and np.all(out[~touched] == 0xEE)
+    # the reverse exchange: receivers send back what they got, from where it landed to where it came from
+    back = np.full((R, si), 0x11, np.uint8)
+    assert oracle.alltoallv(out, back, sb.T.copy(), ro, so) == 0
+    sent = np.zeros((R, si), bool)
+    for p in range(R):
+        for r in range(R):
+            sent[p, so[p, r]:so[p, r] + sb[p, r]] = True
+    assert np.array_equal(back[sent], x[sent]) and np.all(back[~sent] == 0x11)
+
+
+def test_alltoallv_skips_pairs_that_do_not_fit():
+    R = 2
+    x = _bytes(R, 64, 33)
+    out = np.zeros((R, 64), np.uint8)
+    sb = np.array([[16, 32], [0, 16]], np.int64)
+    so = np.array([[0, 48], [0, 0]], np.int64)                 # 48 + 32 > 64: pair (0 -> 1) is skipped
+    ro = np.array([[0, 0], [16, 0]], np.int64)
+    assert oracle.alltoallv(x, out, sb, so, ro) == 1
+    assert np.array_equal(out[0, :16], x[0, :16]) and np.array_equal(out[1, :16], x[1, :16])
+    assert np.all(out[1, 16:] == 0)
+
+
+def test_p2p_copies_one_part():
+    x = _bytes(4, 80, 34)
+    out = np.full((4, 80), 7, np.uint8)
+    oracle.p2p(x, out, 2, 0)
+    assert np.array_equal(out[0], x[2]) and np.all(out[1:] == 7)
+
+
+def test_pair_bytes_recipe():
+    sb = wl.gen_pair_bytes(32, 1 << 20, seed=1)
+    assert sb.shape == (32, 32) and np.all(sb % 16 == 0) and (sb == 0).mean() > 0.03
+    col = sb.sum(axis=0)
+    assert col.max() > 5 * np.median(col)                      # a few hot receivers
+    so, ro, si, st = wl.packed_offsets(sb)
+    assert np.all(so[:, 0] == 0) and np.all(np.diff(so, axis=1) == sb[:, :-1])
+    assert si == sb.sum(axis=1).max() and st == sb.sum(axis=0).max()
