@@ -442,7 +442,7 @@ def timeline_report(cfg: wl.MoEConfig, dev_index: int, trace_path: str = "", pin
     return rep
 
 
-COLLECTIVE_OPS = ("allgather", "alltoall", "broadcast", "reducescatter", "allreduce")
+COLLECTIVE_OPS = ("allgather", "alltoall", "alltoallv", "broadcast", "reducescatter", "allreduce")
 
 
 def collectives_report(dev_index: int, R: int = 32, per_rank_kib=(64, 1024, 16384), iters: int = 10,
@@ -473,6 +473,14 @@ def collectives_report(dev_index: int, R: int = 32, per_rank_kib=(64, 1024, 1638
             "reducescatter": (lambda: ctx.reducescatter(x.view(R, R, E // R), small.view(R, E // R)), R * M + M),
             "allreduce": (lambda: ctx.allreduce(x, same), 2 * R * M),
         }
+        if "alltoallv" in only:
+            # uneven pairs: Zipf(1.2) receiver popularity, 10 % empty pairs, same mean volume as the all-to-all
+            pair = wl.gen_pair_bytes(R, M // R, seed=2000 + kib)
+            so, ro, si, st = wl.packed_offsets(pair)
+            vin = torch.empty((R, si), dtype=torch.uint8, device=dev).random_(0, 256)
+            vout = torch.empty((R, st), dtype=torch.uint8, device=dev)
+            pair_d, so_d, ro_d = (torch.from_numpy(a).to(dev) for a in (pair, so, ro))
+            ops["alltoallv"] = (lambda: ctx.alltoallv(vin, vout, pair_d, so_d, ro_d), 2 * int(pair.sum()))
         entry = {}
         for name, (fn, nbytes) in ops.items():
             if name not in only:
@@ -508,6 +516,12 @@ def collectives_report(dev_index: int, R: int = 32, per_rank_kib=(64, 1024, 1638
             ok = ok and bool(torch.equal(same, same[0].expand(R, E)))
         ctx.alltoall(x.view(R, R, E // R), same.view(R, R, E // R))
         ok = ok and bool(torch.equal(same.view(R, R, E // R), x.view(R, R, E // R).transpose(0, 1)))
+        if "alltoallv" in only:
+            p_, r_ = int(np.argmax(pair.sum(axis=1))), int(np.argmax(pair[int(np.argmax(pair.sum(axis=1)))]))
+            n_ = int(pair[p_, r_])
+            ok = ok and bool(torch.equal(vout[r_, ro[r_, p_]:ro[r_, p_] + n_], vin[p_, so[p_, r_]:so[p_, r_] + n_]))
+            entry["alltoallv"]["max_over_mean_received"] = round(float(pair.sum(axis=0).max() / pair.sum(axis=0).mean()), 2)
+            del vin, vout
         entry["verified"] = ok and ctx.device_status() == B.STRATA_OK
         rep["sizes"][f"{kib}KiB_per_rank"] = entry
         del x, big, same, small

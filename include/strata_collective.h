@@ -53,6 +53,27 @@ strata_status strata_alltoall(strata_ctx* ctx, int32_t R, const void* in, void* 
 strata_status strata_broadcast(strata_ctx* ctx, int32_t R, int32_t root, const void* in, void* out, size_t bytes,
                                void* stream);
 
+/* point-to-point.  in: [R][bytes], out: [R][bytes]; out[dst_rank][j] = in[src_rank][j]; the other parts of
+ * out are not touched.  bytes % 16 == 0. */
+strata_status strata_p2p(strata_ctx* ctx, int32_t R, int32_t src_rank, int32_t dst_rank, const void* in, void* out,
+                         size_t bytes, void* stream);
+
+/* all-to-all-v: pairs exchange different volumes (the operator the paper names, with MoE dispatch/combine,
+ * as the source of uneven traffic, Sec. 6.2).  in: [R][in_stride_bytes], out: [R][out_stride_bytes].
+ * send_bytes, send_offset, recv_offset: DEVICE arrays int64 [R][R], read by the kernel (they may be written
+ * by an earlier kernel on the same stream; nothing is copied to the host):
+ *   rank p sends send_bytes[p][r] bytes, found at in[p] + send_offset[p][r], to rank r, where they land at
+ *   out[r] + recv_offset[r][p].  Bytes of out that no pair addresses are not touched; pairs must not
+ *   overlap in out (not checked).
+ * Counts and offsets must be multiples of 16 and every pair must fit its two buffers: a pair that does
+ * not is skipped and STRATA_ERR_ALIGNMENT / STRATA_ERR_CAPACITY is raised in the device status word.
+ * R <= 32 (STRATA_ERR_SHAPE beyond: the pair table lives in shared memory); strides are non-zero multiples
+ * of 16.  The work is cut into 16 KB units claimed in order by a persistent grid, so a heavy pair is
+ * spread over all CTAs instead of being owned by one. */
+strata_status strata_alltoallv(strata_ctx* ctx, int32_t R, const void* in, size_t in_stride_bytes, void* out,
+                               size_t out_stride_bytes, const int64_t* send_bytes, const int64_t* send_offset,
+                               const int64_t* recv_offset, void* stream);
+
 /* reduce-scatter.  in: bf16 [R][R][elems_per_slice], out: bf16 [R][elems_per_slice];
  * out[r][j] = bf16( sum over p = 0..R-1, in that order, of in[p][r][j] ).  elems_per_slice % 8 == 0. */
 strata_status strata_reducescatter(strata_ctx* ctx, int32_t R, const void* in, void* out, size_t elems_per_slice,

@@ -114,8 +114,9 @@ const char *strata_status_string(strata_status s);
 strata_status strata_ctx_create(strata_ctx **out, const strata_moe_shape *shape, int device);
 strata_status strata_ctx_destroy(strata_ctx *ctx);
 
-/* Scratch memory the layout kernels need for this shape (per-tile histograms,
- * a ticket and the device status word).  The caller allocates at least `bytes`
+/* Scratch memory the kernels need for this shape (the device status word, a ticket
+ * and work-claim counters, the layout's per-tile histograms, and 24.8 KB for the pair
+ * table of strata_alltoallv).  The caller allocates at least `bytes`
  * bytes of device memory, 256-byte aligned, and hands it over with
  * strata_ctx_set_workspace, which zeroes it (synchronously).  It must stay
  * valid and unshared while calls on this context are in flight. */

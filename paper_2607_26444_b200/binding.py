@@ -41,6 +41,7 @@ EXPORTS = [
     "strata_moe_recv_rows",
     "strata_ctx_set_timeline", "strata_timeline_decode",
     "strata_allgather", "strata_alltoall", "strata_broadcast", "strata_reducescatter", "strata_allreduce",
+    "strata_p2p", "strata_alltoallv",
 ]
 
 
@@ -148,6 +149,8 @@ def lib() -> ctypes.CDLL:
         "strata_allgather": [vp, i32, vp, vp, sz, vp],
         "strata_alltoall": [vp, i32, vp, vp, sz, vp],
         "strata_broadcast": [vp, i32, i32, vp, vp, sz, vp],
+        "strata_p2p": [vp, i32, i32, i32, vp, vp, sz, vp],
+        "strata_alltoallv": [vp, i32, vp, sz, vp, sz, vp, vp, vp, vp],
         "strata_reducescatter": [vp, i32, vp, vp, sz, vp],
         "strata_allreduce": [vp, i32, vp, vp, sz, vp],
     }
@@ -372,6 +375,15 @@ def strata_alltoall(ctx, R: int, src: int, dst: int, bytes_per_slice: int, strea
 
 def strata_broadcast(ctx, R: int, root: int, src: int, dst: int, nbytes: int, stream: int) -> int:
     return lib().strata_broadcast(ctx, R, root, src, dst, nbytes, stream)
+
+
+def strata_p2p(ctx, R: int, src_rank: int, dst_rank: int, src: int, dst: int, nbytes: int, stream: int) -> int:
+    return lib().strata_p2p(ctx, R, src_rank, dst_rank, src, dst, nbytes, stream)
+
+
+def strata_alltoallv(ctx, R: int, src: int, in_stride: int, dst: int, out_stride: int, send_bytes: int,
+                     send_offset: int, recv_offset: int, stream: int) -> int:
+    return lib().strata_alltoallv(ctx, R, src, in_stride, dst, out_stride, send_bytes, send_offset, recv_offset, stream)
 
 
 def strata_reducescatter(ctx, R: int, src: int, dst: int, elems_per_slice: int, stream: int) -> int:
@@ -601,6 +613,24 @@ class MoEContext:
         R = src.shape[0]
         _check(strata_broadcast(self.h, R, root, src.data_ptr(), dst.data_ptr(),
                                 src[0].numel() * src.element_size(), self._stream()), "strata_broadcast")
+
+    def p2p(self, src, dst, src_rank: int, dst_rank: int) -> None:
+        """src, dst [R, n]: dst[dst_rank] = src[src_rank]."""
+        R = src.shape[0]
+        _check(strata_p2p(self.h, R, src_rank, dst_rank, src.data_ptr(), dst.data_ptr(),
+                          src[0].numel() * src.element_size(), self._stream()), "strata_p2p")
+
+    def alltoallv(self, src, dst, send_bytes, send_offset, recv_offset) -> None:
+        """src [R, in_stride] and dst [R, out_stride] uint8; the three int64 [R, R] device tensors give, per
+        (sender, receiver), the byte count, the offset in the sender's part and (indexed [receiver, sender])
+        the offset in the receiver's part."""
+        R = src.shape[0]
+        for t in (src, dst, send_bytes, send_offset, recv_offset):
+            if not t.is_contiguous():
+                raise ValueError("alltoallv needs contiguous tensors")
+        _check(strata_alltoallv(self.h, R, src.data_ptr(), src[0].numel() * src.element_size(), dst.data_ptr(),
+                                dst[0].numel() * dst.element_size(), send_bytes.data_ptr(), send_offset.data_ptr(),
+                                recv_offset.data_ptr(), self._stream()), "strata_alltoallv")
 
     def reducescatter(self, src, dst) -> None:
         """src bf16 [R, R, n] -> dst bf16 [R, n], dst[r] = sum over p of src[p, r] (rank order, fp32)."""

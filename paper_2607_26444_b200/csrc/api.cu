@@ -69,7 +69,7 @@ size_t workspace_bytes(const strata_moe_shape& s)
 {
     const LayoutGeom g = layout_geom(s);
     size_t b = (size_t)kWsHeaderBytes + (size_t)g.n_tiles * s.E * sizeof(int);
-    return (b + 255) & ~(size_t)255;
+    return ((b + 255) & ~(size_t)255) + collective_table_bytes();
 }
 
 WorkQueue dispatch_queue(const strata_ctx* c) { return WorkQueue{reinterpret_cast<unsigned int*>(c->ws) + 2}; }
@@ -622,6 +622,52 @@ strata_status strata_broadcast(strata_ctx* ctx, int32_t R, int32_t root, const v
     if (root < 0 || root >= R) return STRATA_ERR_INVALID_ARG;
     return run_copy(ctx, static_cast<const unsigned char*>(in) + (size_t)root * bytes, out, 1ull, bytes, 1u, 0ull, 0ull,
                     R, bytes, stream);
+}
+
+strata_status strata_p2p(strata_ctx* ctx, int32_t R, int32_t src_rank, int32_t dst_rank, const void* in, void* out,
+                         size_t bytes, void* stream)
+{
+    strata_status st = collective_prologue(ctx, R, in, out);
+    if (st != STRATA_OK) return st;
+    if (src_rank < 0 || src_rank >= R || dst_rank < 0 || dst_rank >= R) return STRATA_ERR_INVALID_ARG;
+    return run_copy(ctx, static_cast<const unsigned char*>(in) + (size_t)src_rank * bytes,
+                    static_cast<unsigned char*>(out) + (size_t)dst_rank * bytes, 1ull, bytes, 1u, 0ull, 0ull, 1, 0ull,
+                    stream);
+}
+
+strata_status strata_alltoallv(strata_ctx* ctx, int32_t R, const void* in, size_t in_stride_bytes, void* out,
+                               size_t out_stride_bytes, const int64_t* send_bytes, const int64_t* send_offset,
+                               const int64_t* recv_offset, void* stream)
+{
+    strata_status st = collective_prologue(ctx, R, in, out);
+    if (st != STRATA_OK) return st;
+    if (!send_bytes || !send_offset || !recv_offset) return STRATA_ERR_INVALID_ARG;
+    if (R > collective_max_v_ranks()) return STRATA_ERR_SHAPE;
+    if (in_stride_bytes == 0 || out_stride_bytes == 0 || in_stride_bytes % 16 != 0 || out_stride_bytes % 16 != 0)
+        return STRATA_ERR_SHAPE;
+    // every sender's chunks fit the unit counter whatever the counts turn out to be
+    const unsigned long long chunk = collective_chunk_bytes();
+    if (((unsigned long long)in_stride_bytes / chunk + (unsigned long long)R) * (unsigned long long)R > 0x7fffffffull)
+        return STRATA_ERR_SHAPE;
+    if (((reinterpret_cast<uintptr_t>(send_bytes) | reinterpret_cast<uintptr_t>(send_offset) |
+          reinterpret_cast<uintptr_t>(recv_offset)) & 7u) != 0)
+        return STRATA_ERR_ALIGNMENT;
+    if (ctx->device < 0) return STRATA_ERR_CUDA;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return STRATA_ERR_CUDA;
+    cudaError_t err = launch_slice_copyv(in, in_stride_bytes, out, out_stride_bytes,
+                                         reinterpret_cast<const long long*>(send_bytes),
+                                         reinterpret_cast<const long long*>(send_offset),
+                                         reinterpret_cast<const long long*>(recv_offset), R,
+                                         reinterpret_cast<unsigned char*>(ctx->ws) + workspace_bytes(ctx->shape) -
+                                             collective_table_bytes(),
+                                         ctx->ws,
+                                         collective_queue(ctx), ctx->n_sm, ctx->trace, static_cast<cudaStream_t>(stream));
+    {
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        ctx->launches += 2;                // table kernel + copy kernel
+    }
+    return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
 }
 
 strata_status strata_reducescatter(strata_ctx* ctx, int32_t R, const void* in, void* out, size_t elems_per_slice,

@@ -155,6 +155,202 @@ __global__ void __launch_bounds__(32) slice_copy_kernel(CopyParams p)
     }
 }
 
+// ---- all-to-all-v: the slice map comes from device arrays -------------------------------------
+// Per (sender, receiver) pair a byte count and two offsets, read on the GPU (no host round trip
+// between the kernel that produced the counts, e.g. the routing layout, and this one).
+// Kernel 1 (one CTA, one thread per pair) validates the pairs and writes a table into the workspace:
+// chunks per pair as an inclusive prefix, bytes/16, absolute source and destination offsets.
+// Kernel 2 (persistent single-warp CTAs, launched as a programmatic dependent for small payloads)
+// brings the table into shared memory with one bulk copy and locates each claimed unit by a binary
+// search of the prefix.  Pairs carry different volumes (the paper's first source of core-level long
+// tails, Sec. 6.2); the units are equal-sized chunks claimed in order, so no CTA owns a heavy peer.
+// (Letting every CTA build the table itself cost 14 us of prologue at 32 ranks: 296 CTAs reading the
+// same 24 KB, one of the three arrays transposed.)
+constexpr int kMaxVRanks = 32;
+constexpr int kMaxVPairs = kMaxVRanks * kMaxVRanks;
+
+struct VTable {                            // 24,592 bytes, a multiple of 16
+    unsigned int prefix[kMaxVPairs + 4];   // prefix[i] = chunks of pairs < i; prefix[n_pairs] = all units
+    unsigned int vec16[kMaxVPairs];        // bytes / 16 of the pair, 0 if empty or skipped
+    unsigned long long src_abs[kMaxVPairs];
+    unsigned long long dst_abs[kMaxVPairs];
+};
+static_assert(sizeof(VTable) % 16 == 0, "bulk-copy operand");
+
+struct CopyVParams {
+    const unsigned char* in;
+    unsigned char* out;
+    unsigned long long in_stride, out_stride;
+    const long long* send_bytes;          // [R][R]
+    const long long* send_off;            // [R][R]
+    const long long* recv_off;            // [R][R], indexed [receiver][sender]
+    VTable* table;                        // workspace
+    int R;
+    int* status;
+    WorkQueue wq;
+    TraceBuf trace;
+};
+
+__global__ void __launch_bounds__(kMaxVPairs) copyv_table_kernel(CopyVParams p)
+{
+    __shared__ unsigned int warp_sum[32];
+    const int i = threadIdx.x, lane = i & 31, warp = i >> 5;
+    const int n_pairs = p.R * p.R;
+    griddep_wait();                        // the count and offset arrays may come from the kernel before
+    griddep_launch_dependents();
+    unsigned int chunks = 0, v = 0;
+    unsigned long long sa = 0, da = 0;
+    if (i < n_pairs) {
+        const int snd = i / p.R, rcv = i - snd * p.R;
+        const long long n = p.send_bytes[i], so = p.send_off[i], ro = p.recv_off[rcv * p.R + snd];
+        if (n != 0) {
+            if (n < 0 || so < 0 || ro < 0 || (unsigned long long)(so + n) > p.in_stride ||
+                (unsigned long long)(ro + n) > p.out_stride) {
+                report_status(p.status, STRATA_ERR_CAPACITY);        // pair skipped
+            } else if (((n | so | ro) & 15) != 0) {
+                report_status(p.status, STRATA_ERR_ALIGNMENT);       // pair skipped
+            } else {
+                v = (unsigned int)(n >> 4);
+                chunks = (unsigned int)((n + kCopyChunkBytes - 1) / kCopyChunkBytes);
+            }
+        }
+        sa = (unsigned long long)snd * p.in_stride + (unsigned long long)so;
+        da = (unsigned long long)rcv * p.out_stride + (unsigned long long)ro;
+    }
+    unsigned int incl = chunks;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const unsigned int up = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += up;
+    }
+    if (lane == 31) warp_sum[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        unsigned int w = warp_sum[lane], wi = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned int up = __shfl_up_sync(0xffffffffu, wi, d);
+            if (lane >= d) wi += up;
+        }
+        warp_sum[lane] = wi - w;           // exclusive over warps
+    }
+    __syncthreads();
+    incl += warp_sum[warp];
+    if (i == 0) p.table->prefix[0] = 0;
+    if (i < n_pairs) {
+        p.table->prefix[i + 1] = incl;
+        p.table->vec16[i] = v;
+        p.table->src_abs[i] = sa;
+        p.table->dst_abs[i] = da;
+    }
+}
+
+__global__ void __launch_bounds__(32) slice_copyv_kernel(CopyVParams p)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int n_pairs = p.R * p.R;
+    unsigned char* stages = smem;
+    VTable* tab = reinterpret_cast<VTable*>(smem + (size_t)kCopyStages * kCopyChunkBytes);
+    unsigned long long* s_dst = reinterpret_cast<unsigned long long*>(tab + 1);   // [stages] destination of a stage's unit
+    uint64_t* bars = reinterpret_cast<uint64_t*>(s_dst + kCopyStages);            // [stages + 1], the last for the table
+    unsigned int* s_unit = reinterpret_cast<unsigned int*>(bars + kCopyStages + 1);
+    unsigned int* s_bytes = s_unit + kCopyStages;
+    const int lane = threadIdx.x;
+
+    if (lane == 0) {
+        for (int s = 0; s <= kCopyStages; ++s) mbar_init(&bars[s], 1);
+        for (int s = 0; s < kCopyStages; ++s) s_unit[s] = kNoUnit;
+        mbar_fence_init();
+    }
+    __syncwarp();
+    const uint64_t pol = policy_evict_first();
+    griddep_wait();                        // the table kernel has completed and its writes are visible
+    if (lane == 0) trace_begin(p.trace);
+    Timeline tl(p.trace, STRATA_KERNEL_SLICE_COPY, lane == 0);
+    tl.begin(STRATA_STAGE_KERNEL);
+    if (lane == 0) {
+        mbar_expect_tx(&bars[kCopyStages], (uint32_t)sizeof(VTable));
+        bulk_g2s(tab, p.table, (uint32_t)sizeof(VTable), &bars[kCopyStages], pol);
+    }
+    bool ok = mbar_wait_bounded(&bars[kCopyStages], 0);
+    ok = __all_sync(0xffffffffu, ok);
+    const unsigned int* prefix = tab->prefix;
+    const unsigned int n_units = ok ? prefix[n_pairs] : 0u;
+
+    int cur = 0;                            // lane 0: the pair the last located unit fell into
+    auto locate = [&](unsigned int u) {     // the i with prefix[i] <= u < prefix[i + 1]
+        if (u >= prefix[cur] && u < prefix[cur + 1]) return;
+        int a = 0, b = n_pairs;             // invariant: prefix[a] <= u < prefix[b]
+        while (b - a > 1) {
+            const int m = (a + b) >> 1;
+            if (prefix[m] <= u) a = m; else b = m;
+        }
+        cur = a;
+    };
+    bool triggered = false, exhausted = false;
+    const unsigned int n_static = (unsigned int)(kCopyStages - 1) * gridDim.x;
+    auto issue_load = [&](long long j) {   // lane 0 only
+        const int s = (int)(j % kCopyStages);
+        unsigned int u;
+        if (j < kCopyStages - 1) {
+            u = blockIdx.x + (unsigned int)j * gridDim.x;
+            if (u >= n_units) u = kNoUnit;
+        } else {
+            u = claim_unit(p.wq, n_units, n_static, exhausted);
+        }
+        s_unit[s] = u;
+        if (u == kNoUnit) {
+            if (!triggered) griddep_launch_dependents();
+            triggered = true;
+            return;
+        }
+        locate(u);
+        const unsigned long long off = (unsigned long long)(u - prefix[cur]) * kCopyChunkBytes;
+        const unsigned long long left = (unsigned long long)tab->vec16[cur] * 16ull - off;
+        const uint32_t bytes = left < kCopyChunkBytes ? (uint32_t)left : kCopyChunkBytes;
+        s_bytes[s] = bytes;
+        s_dst[s] = tab->dst_abs[cur] + off;
+        mbar_expect_tx(&bars[s], bytes);
+        bulk_g2s(stages + (size_t)s * kCopyChunkBytes, p.in + tab->src_abs[cur] + off, bytes, &bars[s], pol);
+    };
+
+    if (lane == 0)
+        for (long long j = 0; j < kCopyStages - 1; ++j) issue_load(j);
+    __syncwarp();
+
+    for (long long j = 0; ok; ++j) {
+        const int s = (int)(j % kCopyStages);
+        const uint32_t parity = (uint32_t)((j / kCopyStages) & 1);
+        if (s_unit[s] == kNoUnit) break;
+        tl.begin(STRATA_STAGE_WAIT_IN);
+        ok = mbar_wait_bounded(&bars[s], parity);
+        tl.end(STRATA_STAGE_WAIT_IN);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (lane == 0) {
+            tl.begin(STRATA_STAGE_WORK);
+            bulk_s2g(p.out + s_dst[s], stages + (size_t)s * kCopyChunkBytes, s_bytes[s]);
+            bulk_commit();
+            tl.end(STRATA_STAGE_WORK);
+            tl.begin(STRATA_STAGE_WAIT_OUT);
+            bulk_wait_read<1>();
+            tl.end(STRATA_STAGE_WAIT_OUT);
+            issue_load(j + kCopyStages - 1);
+        }
+        __syncwarp();
+    }
+    if (lane == 0) {
+        if (!ok) report_status(p.status, STRATA_ERR_TIMEOUT);
+        bulk_wait_read<0>();
+        trace_end(p.trace);
+        tl.end(STRATA_STAGE_KERNEL);
+        tl.finish();
+    }
+}
+
+constexpr size_t kCopyVSmem = (size_t)kCopyStages * kCopyChunkBytes + sizeof(VTable) + kCopyStages * 8 +
+                              (kCopyStages + 1) * 8 + 2 * kCopyStages * 4 + 16;
+
 struct ReduceParams {
     const unsigned char* in;
     unsigned char* out;
@@ -249,7 +445,36 @@ constexpr size_t kCopySmem = (size_t)kCopyStages * kCopyChunkBytes + kCopyStages
 
 cudaError_t configure_collective_kernels()
 {
-    return cudaFuncSetAttribute(slice_copy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCopySmem);
+    cudaError_t err = cudaFuncSetAttribute(slice_copy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCopySmem);
+    if (err != cudaSuccess) return err;
+    return cudaFuncSetAttribute(slice_copyv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCopyVSmem);
+}
+
+int collective_max_v_ranks() { return kMaxVRanks; }
+size_t collective_table_bytes() { return (sizeof(VTable) + 255) & ~(size_t)255; }
+
+cudaError_t launch_slice_copyv(const void* in, unsigned long long in_stride, void* out, unsigned long long out_stride,
+                               const long long* send_bytes, const long long* send_off, const long long* recv_off, int R,
+                               void* table, int* status, WorkQueue wq, int n_sm, TraceBuf trace, cudaStream_t st)
+{
+    CopyVParams p{};
+    p.in = static_cast<const unsigned char*>(in);
+    p.out = static_cast<unsigned char*>(out);
+    p.in_stride = in_stride;
+    p.out_stride = out_stride;
+    p.send_bytes = send_bytes;
+    p.send_off = send_off;
+    p.recv_off = recv_off;
+    p.table = static_cast<VTable*>(table);
+    p.R = R;
+    p.status = status;
+    p.wq = wq;
+    p.trace = trace;
+    cudaError_t err = launch_pdl(copyv_table_kernel, 1u, (unsigned)kMaxVPairs, 0, st, p);
+    if (err != cudaSuccess) return err;
+    // the number of units is known only on the device: a full persistent grid, CTAs without work leave at once
+    const bool small = (long long)R * (long long)(in_stride + out_stride) < kPdlMaxBytes;
+    return STRATA_LAUNCH_LONG(small, slice_copyv_kernel, (unsigned)(n_sm * kCopyCtasPerSm), 32, kCopyVSmem, st, p);
 }
 
 uint32_t collective_chunk_bytes() { return kCopyChunkBytes; }

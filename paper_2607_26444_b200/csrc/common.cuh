@@ -15,6 +15,7 @@ namespace strata {
 // word 2: work-claim counter of dispatch, word 4: of combine, word 6: of the collectives (each returns
 //         to 0 inside the kernel)
 // bytes [256, ...): per-tile, per-expert counts, int32 [n_tiles, E]
+// the last collective_table_bytes() bytes: pair table of all-to-all-v
 constexpr int kWsHeaderBytes = 256;
 constexpr int kLayoutThreads = 1024;   // threads per layout CTA
 constexpr int kItemsPerThread = 4;
@@ -89,6 +90,11 @@ cudaError_t launch_slice_copy(const void* in, void* out, unsigned long long n_sl
 cudaError_t launch_slice_reduce(const void* in, void* out, unsigned long long n_vec, int R, int fan, WorkQueue wq,
                                 int n_sm, TraceBuf trace, cudaStream_t st);
 uint32_t collective_chunk_bytes();
+int collective_max_v_ranks();
+size_t collective_table_bytes();     // workspace tail used by all-to-all-v (a multiple of 256)
+cudaError_t launch_slice_copyv(const void* in, unsigned long long in_stride, void* out, unsigned long long out_stride,
+                               const long long* send_bytes, const long long* send_off, const long long* recv_off, int R,
+                               void* table, int* status, WorkQueue wq, int n_sm, TraceBuf trace, cudaStream_t st);
 int partition_max_units_supported();
 int partition_max_cores_supported();
 uint32_t windows_max_row_bytes();

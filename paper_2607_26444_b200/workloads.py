@@ -211,7 +211,8 @@ def packed_offsets(pair_bytes: np.ndarray):
     recv_off = np.cumsum(recv, axis=1) - recv
     in_stride = int(max(16, pair_bytes.sum(axis=1).max()))
     out_stride = int(max(16, recv.sum(axis=1).max()))
-    return send_off.astype(np.int64), recv_off.astype(np.int64), in_stride, out_stride
+    return (np.ascontiguousarray(send_off, dtype=np.int64), np.ascontiguousarray(recv_off, dtype=np.int64),
+            in_stride, out_stride)
 
 
 def generate(cfg: MoEConfig) -> Dict[str, np.ndarray]:

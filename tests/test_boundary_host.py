@@ -60,10 +60,12 @@ def test_bad_shapes_are_rejected(kw):
 
 def test_workspace_size():
     rc, n = B.strata_moe_workspace_bytes(shape())
-    # 4 ranks x ceil(128*2/4096)=1 tile, 16 experts, 256-byte header, rounded to 256
-    assert rc == 0 and n == 512
+    # 4 ranks x ceil(128*2/4096)=1 tile, 16 experts, 256-byte header, rounded to 256; then the pair table of
+    # all-to-all-v (1028 + 1024 uint32, 2 x 1024 uint64 = 24,592 bytes, rounded to 256)
+    table = 24832
+    assert rc == 0 and n == 512 + table
     rc, n = B.strata_moe_workspace_bytes(shape(R=16, T=4096, H=7168, E=256, K=8))
-    assert rc == 0 and n == 256 + 16 * 8 * 256 * 4
+    assert rc == 0 and n == 256 + 16 * 8 * 256 * 4 + table
 
 
 @pytest.fixture
@@ -119,9 +121,9 @@ def test_host_detectable_errors_before_any_launch(ctx):
     n_rows = 4 * 128 * 2
     # no workspace yet
     assert B.strata_moe_layout(ctx, ids, lay, None) == B.STRATA_ERR_WORKSPACE
-    assert B.strata_ctx_set_workspace(ctx, 0x7B00_0000_0010, 4096) == B.STRATA_ERR_ALIGNMENT
+    assert B.strata_ctx_set_workspace(ctx, 0x7B00_0000_0010, 1 << 16) == B.STRATA_ERR_ALIGNMENT
     assert B.strata_ctx_set_workspace(ctx, 0x7B00_0000_0000, 16) == B.STRATA_ERR_CAPACITY
-    assert B.strata_ctx_set_workspace(ctx, 0x7B00_0000_0000, 4096) == 0
+    assert B.strata_ctx_set_workspace(ctx, 0x7B00_0000_0000, 1 << 16) == 0
     # NULLs
     assert B.strata_moe_layout(ctx, None, lay, None) == B.STRATA_ERR_INVALID_ARG
     bad = _fake_layout()
@@ -157,7 +159,7 @@ def test_fp8_context_needs_registered_scales():
     rc, h = B.strata_ctx_create(shape(dt=B.STRATA_FP8_E4M3_B128), -1)
     assert rc == 0
     try:
-        assert B.strata_ctx_set_workspace(h, 0x7B00_0000_0000, 4096) == 0
+        assert B.strata_ctx_set_workspace(h, 0x7B00_0000_0000, 1 << 16) == 0
         lay = _fake_layout()
         x, recv, sc = 0x7D00_0000_0000, 0x7C00_0000_0000, 0x7A00_0000_0000
         n_rows = 1024
@@ -210,6 +212,12 @@ def test_collectives_reject_bad_arguments_before_any_launch():
         assert B.strata_allreduce(h, 4, fake, 2 * fake, 12, None) == B.STRATA_ERR_SHAPE
         assert B.strata_reducescatter(h, 4, fake, 2 * fake, 4, None) == B.STRATA_ERR_SHAPE
         assert B.strata_allgather(h, 4, fake, 2 * fake, 0, None) == B.STRATA_OK        # nothing to move
+        assert B.strata_p2p(h, 4, 4, 0, fake, 2 * fake, 64, None) == B.STRATA_ERR_INVALID_ARG
+        assert B.strata_p2p(h, 4, 0, 1, fake, 2 * fake, 64, None) == B.STRATA_ERR_CUDA
+        assert B.strata_alltoallv(h, 33, fake, 64, 2 * fake, 64, fake, fake, fake, None) == B.STRATA_ERR_SHAPE
+        assert B.strata_alltoallv(h, 4, fake, 0, 2 * fake, 64, fake, fake, fake, None) == B.STRATA_ERR_SHAPE
+        assert B.strata_alltoallv(h, 4, fake, 64, 2 * fake, 64, fake + 4, fake, fake, None) == B.STRATA_ERR_ALIGNMENT
+        assert B.strata_alltoallv(h, 4, fake, 64, 2 * fake, 64, fake, fake, fake, None) == B.STRATA_ERR_CUDA
         # a host-only context never launches
         for rc in (B.strata_allgather(h, 4, fake, 2 * fake, 64, None),
                    B.strata_alltoall(h, 4, fake, 2 * fake, 64, None),

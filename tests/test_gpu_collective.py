@@ -239,3 +239,120 @@ def test_full_size_sampled(ctx):
     want = oracle.allgather(np.ascontiguousarray(host_cols(samp_d)).view(np.uint8))
     got = ag[:, :, samp_d].cpu().numpy().view(np.uint8)
     assert np.array_equal(got, want)
+
+
+# ---- all-to-all-v and point-to-point -----------------------------------------------------------
+
+def run_alltoallv(ctx, x, sb, so, ro, out_stride, fill=0xEE):
+    R = x.shape[0]
+    whole = torch.full((R * out_stride + 2 * GUARD,), fill, dtype=torch.uint8, device=DEV)
+    out = whole[GUARD:GUARD + R * out_stride].view(R, out_stride)
+    ctx.alltoallv(torch.from_numpy(x).to(DEV), out, torch.from_numpy(sb).to(DEV), torch.from_numpy(so).to(DEV),
+                  torch.from_numpy(ro).to(DEV))
+    torch.cuda.synchronize()
+    h = whole.cpu().numpy()
+    assert np.all(h[:GUARD] == fill) and np.all(h[-GUARD:] == fill)
+    return out.cpu().numpy()
+
+
+@pytest.mark.parametrize("R,mean,seed", [(1, 64, 1), (2, 16, 2), (4, 4096, 3), (7, 3 * CHUNK, 4), (16, CHUNK + 4096, 5),
+                                         (32, 2 * CHUNK, 6)])
+def test_alltoallv_uneven_pairs(ctx, R, mean, seed):
+    sb = wl.gen_pair_bytes(R, mean, seed=seed)
+    so, ro, si, st = wl.packed_offsets(sb)
+    so, ro, si, st = so + 16, ro + 48, si + 64, st + 96           # gaps nobody addresses
+    x = payload_bytes(R, si, seed=seed + 40)
+    got = run_alltoallv(ctx, x, sb, so, ro, st)
+    want = np.full((R, st), 0xEE, np.uint8)
+    assert oracle.alltoallv(x, want, sb, so, ro) == 0
+    assert np.array_equal(got, want)
+    assert ctx.device_status() == B.STRATA_OK
+
+
+def test_alltoallv_one_heavy_pair_and_many_empty(ctx):
+    R = 8
+    sb = np.zeros((R, R), np.int64)
+    sb[3, 5] = 40 * CHUNK + 16                                    # one pair carries almost everything
+    sb[0, 0] = 16
+    sb[7, 2] = CHUNK
+    so, ro, si, st = wl.packed_offsets(sb)
+    x = payload_bytes(R, si, seed=77)
+    got = run_alltoallv(ctx, x, sb, so, ro, st)
+    want = np.full((R, st), 0xEE, np.uint8)
+    oracle.alltoallv(x, want, sb, so, ro)
+    assert np.array_equal(got, want)
+
+
+def test_alltoallv_all_empty_and_back_to_back(ctx):
+    R = 4
+    sb = np.zeros((R, R), np.int64)
+    x = payload_bytes(R, 64, seed=78)
+    for _ in range(3):
+        got = run_alltoallv(ctx, x, sb, sb.copy(), sb.copy(), 64)
+        assert np.all(got == 0xEE)
+    sb2 = wl.gen_pair_bytes(R, 8 * CHUNK, seed=9)
+    so, ro, si, st = wl.packed_offsets(sb2)
+    x = payload_bytes(R, si, seed=79)
+    want = np.full((R, st), 0xEE, np.uint8)
+    oracle.alltoallv(x, want, sb2, so, ro)
+    for _ in range(3):                                            # the claim counter re-arms itself every time
+        assert np.array_equal(run_alltoallv(ctx, x, sb2, so, ro, st), want)
+    assert ctx.device_status() == B.STRATA_OK
+
+
+def test_alltoallv_bad_pairs_are_skipped_and_reported(ctx):
+    R = 2
+    x = payload_bytes(R, 256, seed=80)
+    sb = np.array([[32, 128], [16, 24]], np.int64)                # (1 -> 1): 24 is not a multiple of 16
+    so = np.array([[0, 192], [0, 32]], np.int64)                  # (0 -> 1): 192 + 128 > 256
+    ro = np.array([[0, 32], [0, 128]], np.int64)
+    got = run_alltoallv(ctx, x, sb, so, ro, 256)
+    st = ctx.device_status()
+    assert st in (B.STRATA_ERR_CAPACITY, B.STRATA_ERR_ALIGNMENT)
+    want = np.full((R, 256), 0xEE, np.uint8)
+    want[0, 0:32] = x[0, 0:32]                                    # (0 -> 0)
+    want[0, 32:48] = x[1, 0:16]                                   # (1 -> 0)
+    assert np.array_equal(got, want)
+    assert ctx.device_status() == B.STRATA_OK                     # the status word was cleared
+    sb_ok = np.array([[32, 0], [16, 0]], np.int64)
+    assert np.array_equal(run_alltoallv(ctx, x, sb_ok, so, ro, 256), want)
+
+
+def test_alltoallv_counts_from_a_kernel_on_the_same_stream(ctx):
+    """The counts never visit the host: they are produced on the device right before the call."""
+    R = 8
+    sb = wl.gen_pair_bytes(R, 4 * CHUNK, seed=12)
+    so, ro, si, st = wl.packed_offsets(sb)
+    x = payload_bytes(R, si, seed=81)
+    x_d = torch.from_numpy(x).to(DEV)
+    half = torch.from_numpy(sb // 32 * 16).to(DEV)
+    so_d, ro_d = torch.from_numpy(so).to(DEV), torch.from_numpy(ro).to(DEV)
+    out = torch.full((R, st), 0xEE, dtype=torch.uint8, device=DEV)
+    sb_d = half + half                                            # a device computation, no synchronisation
+    ctx.alltoallv(x_d, out, sb_d, so_d, ro_d)
+    torch.cuda.synchronize()
+    want = np.full((R, st), 0xEE, np.uint8)
+    oracle.alltoallv(x, want, (sb // 32 * 16) * 2, so, ro)
+    assert np.array_equal(out.cpu().numpy(), want)
+
+
+def test_alltoallv_rejects_on_the_host(ctx):
+    d = torch.zeros((64, 64), dtype=torch.int64, device=DEV)
+    b = torch.zeros((64 * 64,), dtype=torch.uint8, device=DEV)
+    args = (b.data_ptr(), 64, b.data_ptr(), 64, d.data_ptr(), d.data_ptr(), d.data_ptr(), None)
+    assert B.strata_alltoallv(ctx.h, 33, *args) == B.STRATA_ERR_SHAPE
+    assert B.strata_alltoallv(ctx.h, 4, b.data_ptr(), 40, *args[2:]) == B.STRATA_ERR_SHAPE
+    assert B.strata_alltoallv(ctx.h, 4, b.data_ptr(), 64, b.data_ptr(), 64, None, d.data_ptr(), d.data_ptr(), None) \
+        == B.STRATA_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("R,n,src,dst", [(1, 16, 0, 0), (4, CHUNK + 32, 3, 1), (32, 3 * CHUNK, 5, 5)])
+def test_p2p(ctx, R, n, src, dst):
+    x = payload_bytes(R, n, seed=n + src)
+    whole, out = guarded_out(R * n)
+    ctx.p2p(torch.from_numpy(x).to(DEV), out.view(R, n), src, dst)
+    torch.cuda.synchronize()
+    want = np.full((R, n), SENT8, np.uint8)
+    oracle.p2p(x, want, src, dst)
+    assert np.array_equal(out.cpu().numpy().reshape(R, n), want)
+    assert guards_intact(whole)
