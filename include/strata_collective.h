@@ -10,7 +10,7 @@
  * Here all R ranks are partitions of ONE GPU's memory, as for the MoE path: rank r's input is the
  * r-th equal part of `in`, its output the r-th equal part of `out`.  Nothing crosses a link, so what
  * is measured is the memory system serving the operator's slice map, not a fabric.  One kernel
- * launch per call; every operand of an output vector is seen by one thread, so the reductions need
+ * launch per call (two for all-to-all-v); every operand of an output vector is seen by one thread, so the reductions need
  * neither atomics nor locks.
  *
  * Arithmetic of the reductions (this build's reading; the paper names none): bf16 operands, one
