@@ -714,6 +714,18 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
         gbs, dt, cores, sample = time_oracle(cfg, host_inp, reps=2)
         cpu = {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
                "seconds": round(dt, 3)}
+        # one thread, on a sixteenth of the tokens (same recipe)
+        import oracle
+        scfg = oracle_sample_config(cfg, max(1, cfg.T // 16))
+        sinp = wl.generate(scfg)
+        t0 = time.perf_counter()
+        lay1 = oracle.layout(sinp["ids"], scfg.E)
+        recv1 = oracle.dispatch_bf16(lay1["dst_row"], sinp["x"], nthreads=1)
+        oracle.combine(lay1["dst_row"], recv1, sinp["w"], nthreads=1)
+        dt1 = time.perf_counter() - t0
+        del recv1
+        cpu["single_thread"] = {"value": (scfg.dispatch_bytes() + scfg.combine_bytes()) / dt1 / 1e9, "unit": UNIT,
+                                "sample": f"T={scfg.T} of {cfg.T} tokens/rank, one pass", "seconds": round(dt1, 3)}
     sampler.stop()
 
     line = {
