@@ -24,7 +24,8 @@
  * STRATA_ERR_INVALID_ARG (NULL, R outside [1, 1024], root out of range), STRATA_ERR_SHAPE (a size
  * that is not a multiple of 16 bytes / 8 elements, or more than 2^32-1 work units),
  * STRATA_ERR_ALIGNMENT, STRATA_ERR_WORKSPACE, STRATA_ERR_CUDA (host-only context, launch failure).
- * A size of 0 is legal and launches nothing.  A bounded device wait that runs out reports
+ * The collectives do not consult the registration pool: any device buffers are accepted (only the MoE
+ * receive buffer has a readiness check).  A size of 0 is legal and launches nothing.  A bounded device wait that runs out reports
  * STRATA_ERR_TIMEOUT through strata_device_status().  Like the MoE calls they belong to the
  * context's single stream at a time.
  */
