@@ -47,3 +47,22 @@ def test_gpu_arm_line_on_a_small_workload():
     assert {"sm_mhz", "sm_max_mhz", "reasons"} <= set(d["clocks"])
     cpu = d["cpu_baseline"]
     assert cpu["kind"] == "oracle" and cpu["cores"] >= 1 and cpu["value"] > 0 and "sample" in cpu
+
+
+@pytest.mark.gpu
+def test_collectives_report_mode():
+    d = run_bench("--collectives", "--collective-kib", "64", "256", "--collective-iters", "3")
+    assert d["R"] == 32 and set(d["sizes"]) == {"64KiB_per_rank", "256KiB_per_rank"}
+    for size in d["sizes"].values():
+        assert size["verified"] is True
+        for op in ("allgather", "alltoall", "alltoallv", "broadcast", "reducescatter", "allreduce"):
+            assert size[op]["median_us"] > 0 and size[op]["back_to_back_us"] > 0 and size[op]["bytes"] > 0
+
+
+@pytest.mark.gpu
+def test_timeline_report_mode(tmp_path):
+    trace = tmp_path / "trace.json"
+    d = run_bench("--timeline", "--workload", "tiny", "--timeline-trace", str(trace))
+    assert d["events_dropped"] == 0 and {"dispatch_bf16", "combine"} <= set(d["kernels"])
+    assert d["kernels"]["dispatch_bf16"]["stages"]["work"]["intervals"] == 4 * 128       # one per token
+    assert d["chrome_trace_events"] > 0 and json.loads(trace.read_text())["traceEvents"]
