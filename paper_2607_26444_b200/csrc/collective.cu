@@ -33,6 +33,7 @@ struct CopyParams {
     unsigned char* out;
     unsigned long long slice_bytes;
     unsigned int chunk_bytes;             // <= kCopyChunkBytes, a multiple of 16
+    unsigned int stage_bytes;             // chunk_bytes rounded up to 128: distance between two stages
     unsigned int chunks_per_slice;
     unsigned int fan_groups;              // the fan copies of a chunk are dealt to this many units
     unsigned int fan_per_group;
@@ -50,7 +51,7 @@ struct CopyParams {
 __global__ void __launch_bounds__(32) slice_copy_kernel(CopyParams p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kCopyStages * kCopyChunkBytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kCopyStages * p.stage_bytes);
     unsigned int* s_unit = reinterpret_cast<unsigned int*>(bars + kCopyStages);
     const int lane = threadIdx.x;
     const unsigned int n_units = p.n_units;
@@ -100,7 +101,7 @@ __global__ void __launch_bounds__(32) slice_copy_kernel(CopyParams p)
         int f0;
         decode(u, slice, off, bytes, f0);
         mbar_expect_tx(&bars[s], bytes);
-        bulk_g2s(smem + (size_t)s * kCopyChunkBytes, p.in + (size_t)slice * p.slice_bytes + off, bytes, &bars[s], pol);
+        bulk_g2s(smem + (size_t)s * p.stage_bytes, p.in + (size_t)slice * p.slice_bytes + off, bytes, &bars[s], pol);
     };
 
     if (lane == 0)
@@ -130,7 +131,7 @@ __global__ void __launch_bounds__(32) slice_copy_kernel(CopyParams p)
             tl.begin(STRATA_STAGE_WORK);
             unsigned char* dst = p.out + (size_t)(slice / p.inner) * p.stride_a + (size_t)(slice % p.inner) * p.stride_b + off;
             const int f1 = min(p.fan, f0 + (int)p.fan_per_group);
-            for (int f = f0; f < f1; ++f) bulk_s2g(dst + (size_t)f * p.fan_stride, smem + (size_t)s * kCopyChunkBytes, bytes);
+            for (int f = f0; f < f1; ++f) bulk_s2g(dst + (size_t)f * p.fan_stride, smem + (size_t)s * p.stage_bytes, bytes);
             bulk_commit();
             tl.end(STRATA_STAGE_WORK);
             wait_out.begin();
@@ -488,21 +489,26 @@ cudaError_t launch_slice_copy(const void* in, void* out, unsigned long long n_sl
     p.in = static_cast<const unsigned char*>(in);
     p.out = static_cast<unsigned char*>(out);
     p.slice_bytes = slice_bytes;
-    // Large payloads: 16 KB chunks, all fan copies of a chunk from one load.  When that leaves the grid
-    // short of units (small payloads are latency bound: a unit's stores are issued by one thread), first the
-    // fan copies of a chunk are dealt to several units (each re-reads the chunk, an L2 hit), then the chunks
-    // shrink, down to 2 KB.
-    const unsigned long long want = 2ull * (unsigned long long)n_sm * kCopyCtasPerSm;
+    // Large payloads: 16 KB chunks, all fan copies of a chunk from one load, two CTAs per SM.  When that
+    // leaves the grid short of units the call is latency bound (a unit's copies are issued by one thread,
+    // a CTA takes its units one after the other): first the fan copies of a chunk are dealt to several
+    // units (each re-reads the chunk, an L2 hit), then the chunks shrink, down to 2 KB, until there are
+    // four units per SM; the stages shrink with the chunks, so that up to eight CTAs fit an SM and every
+    // CTA gets one unit.
+    const unsigned long long want_big = 2ull * (unsigned long long)n_sm * kCopyCtasPerSm;
+    const unsigned long long want_small = 4ull * (unsigned long long)n_sm;   // 4, 6, 8, 16 tried: 4 and 6 tie, more is slower
     unsigned long long chunk = kCopyChunkBytes, fpg = (unsigned long long)fan;
     auto units = [&]() {
         return n_slices * ((slice_bytes + chunk - 1) / chunk) * (((unsigned long long)fan + fpg - 1) / fpg);
     };
-    while (units() < want) {
+    const bool latency_bound = units() < want_big;
+    while (latency_bound && units() < want_small) {
         if (fpg > 1) fpg = (fpg + 1) / 2;
         else if (chunk > 2048) chunk /= 2;
         else break;
     }
     p.chunk_bytes = (unsigned int)chunk;
+    p.stage_bytes = (unsigned int)((min(chunk, slice_bytes) + 127) / 128 * 128);
     p.chunks_per_slice = (unsigned int)((slice_bytes + chunk - 1) / chunk);
     p.fan_per_group = (unsigned int)fpg;
     p.fan_groups = (unsigned int)(((unsigned long long)fan + fpg - 1) / fpg);
@@ -515,9 +521,18 @@ cudaError_t launch_slice_copy(const void* in, void* out, unsigned long long n_sl
     p.status = status;
     p.wq = wq;
     p.trace = trace;
-    const unsigned grid = (unsigned)max(1ll, min((long long)n_sm * kCopyCtasPerSm, (long long)p.n_units));
+    const size_t smem = (size_t)kCopyStages * p.stage_bytes + kCopyStages * sizeof(uint64_t) +
+                        kCopyStages * sizeof(unsigned int) + 16;
+    long long max_grid = (long long)n_sm * kCopyCtasPerSm;
+    if (latency_bound) {
+        int per_sm = 0;
+        cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, slice_copy_kernel, 32, smem);
+        if (err != cudaSuccess) return err;
+        max_grid = (long long)n_sm * max(kCopyCtasPerSm, min(per_sm, 8));
+    }
+    const unsigned grid = (unsigned)max(1ll, min(max_grid, (long long)p.n_units));
     const bool small = (long long)(n_slices * slice_bytes) * (fan + 1) < kPdlMaxBytes;
-    return STRATA_LAUNCH_LONG(small, slice_copy_kernel, grid, 32, kCopySmem, st, p);
+    return STRATA_LAUNCH_LONG(small, slice_copy_kernel, grid, 32, smem, st, p);
 }
 
 cudaError_t launch_slice_reduce(const void* in, void* out, unsigned long long n_vec, int R, int fan,
