@@ -442,6 +442,37 @@ def timeline_report(cfg: wl.MoEConfig, dev_index: int, trace_path: str = "", pin
     return rep
 
 
+def sm_budget_report(cfg: wl.MoEConfig, dev_index: int, budgets=(8, 16, 24, 32, 48, 64, 96, 128, 0), iters: int = 10):
+    """Dispatch and combine throughput against the SM budget of the persistent grids (how many SMs' worth of
+    CTAs it takes to saturate HBM; the paper makes the same measurement for its fabric, Sec. 3.2)."""
+    case = DeviceCase(cfg, dev_index)
+    torch = case.torch
+    case.layout()
+    rows = []
+    for b in budgets:
+        case.ctx.sm_budget(b)
+        ent = {"sm_budget": b if b else "all"}
+        for name, fn, nbytes in (("dispatch", case.dispatch, cfg.dispatch_bytes()),
+                                 ("combine", case.combine, cfg.combine_bytes())):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+            torch.cuda._sleep(10_000_000)
+            ev[0].record()
+            for i in range(iters):
+                fn()
+                ev[i + 1].record()
+            torch.cuda.synchronize()
+            ts = sorted(ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(iters))
+            ent[name + "_us"] = round(ts[len(ts) // 2], 1)
+            ent[name + "_GBs"] = round(nbytes / ts[len(ts) // 2] / 1e3, 1)
+        rows.append(ent)
+    case.ctx.sm_budget(0)
+    case.check()
+    return {"workload": cfg.name, "iters": iters, "rows": rows}
+
+
 COLLECTIVE_OPS = ("allgather", "alltoall", "alltoallv", "broadcast", "reducescatter", "allreduce")
 
 
@@ -766,6 +797,8 @@ def main():
                     help="print only the in-kernel timeline summary of one step of --workload (not the bench line)")
     ap.add_argument("--timeline-trace", default="", help="also write a Chrome trace-event file of the first 32 CTAs")
     ap.add_argument("--timeline-pinned", action="store_true", help="kernels write the events into pinned host memory")
+    ap.add_argument("--sm-sweep", action="store_true",
+                    help="print only dispatch/combine throughput against the SM budget for --workload")
     ap.add_argument("--collectives", action="store_true",
                     help="print only the report on the full-mesh collectives (one JSON object; not the bench line)")
     ap.add_argument("--collective-kib", type=int, nargs="+", default=[64, 1024, 16384], help="payload per rank, KiB")
@@ -790,6 +823,13 @@ def main():
             if args.tokens_per_rank:
                 cfg = wl.shrink(cfg, T=args.tokens_per_rank)
             print(json.dumps(timeline_report(cfg, local_rank, args.timeline_trace, args.timeline_pinned)), flush=True)
+        return
+    if args.sm_sweep:
+        if rank == 0:
+            cfg = wl.CONFIGS[args.workload]
+            if args.tokens_per_rank:
+                cfg = wl.shrink(cfg, T=args.tokens_per_rank)
+            print(json.dumps(sm_budget_report(cfg, local_rank)), flush=True)
         return
     if args.collectives:
         if rank == 0:

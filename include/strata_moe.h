@@ -130,6 +130,15 @@ strata_status strata_ctx_set_workspace(strata_ctx *ctx, void *dptr, size_t bytes
 /* Number of kernels this context has launched so far (for accounting). */
 strata_status strata_ctx_launch_count(strata_ctx *ctx, uint64_t *count);
 
+/* SM budget.  Dispatch, combine and the collectives run as persistent grids sized for the whole GPU
+ * (a fixed number of CTAs per SM).  n_sm > 0 sizes them for n_sm SMs instead, so that a compute kernel
+ * running beside them on another stream keeps the rest (the paper's Sec. 3.2 observation that a fraction
+ * of the cores saturates the fabric, and its Sec. 6.3 aim of freeing cores for computation); 0 restores
+ * the default, values above the device's SM count are clamped.  The budget bounds the number of CTAs,
+ * it does not pin them to particular SMs.  Results do not depend on it.  The layout kernels are not
+ * affected. */
+strata_status strata_ctx_set_sm_budget(strata_ctx *ctx, int32_t n_sm);
+
 /* Per-CTA stage probes (after the paper's in-kernel profiler, Sec. 6.4: probes at stage boundaries
  * writing a cycle counter into a per-core slice of a trace buffer).  dptr: device array of
  * 4*capacity_ctas uint64, owned by the caller; while set, CTA b (b < capacity_ctas) of every

@@ -39,7 +39,7 @@ EXPORTS = [
     "strata_moe_roundtrip_host", "strata_moe_layout_noalloc", "strata_ctx_set_trace",
     "strata_moe_partition_max_units", "strata_moe_partition", "strata_moe_dispatch_windows",
     "strata_moe_recv_rows",
-    "strata_ctx_set_timeline", "strata_timeline_decode",
+    "strata_ctx_set_timeline", "strata_timeline_decode", "strata_ctx_set_sm_budget",
     "strata_allgather", "strata_alltoall", "strata_broadcast", "strata_reducescatter", "strata_allreduce",
     "strata_p2p", "strata_alltoallv",
 ]
@@ -144,6 +144,7 @@ def lib() -> ctypes.CDLL:
         "strata_moe_partition": [vp, P(strata_moe_layout_t), P(strata_partition_policy), i32,
                                  P(strata_partition_t), sz, vp],
         "strata_moe_dispatch_windows": [vp, P(strata_moe_layout_t), P(strata_partition_t), i32, vp, vp, sz, vp],
+        "strata_ctx_set_sm_budget": [vp, i32],
         "strata_ctx_set_timeline": [vp, vp, sz, sz],
         "strata_timeline_decode": [vp, sz, sz, vp, sz, P(sz), P(sz)],
         "strata_allgather": [vp, i32, vp, vp, sz, vp],
@@ -285,6 +286,10 @@ def strata_moe_dispatch_windows(ctx, layout: strata_moe_layout_t, partition: str
                                 x: int, recv: int, capacity_rows: int, stream: int) -> int:
     return lib().strata_moe_dispatch_windows(ctx, ctypes.byref(layout), ctypes.byref(partition), n_cores, x, recv,
                                              capacity_rows, stream)
+
+
+def strata_ctx_set_sm_budget(ctx, n_sm: int) -> int:
+    return lib().strata_ctx_set_sm_budget(ctx, n_sm)
 
 
 def strata_ctx_set_timeline(ctx, buf: Optional[int], n_ctas: int, events_per_cta: int) -> int:
@@ -551,6 +556,10 @@ class MoEContext:
                 "finish_spread": float(end.max() - end.min()) / total,
                 "wait_in_share": float((used[:, 2] / busy).mean()),
                 "wait_out_share": float((used[:, 3] / busy).mean())}
+
+    def sm_budget(self, n_sm: int) -> None:
+        """Sizes the persistent grids for n_sm SMs (0: the whole GPU)."""
+        _check(strata_ctx_set_sm_budget(self.h, n_sm), "strata_ctx_set_sm_budget")
 
     def timeline(self, n_ctas: int = 2048, events_per_cta: int = 2048, pinned: bool = False):
         """Turns the event timeline on; returns the zeroed buffer [n_ctas, 1 + events_per_cta] (int64), in

@@ -24,7 +24,8 @@ struct strata_region {
 struct strata_ctx {
     strata_moe_shape shape;
     int device;
-    int n_sm;
+    int n_sm;             // SMs the persistent kernels size their grids for (the device's, or the caller's budget)
+    int n_sm_device;
     int* ws;              // device workspace (header + tile counts)
     size_t ws_bytes;
     uint64_t next_region;
@@ -160,6 +161,7 @@ strata_status strata_ctx_create(strata_ctx** out, const strata_moe_shape* shape,
     c->shape = *shape;
     c->device = device;
     c->n_sm = n_sm;
+    c->n_sm_device = n_sm;
     c->ws = nullptr;
     c->ws_bytes = 0;
     c->next_region = 1;
@@ -231,6 +233,14 @@ strata_status strata_ctx_launch_count(strata_ctx* ctx, uint64_t* count)
     if (!ctx || !count) return STRATA_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lk(ctx->mu);
     *count = ctx->launches;
+    return STRATA_OK;
+}
+
+strata_status strata_ctx_set_sm_budget(strata_ctx* ctx, int32_t n_sm)
+{
+    if (!ctx || n_sm < 0) return STRATA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(ctx->mu);
+    ctx->n_sm = (n_sm == 0 || n_sm > ctx->n_sm_device) ? ctx->n_sm_device : n_sm;
     return STRATA_OK;
 }
 

@@ -617,3 +617,40 @@ def test_fixed_capacity_layout(kw, cap, frac):
     assert B.strata_moe_partition(ctx.h, lay.c, pol, 8, part.c, 64, torch.cuda.current_stream().cuda_stream) \
         == B.STRATA_ERR_SHAPE
     ctx.close()
+
+
+@pytest.mark.parametrize("budget", [1, 7, 40])
+def test_sm_budget_changes_no_result(budget):
+    """Persistent grids sized for a few SMs compute the same as grids sized for the whole GPU."""
+    cfg = wl.shrink(wl.CONFIGS["decode"], R=8, T=200, H=1536, E=32, K=4, seed=77)
+    inp = wl.generate(cfg)
+    ref = oracle.layout(inp["ids"], cfg.E)
+    ref_recv = oracle.dispatch_bf16(ref["dst_row"], inp["x"], nthreads=4)
+    ref_out = oracle.combine(ref["dst_row"], ref_recv, inp["w"], nthreads=4)
+    ctx = make_ctx(cfg)
+    ctx.sm_budget(budget)
+    ids_d, x_d, w_d = to_dev(inp["ids"]), to_dev(inp["x"]), to_dev(inp["w"])
+    recv = torch.full((cfg.n_items, cfg.H), SENTINEL16, dtype=torch.int16, device=DEV)
+    out = torch.full((cfg.n_tok, cfg.H), SENTINEL16, dtype=torch.int16, device=DEV)
+    ctx.register(recv)
+    lay = ctx.layout(ids_d)
+    for _ in range(2):                                  # twice: the claim counters re-arm with the smaller grid too
+        ctx.dispatch(lay, x_d, recv)
+        ctx.combine(lay, recv, w_d, out)
+    torch.cuda.synchronize()
+    assert np.array_equal(u16(recv), ref_recv)
+    assert np.array_equal(u16(out), ref_out)
+    # the collectives follow the same budget
+    R, n = 8, 6 * 16384
+    pay = wl.gen_payload(R, R * n // 2, seed=3)
+    x = to_dev(pay)
+    a2a = torch.empty_like(x)
+    red = torch.empty((R, n // 2), dtype=torch.int16, device=DEV)
+    ctx.alltoall(x.view(R, R, n // 2), a2a.view(R, R, n // 2))
+    ctx.reducescatter(a2a.view(R, R, n // 2), red)
+    t = oracle.alltoall(pay.view(np.uint8).reshape(R, R, n)).view(np.uint16).reshape(R, R, n // 2)
+    assert np.array_equal(u16(a2a).reshape(R, R, n // 2), t)
+    assert np.array_equal(u16(red), oracle.reducescatter(t))
+    assert ctx.device_status() == B.STRATA_OK
+    ctx.sm_budget(0)
+    ctx.close()
