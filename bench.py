@@ -473,6 +473,77 @@ def sm_budget_report(cfg: wl.MoEConfig, dev_index: int, budgets=(8, 16, 24, 32, 
     return {"workload": cfg.name, "iters": iters, "rows": rows}
 
 
+def overlap_report(cfg: wl.MoEConfig, dev_index: int, budgets=(0, 64, 32), gemm_n: int = 8192, reps: int = 12):
+    """Interference between the dispatch/combine kernels and a compute kernel on another stream (the paper
+    reports the slowdown of computation under communication, Sec. 2.2).  The co-runner is a library bf16 GEMM
+    (torch.matmul), used only as a load; times are per call, each side looping while the other runs."""
+    case = DeviceCase(cfg, dev_index)
+    torch = case.torch
+    dev = case.dev
+    a = torch.randn((gemm_n, gemm_n), dtype=torch.bfloat16, device=dev)
+    b = torch.randn((gemm_n, gemm_n), dtype=torch.bfloat16, device=dev)
+    c = torch.empty((gemm_n, gemm_n), dtype=torch.bfloat16, device=dev)
+    s_comm, s_gemm = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    case.layout()
+    torch.cuda.synchronize()
+
+    def comm_loop(n):
+        for _ in range(n):
+            case.dispatch()
+            case.combine()
+
+    def gemm_loop(n):
+        for _ in range(n):
+            torch.matmul(a, b, out=c)
+
+    def timed(stream, fn, n):
+        with torch.cuda.stream(stream):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn(n)
+            e1.record()
+        return e0, e1
+
+    for st_, fn in ((s_comm, comm_loop), (s_gemm, gemm_loop)):
+        with torch.cuda.stream(st_):
+            fn(2)
+    torch.cuda.synchronize()
+    e = timed(s_gemm, gemm_loop, reps)
+    torch.cuda.synchronize()
+    gemm_alone = e[0].elapsed_time(e[1]) / reps
+    flops = 2.0 * gemm_n ** 3
+    step_bytes = cfg.dispatch_bytes() + cfg.combine_bytes()
+    rows = []
+    for bud in budgets:
+        case.ctx.sm_budget(bud)
+        with torch.cuda.stream(s_comm):
+            comm_loop(2)
+        torch.cuda.synchronize()
+        e = timed(s_comm, comm_loop, reps)
+        torch.cuda.synchronize()
+        comm_alone = e[0].elapsed_time(e[1]) / reps
+        # both at once; the communication loop is made long enough to cover the GEMM loop and vice versa
+        n_comm = max(reps, int(reps * gemm_alone / comm_alone * 1.5) + 1)
+        n_gemm = max(reps, int(reps * comm_alone / gemm_alone * 1.5) + 1)
+        ec = timed(s_comm, comm_loop, n_comm)
+        eg = timed(s_gemm, gemm_loop, n_gemm)
+        torch.cuda.synchronize()
+        # the shorter loop ran entirely beside the other one: report it, and the slowdown it saw
+        comm_t, gemm_t = ec[0].elapsed_time(ec[1]) / n_comm, eg[0].elapsed_time(eg[1]) / n_gemm
+        rows.append({"sm_budget": bud if bud else "all",
+                     "dispatch+combine_ms_alone": round(comm_alone, 3), "dispatch+combine_ms_beside_gemm": round(comm_t, 3),
+                     "dispatch+combine_GBs_alone": round(step_bytes / comm_alone / 1e6, 1),
+                     "dispatch+combine_GBs_beside_gemm": round(step_bytes / comm_t / 1e6, 1),
+                     "gemm_ms_beside_comm": round(gemm_t, 3), "gemm_TFLOPs_beside_comm": round(flops / gemm_t / 1e9, 1),
+                     "loops": [n_comm, n_gemm]})
+    case.ctx.sm_budget(0)
+    case.check()
+    return {"workload": cfg.name, "gemm": f"bf16 {gemm_n}^3 (library kernel, load only)", "gemm_ms_alone": round(gemm_alone, 3),
+            "gemm_TFLOPs_alone": round(flops / gemm_alone / 1e9, 1),
+            "note": "both loops start together; per-call means include the part of the longer loop that ran alone",
+            "rows": rows}
+
+
 COLLECTIVE_OPS = ("allgather", "alltoall", "alltoallv", "broadcast", "reducescatter", "allreduce")
 
 
@@ -799,6 +870,8 @@ def main():
     ap.add_argument("--timeline-pinned", action="store_true", help="kernels write the events into pinned host memory")
     ap.add_argument("--sm-sweep", action="store_true",
                     help="print only dispatch/combine throughput against the SM budget for --workload")
+    ap.add_argument("--overlap", action="store_true",
+                    help="print only the interference report: dispatch+combine beside a library GEMM on another stream")
     ap.add_argument("--collectives", action="store_true",
                     help="print only the report on the full-mesh collectives (one JSON object; not the bench line)")
     ap.add_argument("--collective-kib", type=int, nargs="+", default=[64, 1024, 16384], help="payload per rank, KiB")
@@ -830,6 +903,10 @@ def main():
             if args.tokens_per_rank:
                 cfg = wl.shrink(cfg, T=args.tokens_per_rank)
             print(json.dumps(sm_budget_report(cfg, local_rank)), flush=True)
+        return
+    if args.overlap:
+        if rank == 0:
+            print(json.dumps(overlap_report(wl.CONFIGS[args.workload], local_rank)), flush=True)
         return
     if args.collectives:
         if rank == 0:
