@@ -167,7 +167,8 @@ strata_status strata_ctx_set_trace(strata_ctx *ctx, uint64_t *dptr, size_t capac
  * timeline is off (buf = NULL, the default).  CTAs with blockIdx >= n_ctas record nothing.
  * Every probed kernel records its CTA lifetime (STRATA_STAGE_KERNEL).  Inside it, per unit of work: the
  * bf16 dispatch and the collectives' copy kernel record WAIT_IN, WORK and WAIT_OUT; combine and the
- * collectives' reduce kernel record WORK; the fp8 and the window-major dispatch record the lifetime only.
+ * collectives' reduce kernel record WORK; the fp8 dispatch records WAIT_OUT, WAIT_IN (including the block
+ * barrier) and WORK (quantise, scales, store issue); the window-major dispatch records the lifetime only.
  * The layout kernels are not probed. */
 typedef enum {
     STRATA_STAGE_KERNEL = 0,     /* the CTA's lifetime inside one launch                        */
