@@ -53,6 +53,8 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).argtypes = [i32, i64, vp, vp]
         L.oracle_broadcast.restype = None
         L.oracle_broadcast.argtypes = [i32, i32, i64, vp, vp]
+        L.oracle_row_experts.restype = None
+        L.oracle_row_experts.argtypes = [i32, i32, i32, vp, vp, vp, i64, vp]
         L.oracle_alltoallv.restype = i64
         L.oracle_alltoallv.argtypes = [i32, i64, i64, vp, vp, vp, vp, vp]
         L.oracle_p2p.restype = None
@@ -111,6 +113,17 @@ def layout(ids: np.ndarray, E: int, segment_align: int = 1, allow_unrouted: bool
         raise BadExpertId(int(-rc - 1))
     out["src_of_row"] = out["src_of_row"][:int(out["expert_offset"][E])]
     out["dropped"] = int(rc) if slot_capacity > 0 else 0
+    return out
+
+
+def row_experts(lay: Dict[str, np.ndarray], R: int, slot_capacity: int = 0) -> np.ndarray:
+    """int32 [rows of the receive buffer]: the expert of every occupied row, -1 for padding and empty rows."""
+    E = lay["expert_count"].shape[0]
+    n_rows = lay["src_of_row"].shape[0]
+    out = np.empty(n_rows, np.int32)
+    lib().oracle_row_experts(R, E, int(slot_capacity), _p(_c(lay["expert_count"], np.int32)),
+                             _p(_c(lay["expert_offset"], np.int32)), _p(_c(lay["src_expert_count"], np.int32)),
+                             n_rows, _p(out))
     return out
 
 

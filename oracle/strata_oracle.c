@@ -539,6 +539,29 @@ void oracle_dispatch_windows(int32_t R, int32_t E, int32_t K, int32_t H, int32_t
 }
 
 /* ------------------------------------------------------------------ */
+/* Row -> expert map of the receive buffer: what a grouped expert GEMM  */
+/* that reads the buffer in place needs per row (this build's reading   */
+/* of "zero staging copy into the expert computation"; the paper names  */
+/* no such array).  row_expert[row] = the expert whose segment holds    */
+/* the row if a token was placed there, -1 for padding and empty rows.  */
+/*  packed / aligned segments: rows offset[e] .. offset[e]+count[e]-1.  */
+/*  fixed capacity C: rows (e*R + r)*C + j for j < src_expert_count[r][e]*/
+/* ------------------------------------------------------------------ */
+void oracle_row_experts(int32_t R, int32_t E, int32_t C, const int32_t *expert_count, const int32_t *expert_offset,
+                        const int32_t *src_expert_count, int64_t n_rows, int32_t *row_expert)
+{
+    for (int64_t j = 0; j < n_rows; ++j) row_expert[j] = -1;
+    for (int32_t e = 0; e < E; ++e) {
+        if (C > 0) {
+            for (int32_t r = 0; r < R; ++r)
+                for (int32_t j = 0; j < src_expert_count[r * E + e]; ++j) row_expert[((int64_t)e * R + r) * C + j] = e;
+        } else {
+            for (int32_t j = 0; j < expert_count[e]; ++j) row_expert[(int64_t)expert_offset[e] + j] = e;
+        }
+    }
+}
+
+/* ------------------------------------------------------------------ */
 /* O6: full-mesh collectives over R emulated ranks (paper Sec. 6.1).    */
 /* Every rank's buffer is one partition of a slab: rank r's input is    */
 /* in[r], its output out[r].  Data-movement operators follow the pull   */

@@ -183,6 +183,7 @@ def test_worked_example_padded_unrouted():
     for key in ("expert_count", "expert_offset", "rank_count", "rank_offset", "src_expert_count", "dst_row",
                 "src_of_row"):
         assert np.array_equal(lay[key].ravel(), rows[key]), key
+    assert np.array_equal(oracle.row_experts(lay, int(R)), rows["row_expert"])
 
 
 @pytest.mark.parametrize("seed", range(8))
@@ -279,6 +280,7 @@ def test_worked_example_fixed_capacity():
                 "src_of_row"):
         assert np.array_equal(lay[key].ravel(), rows[key]), key
     assert lay["dropped"] == rows["dropped"][0]
+    assert np.array_equal(oracle.row_experts(lay, int(R), int(rows["capacity"][0])), rows["row_expert"])
 
 
 @pytest.mark.parametrize("seed", range(6))
@@ -315,3 +317,24 @@ def test_fixed_capacity_matches_brute_force(seed):
     assert np.array_equal(big["expert_count"], oracle.layout(ids, E, allow_unrouted=True)["expert_count"])
     with pytest.raises(ValueError):
         oracle.layout(ids, E, allow_unrouted=True, slot_capacity=C, segment_align=4)
+
+
+@pytest.mark.parametrize("align,cap,frac", [(1, 0, 0.0), (8, 0, 0.15), (1, 5, 0.1), (128, 0, 0.0)])
+def test_row_experts_is_the_id_of_the_item_placed_in_the_row(align, cap, frac):
+    # independent statement: a row's expert is the id of the item that src_of_row names, -1 where nothing was placed
+    rng = np.random.default_rng(align * 10 + cap)
+    R, T, K, E = 4, 37, 3, 8
+    ids = rng.integers(0, E, size=(R, T, K)).astype(np.int32)
+    if frac:
+        ids[rng.uniform(size=ids.shape) < frac] = -1
+    lay = oracle.layout(ids, E, segment_align=align, allow_unrouted=frac > 0, slot_capacity=cap)
+    src = lay["src_of_row"]
+    want = np.where(src >= 0, ids.ravel()[np.maximum(src, 0)], -1)
+    got = oracle.row_experts(lay, R, cap)
+    assert np.array_equal(got, want)
+    for e in range(E):
+        assert (got == e).sum() == lay["expert_count"][e]
+    if align > 1:                                   # every tile of `align` rows belongs to one expert (or is empty)
+        tiles = got.reshape(-1, align)
+        for t in tiles:
+            assert len(set(t[t >= 0].tolist())) <= 1
