@@ -279,6 +279,17 @@ strata_status strata_moe_dispatch(strata_ctx *ctx, const strata_moe_layout_t *la
 strata_status strata_moe_combine(strata_ctx *ctx, const strata_moe_layout_t *layout, const void *y,
                                  size_t y_rows, const float *topk_w, void *out, void *stream);
 
+/* Row -> expert map of the receive buffer (production variant; the paper names no such array): the per-row
+ * group index a grouped expert GEMM needs to read the receive buffer in place, completing the zero-copy
+ * hand-over (with segment_align set to the GEMM's tile height, every tile of rows belongs to one expert or
+ * is empty).  row_expert: device int32 [capacity_rows >= strata_moe_recv_rows]; row_expert[row] = the
+ * expert whose segment holds the row if the layout placed a token there, -1 for the padding of aligned
+ * segments and the empty rows of the fixed-capacity layout (rows beyond strata_moe_recv_rows are not
+ * written).  Reads expert_count and expert_offset (and src_expert_count for the fixed-capacity layout,
+ * where it must be present) as the layout call on the same stream left them.  One launch. */
+strata_status strata_moe_row_experts(strata_ctx *ctx, const strata_moe_layout_t *layout, int32_t *row_expert,
+                                     size_t capacity_rows, void *stream);
+
 /* ---- optional: the paper's hierarchical workload partitioning (Sec. 6.2, App. B to D) -----------
  * The default dispatch balances at run time by ordered work claiming.  These two calls build and run
  * the paper's own static scheme instead, so that it can be compared on this hardware:

@@ -39,7 +39,7 @@ EXPORTS = [
     "strata_moe_roundtrip_host", "strata_moe_layout_noalloc", "strata_ctx_set_trace",
     "strata_moe_partition_max_units", "strata_moe_partition", "strata_moe_dispatch_windows",
     "strata_moe_recv_rows",
-    "strata_ctx_set_timeline", "strata_timeline_decode", "strata_ctx_set_sm_budget",
+    "strata_ctx_set_timeline", "strata_timeline_decode", "strata_ctx_set_sm_budget", "strata_moe_row_experts",
     "strata_allgather", "strata_alltoall", "strata_broadcast", "strata_reducescatter", "strata_allreduce",
     "strata_p2p", "strata_alltoallv",
 ]
@@ -145,6 +145,7 @@ def lib() -> ctypes.CDLL:
                                  P(strata_partition_t), sz, vp],
         "strata_moe_dispatch_windows": [vp, P(strata_moe_layout_t), P(strata_partition_t), i32, vp, vp, sz, vp],
         "strata_ctx_set_sm_budget": [vp, i32],
+        "strata_moe_row_experts": [vp, P(strata_moe_layout_t), vp, sz, vp],
         "strata_ctx_set_timeline": [vp, vp, sz, sz],
         "strata_timeline_decode": [vp, sz, sz, vp, sz, P(sz), P(sz)],
         "strata_allgather": [vp, i32, vp, vp, sz, vp],
@@ -286,6 +287,10 @@ def strata_moe_dispatch_windows(ctx, layout: strata_moe_layout_t, partition: str
                                 x: int, recv: int, capacity_rows: int, stream: int) -> int:
     return lib().strata_moe_dispatch_windows(ctx, ctypes.byref(layout), ctypes.byref(partition), n_cores, x, recv,
                                              capacity_rows, stream)
+
+
+def strata_moe_row_experts(ctx, layout: strata_moe_layout_t, row_expert: int, capacity_rows: int, stream: int) -> int:
+    return lib().strata_moe_row_experts(ctx, ctypes.byref(layout), row_expert, capacity_rows, stream)
 
 
 def strata_ctx_set_sm_budget(ctx, n_sm: int) -> int:
@@ -532,6 +537,15 @@ class MoEContext:
     def combine(self, layout: Layout, y, w, out) -> None:
         _check(strata_moe_combine(self.h, layout.c, y.data_ptr(), y.shape[0], w.data_ptr(), out.data_ptr(),
                                   self._stream()), "strata_moe_combine")
+
+    def row_experts(self, layout: Layout, out=None):
+        """int32 [recv_rows]: the expert of every occupied receive row, -1 for padding and empty rows."""
+        import torch
+        if out is None:
+            out = torch.empty((self.recv_rows,), dtype=torch.int32, device=self.device)
+        _check(strata_moe_row_experts(self.h, layout.c, out.data_ptr(), out.shape[0], self._stream()),
+               "strata_moe_row_experts")
+        return out
 
     def trace(self, capacity_ctas: int = 4096):
         """Turns per-CTA probes on; returns the tensor [capacity, 4] = (start_ns, end_ns, wait_in_ns, wait_out_ns)."""

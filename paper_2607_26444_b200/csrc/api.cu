@@ -457,6 +457,28 @@ strata_status strata_moe_combine(strata_ctx* ctx, const strata_moe_layout_t* lay
     return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
 }
 
+strata_status strata_moe_row_experts(strata_ctx* ctx, const strata_moe_layout_t* layout, int32_t* row_expert,
+                                     size_t capacity_rows, void* stream)
+{
+    if (!ctx || !row_expert) return STRATA_ERR_INVALID_ARG;
+    strata_status st = check_layout_ptrs(layout, true);
+    if (st != STRATA_OK) return st;
+    const strata_moe_shape& s = ctx->shape;
+    if (s.slot_capacity > 0 && !layout->src_expert_count) return STRATA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(row_expert) & 3u) != 0) return STRATA_ERR_ALIGNMENT;
+    const size_t n_rows = (size_t)recv_rows(s);
+    if (capacity_rows < n_rows) return STRATA_ERR_CAPACITY;
+    if (ctx->device < 0) return STRATA_ERR_CUDA;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return STRATA_ERR_CUDA;
+    cudaError_t err = launch_row_experts(s, *layout, row_expert, (long long)n_rows, static_cast<cudaStream_t>(stream));
+    {
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        ctx->launches += 1;
+    }
+    return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
+}
+
 namespace {
 strata_status check_policy(const strata_moe_shape& s, const strata_partition_policy* pol)
 {

@@ -654,3 +654,57 @@ def test_sm_budget_changes_no_result(budget):
     assert ctx.device_status() == B.STRATA_OK
     ctx.sm_budget(0)
     ctx.close()
+
+
+@pytest.mark.parametrize("kw,align,cap,frac", [
+    (dict(R=4, T=128, H=64, E=16, K=2), 0, 0, 0.0),                 # packed
+    (dict(R=4, T=300, H=64, E=16, K=4), 128, 0, 0.1),               # GEMM-tile-aligned segments, unrouted slots
+    (dict(R=8, T=1500, H=64, E=32, K=4), 64, 0, 0.0),               # tiled layout path
+    (dict(R=16, T=128, H=64, E=256, K=8), 0, 16, 0.0),              # decode shape, fixed capacity
+    (dict(R=2, T=60, H=64, E=4, K=3), 0, 7, 0.2),
+    (dict(R=1, T=5, H=64, E=1024, K=1), 8, 0, 0.0),                 # more experts than rows
+], ids=lambda v: str(v) if not isinstance(v, dict) else "R{R}T{T}E{E}K{K}".format(**v))
+def test_row_experts(kw, align, cap, frac):
+    cfg = wl.shrink(wl.CONFIGS["tiny"], seed=321, **kw)
+    inp = wl.generate(cfg)
+    ids = inp["ids"].copy()
+    if frac:
+        rng = np.random.default_rng(5)
+        ids[rng.uniform(size=ids.shape) < frac] = -1
+    ref = oracle.layout(ids, cfg.E, segment_align=max(1, align), allow_unrouted=frac > 0, slot_capacity=cap)
+    want = oracle.row_experts(ref, cfg.R, cap)
+    ctx = B.MoEContext(cfg.R, cfg.T, cfg.H, cfg.E, cfg.K, segment_align=align, allow_unrouted=frac > 0,
+                       slot_capacity=cap)
+    lay = ctx.layout(to_dev(ids))
+    whole = torch.full((ctx.recv_rows + 2 * GUARD,), -7, dtype=torch.int32, device=DEV)
+    got = ctx.row_experts(lay, whole[GUARD:GUARD + ctx.recv_rows])
+    torch.cuda.synchronize()
+    h = whole.cpu().numpy()
+    assert np.all(h[:GUARD] == -7) and np.all(h[-GUARD:] == -7)
+    g = got.cpu().numpy()                            # the oracle's arrays end at expert_offset[E]; the buffer may be longer
+    assert want.shape[0] <= ctx.recv_rows
+    assert np.array_equal(g[:want.shape[0]], want) and np.all(g[want.shape[0]:] == -1)
+    if cap:
+        ctx.device_status()                          # CAPACITY is raised when slots overflow: expected here
+    else:
+        assert ctx.device_status() == B.STRATA_OK
+    ctx.close()
+
+
+def test_row_experts_full_prefill_shape():
+    cfg = wl.CONFIGS["prefill"]
+    ids = wl.gen_topk_ids(cfg)
+    ctx = B.MoEContext(cfg.R, cfg.T, cfg.H, cfg.E, cfg.K, segment_align=128)
+    lay = ctx.layout(to_dev(ids))
+    got = ctx.row_experts(lay).cpu().numpy()
+    ref = oracle.layout(ids, cfg.E, segment_align=128)
+    want = oracle.row_experts(ref, cfg.R)
+    assert np.array_equal(got[:want.shape[0]], want) and np.all(got[want.shape[0]:] == -1)
+    # every 128-row tile belongs to one expert or is empty, and occupied rows carry the id of their item
+    tiles = got.reshape(-1, 128)
+    first = tiles[:, :1]
+    assert np.all((tiles == first) | (tiles == -1))
+    src = lay.src_of_row.cpu().numpy()[:want.shape[0]]
+    occ = src >= 0
+    assert np.array_equal(got[:want.shape[0]][occ], ids.ravel()[src[occ]]) and np.all(got[:want.shape[0]][~occ] == -1)
+    ctx.close()
