@@ -224,7 +224,7 @@ strata_status strata_pool_reset(strata_ctx *ctx, uint64_t region_id);
  * (dst_row = -1, not counted) and raises BAD_EXPERT_ID on the device status
  * (except -1 under STRATA_FLAG_ALLOW_UNROUTED, which is legal).
  * Needs a workspace.  One kernel launch for up to 32,768 items, two beyond
- * (and always two for the fixed-capacity layout). */
+ * (fixed-capacity layout: one launch while T*K <= 4096, else two). */
 strata_status strata_moe_layout(strata_ctx *ctx, const int32_t *topk_ids,
                                 const strata_moe_layout_t *layout, void *stream);
 

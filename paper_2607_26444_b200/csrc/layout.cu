@@ -545,6 +545,137 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_cluster_kernel(LayoutPa
     cluster.sync();                       // no CTA leaves while another may still read its shared memory
 }
 
+// ---- fixed-capacity layout of small batches: one launch, one CTA per source rank ---------------
+// In the [E][R][C] layout a row depends only on the items of the same source rank (the index of an
+// item inside its (expert, rank) slot), and the offsets are constants, so the ranks are independent:
+// CTA r counts and ranks the T*K <= 4096 items of rank r entirely in shared memory, fills its own
+// slots of src_of_row (placed items and -1 for the empty rows), and leaves its clamped counts in the
+// workspace; the CTA that draws the last ticket adds them up over the ranks.  Nothing waits.
+__global__ void __launch_bounds__(kLayoutThreads) layout_capacity_kernel(LayoutParams p)
+{
+    extern __shared__ int sm[];          // warp_cnt[32*E] | kept[E]
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int E = p.E, C = p.capacity, r = blockIdx.x;
+    int* warp_cnt = sm;
+    int* kept = sm + 32 * E;
+    int* mine = warp_cnt + wid * E;
+    const int ebits = key_bits(E);
+    const long long rank_base = (long long)r * p.items_per_rank;
+    const int warp_first = wid * kWarpItems;
+
+    for (int x = tid; x < 32 * E; x += kLayoutThreads) warp_cnt[x] = 0;
+    griddep_wait();
+    griddep_launch_dependents();
+    int ids[kItemsPerThread];
+#pragma unroll
+    for (int q = 0; q < kItemsPerThread; ++q) {
+        const int in_rank = warp_first + q * 32 + lane;
+        ids[q] = in_rank < p.items_per_rank ? p.ids[rank_base + in_rank] : -1;
+    }
+    __syncthreads();
+
+    // pass 1: per-warp counts
+#pragma unroll
+    for (int q = 0; q < kItemsPerThread; ++q) {
+        const int in_rank = warp_first + q * 32 + lane;
+        bool valid = in_rank < p.items_per_rank;
+        int e = ids[q];
+        if (valid && (unsigned)e >= (unsigned)E) {
+            if (!(p.allow_unrouted && e == -1)) report_status(p.status, STRATA_ERR_BAD_EXPERT_ID);
+            valid = false;
+        }
+        if (!valid) e = -1;
+        ids[q] = e;
+        const unsigned peers = same_key_lanes(e, ebits);
+        if (valid && lane == __ffs(peers) - 1) mine[e] += __popc(peers);
+        __syncwarp();
+    }
+    __syncthreads();
+    // exclusive prefix over the 32 warps per expert; the total is this rank's count for the expert
+    for (int x = tid; x < E; x += kLayoutThreads) {
+        int running = 0;
+#pragma unroll 8
+        for (int w = 0; w < 32; ++w) {
+            const int c = warp_cnt[w * E + x];
+            warp_cnt[w * E + x] = running;
+            running += c;
+        }
+        const int k = min(running, C);
+        if (running > C) report_status(p.status, STRATA_ERR_CAPACITY);       // items beyond the capacity are dropped
+        kept[x] = k;
+        p.tile_cnt[(size_t)r * E + x] = k;
+        if (p.src_expert_count) p.src_expert_count[(size_t)r * E + x] = k;
+    }
+    __syncthreads();
+
+    // pass 2: rows.  mine[e] counts the same-id items of earlier warps and earlier rounds of this rank.
+    const unsigned lt = (1u << lane) - 1u;
+#pragma unroll
+    for (int q = 0; q < kItemsPerThread; ++q) {
+        const int in_rank = warp_first + q * 32 + lane;
+        const int e = ids[q];
+        const bool valid = e >= 0;
+        const unsigned peers = same_key_lanes(e, ebits);
+        const int leader = __ffs(peers) - 1;
+        int old = 0;
+        if (valid && lane == leader) {
+            old = mine[e];
+            mine[e] = old + __popc(peers);
+        }
+        old = __shfl_sync(0xffffffffu, old, leader);
+        if (valid) {
+            const int idx = old + __popc(peers & lt);
+            const int row = idx < C ? (e * p.R + r) * C + idx : -1;
+            p.dst_row[rank_base + in_rank] = row;
+            if (p.src_of_row && row >= 0) p.src_of_row[row] = (int32_t)(rank_base + in_rank);
+        } else if (in_rank < p.items_per_rank) {
+            p.dst_row[rank_base + in_rank] = -1;
+        }
+        __syncwarp();
+    }
+    // the empty rows of this rank's slots
+    if (p.src_of_row)
+        for (int x = tid; x < E * C; x += kLayoutThreads) {
+            const int e = x / C, j = x - e * C;
+            if (j >= kept[e]) p.src_of_row[(size_t)(e * p.R + r) * C + j] = -1;
+        }
+
+    // ---- last CTA to finish adds the ranks up (a ticket, never a wait) ----
+    __shared__ int s_last;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = (atomicAdd(p.ticket, 1) == p.R - 1);
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    int* sum_e = warp_cnt;                // reused: [E]
+    for (int x = tid; x < E; x += kLayoutThreads) {
+        int sum = 0;
+        for (int r0 = 0; r0 < p.R; r0 += 8) {
+            int v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = (r0 + i < p.R) ? __ldcg(p.tile_cnt + (size_t)(r0 + i) * E + x) : 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) sum += v[i];
+        }
+        sum_e[x] = sum;
+        p.expert_count[x] = sum;
+        p.expert_offset[x] = x * p.R * C;
+    }
+    if (tid == 0) {
+        p.expert_offset[E] = E * p.R * C;
+        p.rank_offset[p.R] = E * p.R * C;
+    }
+    __syncthreads();
+    for (int d = tid; d < p.R; d += kLayoutThreads) {
+        int real = 0;
+        for (int e2 = d * p.e_loc; e2 < (d + 1) * p.e_loc; ++e2) real += sum_e[e2];
+        p.rank_count[d] = real;
+        p.rank_offset[d] = d * p.e_loc * p.R * C;
+    }
+    if (tid == 0) *p.ticket = 0;          // ready for the next call on this stream
+}
+
 // shared memory of the cluster kernel; the per-source-rank table is only there when asked for
 size_t small_smem(int E, int R, bool with_src)
 {
@@ -564,6 +695,9 @@ cudaError_t configure_layout_kernels()
 {
     cudaError_t err = cudaFuncSetAttribute(layout_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            32 * kMaxExperts * (int)sizeof(int));
+    if (err != cudaSuccess) return err;
+    err = cudaFuncSetAttribute(layout_capacity_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               33 * kMaxExperts * (int)sizeof(int));
     if (err != cudaSuccess) return err;
     return cudaFuncSetAttribute(layout_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)kSmallSmemLimit);
@@ -597,12 +731,17 @@ cudaError_t launch_layout(const strata_moe_shape& s, const int32_t* ids, const s
 
     const long long n_items = (long long)s.R * s.T * s.K;
     const size_t small_bytes = small_smem(s.E, s.R, L.src_expert_count != nullptr);
-    // the fixed-capacity layout needs per-source-rank prefixes, which only the tiled path keeps
+    // the fixed-capacity layout ranks items per source rank: its own one-launch kernel below when a rank
+    // fits one tile, else the tiled path
     if (p.capacity == 0 && n_items <= (long long)kSmallItems * kLayoutCluster && small_bytes <= kSmallSmemLimit) {
         const unsigned n_cta = n_items <= kSmallItems ? 1u : (unsigned)kLayoutCluster;
         *n_launches = 1;
         return launch_pdl_cluster(layout_cluster_kernel, n_cta, kLayoutThreads, small_bytes, n_cta, st, p,
                                   (int)n_items);
+    }
+    if (p.capacity > 0 && g.tiles_per_rank == 1) {
+        *n_launches = 1;
+        return launch_pdl(layout_capacity_kernel, (unsigned)s.R, kLayoutThreads, (size_t)33 * s.E * sizeof(int), st, p);
     }
     *n_launches = 2;
     cudaError_t err = launch_pdl(layout_count_scan_kernel, (unsigned)g.n_tiles, kLayoutThreads, count_scan_smem(s.E), st, p);

@@ -581,6 +581,9 @@ def test_cuda_graph_replay(kw):
     (dict(R=16, T=128, H=7168, E=256, K=8), 16, 0.0),             # decode shape, static [256][16][16] buffer
     (dict(R=8, T=1500, H=128, E=32, K=4), 200, 0.2),              # several tiles per rank, unrouted slots
     (dict(R=2, T=60, H=64, E=4, K=3), 1000, 0.0),                 # capacity nobody reaches
+    (dict(R=1, T=100, H=64, E=1024, K=8), 3, 0.0),                # one rank, the largest expert table
+    (dict(R=64, T=64, H=64, E=64, K=1), 2, 0.1),                  # many ranks, one item per token
+    (dict(R=4, T=1024, H=64, E=16, K=4), 300, 0.0),               # a rank fills its tile exactly (4096 items)
 ], ids=lambda v: str(v) if not isinstance(v, dict) else "R{R}T{T}H{H}E{E}K{K}".format(**v))
 def test_fixed_capacity_layout(kw, cap, frac):
     cfg = wl.shrink(wl.CONFIGS["tiny"], seed=555, **kw)
