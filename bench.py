@@ -308,6 +308,15 @@ def per_call_us(case: DeviceCase, iters: int = 30, warmup: int = 3):
         torch.cuda.synchronize()
         ts = sorted(ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(iters))
         out[name] = {"median_us": ts[len(ts) // 2], "min_us": ts[0], "p95_us": ts[int(0.95 * (len(ts) - 1))]}
+        # the same calls with no event between them (an event record between two short kernels adds to both
+        # and keeps the next launch from overlapping the tail of the previous kernel; events tick in ~2 us steps)
+        torch.cuda._sleep(10_000_000)
+        ev[0].record()
+        for i in range(iters):
+            fn()
+        ev[1].record()
+        torch.cuda.synchronize()
+        out[name]["back_to_back_us"] = ev[0].elapsed_time(ev[1]) * 1e3 / iters
     # the same three calls captured once in a CUDA graph and replayed (launch overhead paid once)
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
@@ -784,6 +793,7 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
                 "dispatch_GBs": round(db / us["dispatch"]["median_us"] / 1e3, 1),
                 "combine_GBs": round(cb / us["combine"]["median_us"] / 1e3, 1),
                 "min_p95_us": {k: [round(v["min_us"], 2), round(v["p95_us"], 2)] for k, v in us.items()},
+                "back_to_back_us": {k: round(v["back_to_back_us"], 2) for k, v in us.items() if "back_to_back_us" in v},
                 "iters": 30,
             }
             if name == "skew":
