@@ -711,3 +711,30 @@ def test_row_experts_full_prefill_shape():
     occ = src >= 0
     assert np.array_equal(got[:want.shape[0]][occ], ids.ravel()[src[occ]]) and np.all(got[:want.shape[0]][~occ] == -1)
     ctx.close()
+
+
+def test_fixed_capacity_with_e4m3_dispatch():
+    """The low-latency pairing: static [E][R][C] receive buffer, e4m3 payload with per-128-column scales."""
+    cfg = wl.shrink(wl.CONFIGS["fp8"], R=8, T=96, H=1024, E=32, K=4, seed=909)
+    cap = 20
+    inp = wl.generate(cfg)
+    ref = oracle.layout(inp["ids"], cfg.E, slot_capacity=cap)
+    ctx = B.MoEContext(cfg.R, cfg.T, cfg.H, cfg.E, cfg.K, cfg.dispatch_dtype, slot_capacity=cap)
+    n_rows = ctx.recv_rows
+    lay = ctx.layout(to_dev(inp["ids"]))
+    whole_q, recv_q = guarded(n_rows, cfg.H, torch.uint8, 0x7F)
+    whole_s, recv_s = guarded(n_rows, cfg.H // 128, torch.float32, -1.0)
+    ctx.register(whole_q)
+    ctx.register(whole_s)
+    ctx.dispatch(lay, to_dev(inp["x"]), recv_q, recv_s)
+    torch.cuda.synchronize()
+    q, s = oracle.dispatch_fp8(ref["dst_row"], inp["x"], n_rows=n_rows)
+    used = ref["src_of_row"] >= 0
+    assert used.sum() == (ref["dst_row"] >= 0).sum() > 0
+    gq, gs = recv_q.cpu().numpy(), recv_s.cpu().numpy()
+    assert np.array_equal(gq[used], q[used]) and np.all(gq[~used] == 0x7F)
+    assert np.array_equal(gs[used].view(np.uint32), s[used].view(np.uint32)) and np.all(gs[~used] == -1.0)
+    assert np.all(whole_q.cpu().numpy()[:GUARD] == 0x7F) and np.all(whole_s.cpu().numpy()[-GUARD:] == -1.0)
+    st = ctx.device_status()
+    assert st == (B.STRATA_ERR_CAPACITY if ref["dropped"] else B.STRATA_OK)
+    ctx.close()
