@@ -28,6 +28,10 @@ CASES = [
     (dict(R=32, T=512, H=4096, E=128, K=8, routing="zipf"), [(200, 1024, 128, 6), (700, 800, 96, 4)], 8, 8, 444),
     (dict(R=3, T=50, H=64, E=6, K=3), [(0, 1, 1000000, 1)], 1, 1, 5),                   # one unit per peer window, cap 1
     (dict(R=2, T=700, H=128, E=4, K=2), [(5, 16, 3, 1000)], 1, 1, 1000),                # more cores than needed
+    (dict(R=16, T=128, H=7168, E=256, K=8), [(200, 1024, 64, 296)], 1, 1, 296),        # a cap that cannot bind: register-min loop
+    (dict(R=32, T=512, H=4096, E=128, K=8, routing="zipf"), [(1000, 22, 64, 300), (700, 20, 96, 500)], 8, 8, 296),
+    (dict(R=8, T=256, H=2048, E=32, K=4), [(900000, 1, 32, 64)], 1, 1, 64),            # loads leave the 21-bit keys mid-run
+    (dict(R=4, T=128, H=1024, E=16, K=2), [(10, 64, 16, 33)], 1, 1, 33),               # 33 cores: two cores on lane 0
 ]
 
 
