@@ -738,3 +738,31 @@ def test_fixed_capacity_with_e4m3_dispatch():
     st = ctx.device_status()
     assert st == (B.STRATA_ERR_CAPACITY if ref["dropped"] else B.STRATA_OK)
     ctx.close()
+
+
+def test_usage_with_bfloat16_tensors_against_torch_ops():
+    """The calls as a torch user makes them (bfloat16 tensors), cross-checked with plain torch ops:
+    dispatch is an index copy, combine a weighted sum in fp32 (within 1 bf16 ulp of torch's own order)."""
+    R, T, H, E, K = 4, 96, 512, 16, 4
+    g = torch.Generator(device=DEV).manual_seed(5)
+    x = torch.randn((R, T, H), generator=g, device=DEV).to(torch.bfloat16)
+    ids = torch.stack([torch.randperm(E, generator=g, device=DEV)[:K] for _ in range(R * T)]).view(R, T, K).to(torch.int32)
+    w = torch.softmax(torch.randn((R, T, K), generator=g, device=DEV), dim=-1)
+    ctx = B.MoEContext(R, T, H, E, K)
+    recv = torch.zeros((ctx.recv_rows, H), dtype=torch.bfloat16, device=DEV)
+    ctx.register(recv)
+    lay = ctx.layout(ids)
+    ctx.dispatch(lay, x, recv)
+    rows = lay.dst_row.view(-1).long()
+    src = x.view(R * T, H).repeat_interleave(K, dim=0)
+    assert torch.equal(recv[rows], src)                              # every item's row holds its token
+    order = torch.argsort(ids.view(-1).long() * (R * T * K) + torch.arange(R * T * K, device=DEV))
+    assert torch.equal(rows[order], torch.arange(R * T * K, device=DEV))   # expert, then item order
+    y = (recv.float() * 1.5).to(torch.bfloat16)
+    out = torch.empty((R, T, H), dtype=torch.bfloat16, device=DEV)
+    ctx.combine(lay, y, w, out)
+    want = (y[rows].float().view(R * T, K, H) * w.view(R * T, K, 1)).sum(dim=1).to(torch.bfloat16).view(R, T, H)
+    a, b = out.view(torch.int16).cpu().numpy().view(np.uint16), want.view(torch.int16).cpu().numpy().view(np.uint16)
+    assert ulp_distance(a, b).max() <= 1
+    assert ctx.device_status() == B.STRATA_OK
+    ctx.close()
