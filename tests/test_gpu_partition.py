@@ -32,6 +32,10 @@ CASES = [
     (dict(R=32, T=512, H=4096, E=128, K=8, routing="zipf"), [(1000, 22, 64, 300), (700, 20, 96, 500)], 8, 8, 296),
     (dict(R=8, T=256, H=2048, E=32, K=4), [(900000, 1, 32, 64)], 1, 1, 64),            # loads leave the 21-bit keys mid-run
     (dict(R=4, T=128, H=1024, E=16, K=2), [(10, 64, 16, 33)], 1, 1, 33),               # 33 cores: two cores on lane 0
+    (dict(R=16, T=1024, H=512, E=64, K=4), [(1000, 22, 32, 296)], 1, 1, 296),           # long runs of equal-cost units: rounds
+    (dict(R=16, T=1024, H=512, E=64, K=4), [(1000, 22, 32, 100), (1, 22, 16, 100)], 4, 4, 100),   # two tiers, two long runs
+    (dict(R=8, T=2048, H=256, E=32, K=2), [(7, 64, 8, 40)], 1, 1, 40),                  # many rounds on few cores
+    (dict(R=16, T=1024, H=512, E=64, K=4), [(0, 1 << 40, 32, 64)], 1, 1, 64),           # every unit costs 1
 ]
 
 
