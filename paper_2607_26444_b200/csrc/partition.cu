@@ -9,7 +9,8 @@
 //            issue stripe still has room for the unit's destination rank (fan-out cap H_t); the output
 //            is one task list per core, which the window-major dispatch kernel simply follows.
 // The policy is generated ON the GPU by one CTA (no host round trip): a bitonic sort of the units and a
-// sequential greedy loop whose "least-loaded feasible core" step is a block-wide arg-min.
+// greedy loop run by one warp, whose "least-loaded feasible core" step is a warp-wide arg-min; where the
+// fan-out cap cannot bind, runs of equal-cost units are handed out in closed-form rounds.
 #include "common.cuh"
 
 namespace strata {
@@ -18,7 +19,7 @@ namespace {
 
 constexpr int kPartThreads = 1024;
 constexpr int kPartMaxUnits = 8192;       // sort keys live in shared memory
-constexpr int kPartMaxCores = 1024;       // one thread per core in the arg-min
+constexpr int kPartMaxCores = 1024;       // core ids take 10 bits of the arg-min keys
 constexpr int kFanSmemInts = 12288;       // fan-out counts F[stripe][dest] kept in shared memory
 constexpr int kMaxTiers = 3;
 
