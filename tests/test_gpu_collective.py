@@ -356,3 +356,44 @@ def test_p2p(ctx, R, n, src, dst):
     oracle.p2p(x, want, src, dst)
     assert np.array_equal(out.cpu().numpy().reshape(R, n), want)
     assert guards_intact(whole)
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_shapes_all_operators(ctx, seed):
+    """Random rank counts and sizes (any multiple of 16 bytes / 8 elements), every operator against the oracle."""
+    rng = np.random.default_rng(1000 + seed)
+    R = int(rng.integers(1, 33))
+    n = int(rng.integers(1, 6000)) * 16                     # bytes per slice, up to 96 KB
+    S = n // 2                                              # bf16 elements per slice
+    xb = payload_bytes(R, R * n, seed=seed).reshape(R, R, n)
+    x_d = torch.from_numpy(xb).to(DEV)
+    out = torch.empty((R, R, n), dtype=torch.uint8, device=DEV)
+    ctx.alltoall(x_d, out)
+    assert np.array_equal(out.cpu().numpy(), oracle.alltoall(xb))
+    small = np.ascontiguousarray(xb[:, 0, :])               # [R, n]
+    ag = torch.empty((R, R, n), dtype=torch.uint8, device=DEV)
+    ctx.allgather(torch.from_numpy(small).to(DEV), ag)
+    assert np.array_equal(ag.cpu().numpy(), oracle.allgather(small))
+    root = int(rng.integers(0, R))
+    bc = torch.empty((R, n), dtype=torch.uint8, device=DEV)
+    ctx.broadcast(torch.from_numpy(small).to(DEV), bc, root)
+    assert np.array_equal(bc.cpu().numpy(), oracle.broadcast(small, root))
+    xs = xb.view(np.uint16).reshape(R, R, S)
+    # finite operands: clear the top exponent bit
+    xs = (xs & np.uint16(0xBFFF)).astype(np.uint16)
+    xs_d = torch.from_numpy(xs.view(np.int16)).to(DEV)
+    rs = torch.empty((R, S), dtype=torch.int16, device=DEV)
+    ctx.reducescatter(xs_d, rs)
+    assert np.array_equal(rs.cpu().numpy().view(np.uint16), oracle.reducescatter(xs))
+    ar = torch.empty((R, R * S), dtype=torch.int16, device=DEV)
+    ctx.allreduce(xs_d.view(R, R * S), ar)
+    assert np.array_equal(ar.cpu().numpy().view(np.uint16), oracle.allreduce(xs.reshape(R, R * S)))
+    sb = wl.gen_pair_bytes(R, max(16, n // 4), seed=seed, skew=float(rng.uniform(0.0, 2.0)),
+                           zero_frac=float(rng.uniform(0.0, 0.5)))
+    so, ro, si, st = wl.packed_offsets(sb)
+    xv = payload_bytes(R, si, seed=seed + 500)             # si is a multiple of 16
+    got = run_alltoallv(ctx, xv, sb, so, ro, st)
+    want = np.full((R, st), 0xEE, np.uint8)
+    assert oracle.alltoallv(xv, want, sb, so, ro) == 0
+    assert np.array_equal(got, want)
+    assert ctx.device_status() == B.STRATA_OK
