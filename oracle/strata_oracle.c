@@ -32,6 +32,8 @@
  * for the partitioning: exact cover of the receive rows, Graham's tight LPT
  * example, the 4/3 - 1/(3C) bound against a brute-force optimum, the fan-out
  * cap, and equality of window-major with token-major dispatch.
+ * The row -> expert map: the worked examples and "a row's expert is the id of
+ * the item src_of_row names".
  * For the full-mesh collectives (tests/test_oracle_collectives.py): counter
  * patterns with closed-form results, the involution of all-to-all, exact
  * integer sums, a hand-worked order-sensitive sum, all-reduce = reduce-scatter
