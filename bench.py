@@ -425,6 +425,7 @@ def window_partitioning_report(cfg: wl.MoEConfig, dev_index: int, unit_rows: int
 def timeline_report(cfg: wl.MoEConfig, dev_index: int, trace_path: str = "", pinned: bool = False):
     """One step with the in-kernel event timeline on (paper Sec. 6.4): per kernel the CTA count, wall time,
     finish-time spread and the share of CTA time per stage.  Probes cost time: these are not bench numbers."""
+    from paper_2607_26444_b200 import timeline as TL
     case = DeviceCase(cfg, dev_index)
     torch, B = case.torch, case.B
     for _ in range(3):
@@ -438,7 +439,7 @@ def timeline_report(cfg: wl.MoEConfig, dev_index: int, trace_path: str = "", pin
     case.ctx.timeline_off()
     case.check()
     rep = {"workload": cfg.name, "buffer": "pinned host" if pinned else "device", "events_per_cta": cap,
-           "spans": int(spans.size), "events_dropped": int(dropped), "kernels": B.timeline_summary(spans)}
+           "spans": int(spans.size), "events_dropped": int(dropped), "kernels": TL.timeline_summary(spans)}
     for k in rep["kernels"].values():
         k["wall_us"] = round(k["wall_us"], 2)
         k["finish_spread"] = round(k["finish_spread"], 4)
@@ -447,7 +448,7 @@ def timeline_report(cfg: wl.MoEConfig, dev_index: int, trace_path: str = "", pin
             st["share_of_cta_time"] = round(st["share_of_cta_time"], 4)
             st["mean_ns"] = round(st["mean_ns"], 1)
     if trace_path:
-        rep["chrome_trace_events"] = B.timeline_chrome_trace(spans, trace_path, max_ctas=32)
+        rep["chrome_trace_events"] = TL.timeline_chrome_trace(spans, trace_path, max_ctas=32)
     return rep
 
 

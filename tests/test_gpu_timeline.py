@@ -6,6 +6,7 @@ import torch
 
 import oracle
 from paper_2607_26444_b200 import binding as B
+from paper_2607_26444_b200 import timeline as TL
 from paper_2607_26444_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -68,7 +69,7 @@ def test_step_timeline(pinned):
     # combine started after dispatch ended (stream order)
     assert comb["begin_ns"].min() >= disp[disp["stage"] == KERNEL]["end_ns"].max()
 
-    s = B.timeline_summary(spans)
+    s = TL.timeline_summary(spans)
     assert s["dispatch_bf16"]["ctas"] == life.size
     assert 0.0 < s["dispatch_bf16"]["stages"]["wait_in"]["share_of_cta_time"] < 1.0
     assert 0.0 <= s["dispatch_bf16"]["finish_spread"] <= 1.0
@@ -89,7 +90,7 @@ def test_small_slices_count_what_they_drop_and_stay_inside():
     B.strata_ctx_set_timeline(ctx.h, None, 0, 0)
     h = whole.cpu().numpy()
     assert np.all(h[0] == -1) and np.all(h[-1] == -1)                    # neighbours untouched
-    spans, dropped = B.decode_timeline(h[1:-1].view(np.uint64))
+    spans, dropped = TL.decode_timeline(h[1:-1].view(np.uint64))
     assert dropped > 0
     assert np.all(h[1:-1, 0] >= cap)                                     # every slice was filled and kept counting
     assert spans["cta"].max() < n_ctas
