@@ -487,48 +487,9 @@ class MoEContext:
 
     @staticmethod
     def trace_summary(trace) -> dict:
-        """Decodes a trace tensor after a launch: kernel time, finish-time spread and stage shares."""
-        import numpy as np
-        rec = trace.cpu().numpy()
-        used = rec[rec[:, 0] != 0]
-        if used.shape[0] == 0:
-            return {"ctas": 0}
-        start, end = used[:, 0], used[:, 1]
-        total = float(end.max() - start.min())
-        busy = (end - start).astype(np.float64)
-        return {"ctas": int(used.shape[0]), "kernel_us": total / 1e3,
-                "finish_spread": float(end.max() - end.min()) / total,
-                "wait_in_share": float((used[:, 2] / busy).mean()),
-                "wait_out_share": float((used[:, 3] / busy).mean())}
-
-    def sm_budget(self, n_sm: int) -> None:
-        """Sizes the persistent grids for n_sm SMs (0: the whole GPU)."""
-        _check(strata_ctx_set_sm_budget(self.h, n_sm), "strata_ctx_set_sm_budget")
-
-    def timeline(self, n_ctas: int = 2048, events_per_cta: int = 2048, pinned: bool = False):
-        """Turns the event timeline on; returns the zeroed buffer [n_ctas, 1 + events_per_cta] (int64), in
-        device memory or, with pinned=True, in page-locked host memory that the kernels write in place."""
-        import torch
-        if pinned:
-            t = torch.zeros((n_ctas, 1 + events_per_cta), dtype=torch.int64, pin_memory=True)
-        else:
-            t = torch.zeros((n_ctas, 1 + events_per_cta), dtype=torch.int64, device=self.device)
-        torch.cuda.synchronize(self.device)
-        _check(strata_ctx_set_timeline(self.h, t.data_ptr(), n_ctas, events_per_cta), "strata_ctx_set_timeline")
-        self._timeline = t
-        return t
-
-    def timeline_off(self) -> None:
-        _check(strata_ctx_set_timeline(self.h, None, 0, 0), "strata_ctx_set_timeline")
-        self._timeline = None
-
-    @staticmethod
-    def timeline_spans(t):
-        """Synchronises and decodes a timeline buffer; returns (spans, dropped)."""
-        import torch
-        from .timeline import decode_timeline
-        torch.cuda.synchronize()
-        return decode_timeline(t.cpu().numpy().view("uint64"))
+        """Decodes a trace tensor after a launch (see timeline.trace_summary)."""
+        from .timeline import trace_summary
+        return trace_summary(trace.cpu().numpy())
 
     def trace_off(self) -> None:
         _check(strata_ctx_set_trace(self.h, None, 0), "strata_ctx_set_trace")

@@ -79,3 +79,19 @@ def timeline_chrome_trace(spans, path: str, max_ctas: int = 64) -> int:
     with open(path, "w") as f:
         json.dump({"traceEvents": ev, "displayTimeUnit": "ns"}, f)
     return len(ev)
+
+
+def trace_summary(rec) -> dict:
+    """rec: numpy int64 [capacity, 4] = (start_ns, end_ns, wait_in_ns, wait_out_ns) per CTA, as the per-CTA
+    stage probes leave it: kernel time, finish-time spread and the shares of the two waits."""
+    import numpy as np
+    used = rec[rec[:, 0] != 0]
+    if used.shape[0] == 0:
+        return {"ctas": 0}
+    start, end = used[:, 0], used[:, 1]
+    total = float(end.max() - start.min())
+    busy = (end - start).astype(np.float64)
+    return {"ctas": int(used.shape[0]), "kernel_us": total / 1e3,
+            "finish_spread": float(end.max() - end.min()) / total,
+            "wait_in_share": float((used[:, 2] / busy).mean()),
+            "wait_out_share": float((used[:, 3] / busy).mean())}
