@@ -279,6 +279,16 @@ strata_status strata_moe_dispatch(strata_ctx *ctx, const strata_moe_layout_t *la
 strata_status strata_moe_combine(strata_ctx *ctx, const strata_moe_layout_t *layout, const void *y,
                                  size_t y_rows, const float *topk_w, void *out, void *stream);
 
+/* Ranks with different token counts (production variant; the paper's Sec. 5.3 motivates batch sizes that
+ * change from step to step, it defines no interface).  The batch is stored as R x T with T the largest count;
+ * this call writes -1 ("not routed") into the K slots of every token t >= tokens_per_rank[r], in place, so
+ * that the layout call that follows on the same stream skips them: the real items then get exactly the rows
+ * of the compacted ragged batch, dispatch writes nothing for the padding tokens and combine returns zero rows
+ * for them.  tokens_per_rank: device int32 [R] (values above T keep the whole rank, negative values mask it);
+ * topk_ids: device int32 [R,T,K].  The context must have been created with STRATA_FLAG_ALLOW_UNROUTED
+ * (STRATA_ERR_SHAPE otherwise).  One launch. */
+strata_status strata_moe_mask_ragged(strata_ctx *ctx, const int32_t *tokens_per_rank, int32_t *topk_ids, void *stream);
+
 /* Row -> expert map of the receive buffer (production variant; the paper names no such array): the per-row
  * group index a grouped expert GEMM needs to read the receive buffer in place, completing the zero-copy
  * hand-over (with segment_align set to the GEMM's tile height, every tile of rows belongs to one expert or

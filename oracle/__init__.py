@@ -53,6 +53,8 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).argtypes = [i32, i64, vp, vp]
         L.oracle_broadcast.restype = None
         L.oracle_broadcast.argtypes = [i32, i32, i64, vp, vp]
+        L.oracle_mask_ragged.restype = None
+        L.oracle_mask_ragged.argtypes = [i32, i32, i32, vp, vp]
         L.oracle_row_experts.restype = None
         L.oracle_row_experts.argtypes = [i32, i32, i32, vp, vp, vp, i64, vp]
         L.oracle_alltoallv.restype = i64
@@ -113,6 +115,16 @@ def layout(ids: np.ndarray, E: int, segment_align: int = 1, allow_unrouted: bool
         raise BadExpertId(int(-rc - 1))
     out["src_of_row"] = out["src_of_row"][:int(out["expert_offset"][E])]
     out["dropped"] = int(rc) if slot_capacity > 0 else 0
+    return out
+
+
+def mask_ragged(ids: np.ndarray, tokens_per_rank) -> np.ndarray:
+    """A copy of ids int32 [R,T,K] with the slots of tokens t >= tokens_per_rank[r] set to -1."""
+    out = _c(ids, np.int32).copy()
+    R, T, K = out.shape
+    tpr = _c(tokens_per_rank, np.int32)
+    assert tpr.shape == (R,)
+    lib().oracle_mask_ragged(R, T, K, _p(tpr), _p(out))
     return out
 
 

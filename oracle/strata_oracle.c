@@ -541,6 +541,20 @@ void oracle_dispatch_windows(int32_t R, int32_t E, int32_t K, int32_t H, int32_t
 }
 
 /* ------------------------------------------------------------------ */
+/* Ranks with different token counts (paper Sec. 5.3 motivates dynamic  */
+/* batch sizes; this build's reading): the batch is stored as R x T     */
+/* with T the largest count; the slots of tokens t >= tokens_per_rank[r]*/
+/* are marked "not routed" (-1) so that the layout skips them.          */
+/* ------------------------------------------------------------------ */
+void oracle_mask_ragged(int32_t R, int32_t T, int32_t K, const int32_t *tokens_per_rank, int32_t *ids)
+{
+    for (int32_t r = 0; r < R; ++r)
+        for (int32_t t = 0; t < T; ++t)
+            if (t >= tokens_per_rank[r])
+                for (int32_t k = 0; k < K; ++k) ids[((size_t)r * T + t) * K + k] = -1;
+}
+
+/* ------------------------------------------------------------------ */
 /* Row -> expert map of the receive buffer: what a grouped expert GEMM  */
 /* that reads the buffer in place needs per row (this build's reading   */
 /* of "zero staging copy into the expert computation"; the paper names  */

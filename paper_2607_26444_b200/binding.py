@@ -40,6 +40,7 @@ EXPORTS = [
     "strata_moe_partition_max_units", "strata_moe_partition", "strata_moe_dispatch_windows",
     "strata_moe_recv_rows",
     "strata_ctx_set_timeline", "strata_timeline_decode", "strata_ctx_set_sm_budget", "strata_moe_row_experts",
+    "strata_moe_mask_ragged",
     "strata_allgather", "strata_alltoall", "strata_broadcast", "strata_reducescatter", "strata_allreduce",
     "strata_p2p", "strata_alltoallv",
 ]
@@ -141,6 +142,7 @@ def lib() -> ctypes.CDLL:
         "strata_moe_dispatch_windows": [vp, P(strata_moe_layout_t), P(strata_partition_t), i32, vp, vp, sz, vp],
         "strata_ctx_set_sm_budget": [vp, i32],
         "strata_moe_row_experts": [vp, P(strata_moe_layout_t), vp, sz, vp],
+        "strata_moe_mask_ragged": [vp, vp, vp, vp],
         "strata_ctx_set_timeline": [vp, vp, sz, sz],
         "strata_timeline_decode": [vp, sz, sz, vp, sz, P(sz), P(sz)],
         "strata_allgather": [vp, i32, vp, vp, sz, vp],
@@ -286,6 +288,10 @@ def strata_moe_dispatch_windows(ctx, layout: strata_moe_layout_t, partition: str
 
 def strata_moe_row_experts(ctx, layout: strata_moe_layout_t, row_expert: int, capacity_rows: int, stream: int) -> int:
     return lib().strata_moe_row_experts(ctx, ctypes.byref(layout), row_expert, capacity_rows, stream)
+
+
+def strata_moe_mask_ragged(ctx, tokens_per_rank: int, topk_ids: int, stream: int) -> int:
+    return lib().strata_moe_mask_ragged(ctx, tokens_per_rank, topk_ids, stream)
 
 
 def strata_ctx_set_sm_budget(ctx, n_sm: int) -> int:
@@ -467,6 +473,11 @@ class MoEContext:
     def combine(self, layout: Layout, y, w, out) -> None:
         _check(strata_moe_combine(self.h, layout.c, y.data_ptr(), y.shape[0], w.data_ptr(), out.data_ptr(),
                                   self._stream()), "strata_moe_combine")
+
+    def mask_ragged(self, tokens_per_rank, ids) -> None:
+        """Marks, in place, the slots of the tokens t >= tokens_per_rank[r] as not routed (-1)."""
+        _check(strata_moe_mask_ragged(self.h, tokens_per_rank.data_ptr(), ids.data_ptr(), self._stream()),
+               "strata_moe_mask_ragged")
 
     def row_experts(self, layout: Layout, out=None):
         """int32 [recv_rows]: the expert of every occupied receive row, -1 for padding and empty rows."""

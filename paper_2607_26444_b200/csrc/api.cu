@@ -457,6 +457,24 @@ strata_status strata_moe_combine(strata_ctx* ctx, const strata_moe_layout_t* lay
     return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
 }
 
+strata_status strata_moe_mask_ragged(strata_ctx* ctx, const int32_t* tokens_per_rank, int32_t* topk_ids, void* stream)
+{
+    if (!ctx || !tokens_per_rank || !topk_ids) return STRATA_ERR_INVALID_ARG;
+    if ((ctx->shape.flags & STRATA_FLAG_ALLOW_UNROUTED) == 0) return STRATA_ERR_SHAPE;   // -1 must be a legal id
+    if (((reinterpret_cast<uintptr_t>(tokens_per_rank) | reinterpret_cast<uintptr_t>(topk_ids)) & 3u) != 0)
+        return STRATA_ERR_ALIGNMENT;
+    if (ctx->device < 0) return STRATA_ERR_CUDA;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return STRATA_ERR_CUDA;
+    cudaError_t err = launch_mask_ragged(ctx->shape, tokens_per_rank, topk_ids, ctx->n_sm_device,
+                                         static_cast<cudaStream_t>(stream));
+    {
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        ctx->launches += 1;
+    }
+    return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
+}
+
 strata_status strata_moe_row_experts(strata_ctx* ctx, const strata_moe_layout_t* layout, int32_t* row_expert,
                                      size_t capacity_rows, void* stream)
 {

@@ -95,6 +95,8 @@ size_t collective_table_bytes();     // workspace tail used by all-to-all-v (a m
 cudaError_t launch_slice_copyv(const void* in, unsigned long long in_stride, void* out, unsigned long long out_stride,
                                const long long* send_bytes, const long long* send_off, const long long* recv_off, int R,
                                void* table, int* status, WorkQueue wq, int n_sm, TraceBuf trace, cudaStream_t st);
+cudaError_t launch_mask_ragged(const strata_moe_shape& s, const int32_t* tokens_per_rank, int32_t* ids, int n_sm,
+                               cudaStream_t st);
 cudaError_t launch_row_experts(const strata_moe_shape& s, const strata_moe_layout_t& L, int32_t* row_expert,
                                long long n_rows, cudaStream_t st);
 int partition_max_units_supported();

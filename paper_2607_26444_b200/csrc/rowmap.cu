@@ -1,3 +1,4 @@
+// Small helpers around the layout.
 // Row -> expert map of the receive buffer: the per-row group index a grouped expert GEMM needs to
 // read the buffer in place (one expert per tile once the segments are aligned to the tile height).
 // row_expert[row] = the expert whose segment holds the row if a token was placed there, else -1.
@@ -59,7 +60,30 @@ __global__ void __launch_bounds__(kRowMapThreads) row_experts_kernel(RowMapParam
     }
 }
 
+// Ranks with different token counts: the slots of the tokens t >= tokens_per_rank[r] become -1 ("not routed").
+__global__ void __launch_bounds__(kRowMapThreads) mask_ragged_kernel(const int32_t* tokens_per_rank, int32_t* ids, int R,
+                                                                      int T, int K)
+{
+    griddep_wait();
+    griddep_launch_dependents();
+    const long long n = (long long)R * T * K;
+    const long long per_rank = (long long)T * K;
+    for (long long i = (long long)blockIdx.x * kRowMapThreads + threadIdx.x; i < n; i += (long long)gridDim.x * kRowMapThreads) {
+        const int r = (int)(i / per_rank);
+        const int t = (int)((i - (long long)r * per_rank) / K);
+        if (t >= tokens_per_rank[r]) ids[i] = -1;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_mask_ragged(const strata_moe_shape& s, const int32_t* tokens_per_rank, int32_t* ids, int n_sm,
+                               cudaStream_t st)
+{
+    const long long n = (long long)s.R * s.T * s.K;
+    const unsigned grid = (unsigned)max(1ll, min((long long)n_sm * 8, (n + kRowMapThreads - 1) / kRowMapThreads));
+    return launch_pdl(mask_ragged_kernel, grid, kRowMapThreads, 0, st, tokens_per_rank, ids, (int)s.R, (int)s.T, (int)s.K);
+}
 
 cudaError_t launch_row_experts(const strata_moe_shape& s, const strata_moe_layout_t& L, int32_t* row_expert,
                                long long n_rows, cudaStream_t st)

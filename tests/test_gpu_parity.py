@@ -766,3 +766,45 @@ def test_usage_with_bfloat16_tensors_against_torch_ops():
     assert ulp_distance(a, b).max() <= 1
     assert ctx.device_status() == B.STRATA_OK
     ctx.close()
+
+
+@pytest.mark.parametrize("kw,tokens", [
+    (dict(R=4, T=30, H=256, E=8, K=3), [30, 7, 0, 19]),
+    (dict(R=8, T=1200, H=64, E=32, K=4), [1200, 1, 600, 0, 1199, 37, 1200, 900]),     # tiled layout path
+    (dict(R=2, T=5, H=64, E=4, K=2), [9, -3]),                                         # above T, below 0
+], ids=lambda v: str(len(v)) if isinstance(v, list) else "R{R}T{T}E{E}K{K}".format(**v))
+def test_ragged_ranks_through_the_mask_call(kw, tokens):
+    """Per-rank token counts: mask, layout, dispatch, combine; the real tokens behave as in the compacted batch."""
+    cfg = wl.shrink(wl.CONFIGS["tiny"], seed=4242, **kw)
+    inp = wl.generate(cfg)
+    tpr = np.array(tokens, np.int32)
+    want_ids = oracle.mask_ragged(inp["ids"], tpr)
+    ctx = B.MoEContext(cfg.R, cfg.T, cfg.H, cfg.E, cfg.K, allow_unrouted=True)
+    ids_d = to_dev(inp["ids"].copy())
+    ctx.mask_ragged(to_dev(tpr), ids_d)
+    torch.cuda.synchronize()
+    assert np.array_equal(ids_d.cpu().numpy(), want_ids)
+    ref = oracle.layout(want_ids, cfg.E, allow_unrouted=True)
+    lay = ctx.layout(ids_d)
+    for key in ("expert_count", "expert_offset", "rank_count", "rank_offset", "src_expert_count", "dst_row"):
+        assert np.array_equal(getattr(lay, key).cpu().numpy().ravel(), ref[key].ravel()), key
+    n_rows = int(ref["expert_offset"][-1])
+    recv = torch.full((cfg.n_items, cfg.H), SENTINEL16, dtype=torch.int16, device=DEV)
+    ctx.register(recv)
+    ctx.dispatch(lay, to_dev(inp["x"]), recv)
+    out = torch.full((cfg.n_tok, cfg.H), SENTINEL16, dtype=torch.int16, device=DEV)
+    ctx.combine(lay, recv, to_dev(inp["w"]), out)
+    torch.cuda.synchronize()
+    want_recv = oracle.dispatch_bf16(ref["dst_row"], inp["x"], n_rows=cfg.n_items)
+    got = u16(recv)
+    assert np.array_equal(got[:n_rows], want_recv[:n_rows]) and np.all(got[n_rows:] == SENTINEL16)
+    want_out = oracle.combine(ref["dst_row"], want_recv, inp["w"])
+    assert np.array_equal(u16(out), want_out)
+    pad = (want_ids.reshape(cfg.n_tok, cfg.K) < 0).all(axis=1)
+    assert np.all(u16(out)[pad] == 0)                       # padding tokens combine to zero rows
+    assert ctx.device_status() == B.STRATA_OK
+    # without the flag the call is refused
+    plain = B.MoEContext(cfg.R, cfg.T, cfg.H, cfg.E, cfg.K)
+    assert B.strata_moe_mask_ragged(plain.h, to_dev(tpr).data_ptr(), ids_d.data_ptr(), None) == B.STRATA_ERR_SHAPE
+    plain.close()
+    ctx.close()

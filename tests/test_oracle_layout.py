@@ -338,3 +338,19 @@ def test_row_experts_is_the_id_of_the_item_placed_in_the_row(align, cap, frac):
         tiles = got.reshape(-1, align)
         for t in tiles:
             assert len(set(t[t >= 0].tolist())) <= 1
+
+
+def test_mask_ragged_marks_exactly_the_padding_tokens():
+    rng = np.random.default_rng(3)
+    R, T, K, E = 4, 9, 3, 8
+    ids = rng.integers(0, E, size=(R, T, K)).astype(np.int32)
+    tokens = np.array([9, 0, 4, 12], np.int32)              # a count above T keeps the whole rank
+    got = oracle.mask_ragged(ids, tokens)
+    t = np.arange(T)[None, :, None]
+    want = np.where(t < tokens[:, None, None], ids, -1)
+    assert np.array_equal(got, want)
+    # and the layout of the masked batch is the layout of the compacted ragged batch
+    lay = oracle.layout(got, E, allow_unrouted=True)
+    compact = np.concatenate([ids[r, :min(int(n), T)].reshape(-1, K) for r, n in enumerate(tokens)])
+    ref = oracle.layout(compact.reshape(1, -1, K), E)
+    assert np.array_equal(lay["dst_row"].ravel()[got.ravel() >= 0], ref["dst_row"].ravel())
