@@ -778,7 +778,7 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
     if not args.no_other:
         del case
         torch.cuda.empty_cache()
-        for name in ("decode", "skew", "fp8"):
+        for name in ("tiny", "decode", "skew", "fp8"):       # tiny is L2 resident: its GB/s are not HBM figures
             c = wl.CONFIGS[name]
             dc = DeviceCase(c, local_rank)
             us = per_call_us(dc)
