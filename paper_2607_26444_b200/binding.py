@@ -506,6 +506,35 @@ class MoEContext:
         _check(strata_ctx_set_trace(self.h, None, 0), "strata_ctx_set_trace")
         self._trace = None
 
+    def sm_budget(self, n_sm: int) -> None:
+        """Sizes the persistent grids for n_sm SMs (0: the whole GPU)."""
+        _check(strata_ctx_set_sm_budget(self.h, n_sm), "strata_ctx_set_sm_budget")
+
+    def timeline(self, n_ctas: int = 2048, events_per_cta: int = 2048, pinned: bool = False):
+        """Turns the event timeline on; returns the zeroed buffer [n_ctas, 1 + events_per_cta] (int64), in
+        device memory or, with pinned=True, in page-locked host memory that the kernels write in place."""
+        import torch
+        if pinned:
+            t = torch.zeros((n_ctas, 1 + events_per_cta), dtype=torch.int64, pin_memory=True)
+        else:
+            t = torch.zeros((n_ctas, 1 + events_per_cta), dtype=torch.int64, device=self.device)
+        torch.cuda.synchronize(self.device)
+        _check(strata_ctx_set_timeline(self.h, t.data_ptr(), n_ctas, events_per_cta), "strata_ctx_set_timeline")
+        self._timeline = t
+        return t
+
+    def timeline_off(self) -> None:
+        _check(strata_ctx_set_timeline(self.h, None, 0, 0), "strata_ctx_set_timeline")
+        self._timeline = None
+
+    @staticmethod
+    def timeline_spans(t):
+        """Synchronises and decodes a timeline buffer (see timeline.decode_timeline); returns (spans, dropped)."""
+        import torch
+        from .timeline import decode_timeline
+        torch.cuda.synchronize()
+        return decode_timeline(t.cpu().numpy().view("uint64"))
+
     # the paper's static window partitioning, as an alternative to run-time work claiming ------------
     def partition(self, layout: Layout, policy: strata_partition_policy, n_cores: int,
                   part: Optional[Partition] = None) -> Partition:
