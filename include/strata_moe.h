@@ -237,13 +237,16 @@ strata_status strata_moe_layout(strata_ctx *ctx, const int32_t *topk_ids,
  * the kernels' scratch lives in a fixed 2 MiB array inside the library (each GPU that loads the
  * library holds it until the process exits) instead of a caller workspace.
  *  - Runs on the CURRENT CUDA device; no context is needed.  `shape->H` and `dispatch_dtype` are ignored;
- *    segment_align and flags are honoured.
+ *    segment_align, flags and slot_capacity are honoured and checked as strata_ctx_create checks them
+ *    (an unknown flag bit, or aligned segments together with fixed slots: STRATA_ERR_SHAPE).
  *  - Limit: 256 + ceil(T*K/4096) * R * E * 4 bytes must fit in 2 MiB (all five benchmark shapes do;
  *    the prefill shape needs 0.13 MiB).  Larger shapes return STRATA_ERR_CAPACITY and launch nothing:
  *    use strata_moe_layout with a workspace for those.
  *  - device_status: device pointer to one int32 owned by the caller, zeroed by the caller; receives
- *    STRATA_ERR_BAD_EXPERT_ID if an id outside [0,E) was skipped.  May be NULL (skipped items are then
- *    only visible as dst_row = -1).
+ *    STRATA_ERR_BAD_EXPERT_ID if an id outside [0,E) was skipped and, under slot_capacity > 0,
+ *    STRATA_ERR_CAPACITY if a slot overflowed (the first error wins).  May be NULL: skipped and
+ *    dropped items are then only visible as dst_row = -1, and a caller that must tell an overflow
+ *    from an unrouted slot has to pass the word.
  *  - The first call on each device resolves the array's device address and sets one kernel
  *    attribute (no allocation).  Make that first call before any stream capture begins.
  *  - All calls on a device share the one array, which keeps the previous call's contents; the

@@ -43,26 +43,17 @@ namespace {
 
 using namespace strata;
 
-// rows of the receive buffer: all items plus the worst-case padding of aligned segments
-long long recv_rows(const strata_moe_shape& s)
-{
-    if (s.slot_capacity > 0) return (long long)s.E * s.R * s.slot_capacity;
-    const long long pad = s.segment_align > 1 ? s.segment_align - 1 : 0;
-    return (long long)s.R * s.T * s.K + (long long)s.E * pad;
-}
-
 strata_status check_shape(const strata_moe_shape* s)
 {
     if (!s) return STRATA_ERR_INVALID_ARG;
-    if (s->R <= 0 || s->T <= 0 || s->H <= 0 || s->E <= 0 || s->K <= 0) return STRATA_ERR_SHAPE;
-    if (s->E % s->R != 0 || s->E > kMaxExperts || s->K > kMaxTopK) return STRATA_ERR_SHAPE;
-    if (s->H % 8 != 0) return STRATA_ERR_SHAPE;
+    if (s->H <= 0 || s->H % 8 != 0) return STRATA_ERR_SHAPE;
+    const strata_status st = check_layout_shape(*s);
+    if (st != STRATA_OK) return st;
     if (s->dispatch_dtype != STRATA_BF16 && s->dispatch_dtype != STRATA_FP8_E4M3_B128) return STRATA_ERR_SHAPE;
     if (s->dispatch_dtype == STRATA_FP8_E4M3_B128 && s->H % 128 != 0) return STRATA_ERR_SHAPE;
-    if (s->segment_align < 0 || s->segment_align > 65536) return STRATA_ERR_SHAPE;
-    if ((s->flags & ~STRATA_FLAG_ALLOW_UNROUTED) != 0) return STRATA_ERR_SHAPE;
-    if (s->slot_capacity < 0 || (s->slot_capacity > 0 && s->segment_align > 1)) return STRATA_ERR_SHAPE;
-    if (recv_rows(*s) >= (1ll << 31)) return STRATA_ERR_SHAPE;
+    // Dispatch and combine number their work units (a token, or a column piece of one never shorter than
+    // 1 KB) with 32-bit counters whose top values are reserved.
+    if ((long long)s->R * s->T * (((long long)s->H * 2 + 1023) / 1024) >= (1ll << 32) - (1ll << 20)) return STRATA_ERR_SHAPE;
     return STRATA_OK;
 }
 
@@ -561,7 +552,8 @@ strata_status strata_moe_dispatch_windows(strata_ctx* ctx, const strata_moe_layo
 {
     if (!ctx || !layout || !partition || !x || !recv) return STRATA_ERR_INVALID_ARG;
     if (!layout->src_expert_count || !layout->src_of_row) return STRATA_ERR_INVALID_ARG;
-    if (!partition->win_base || !partition->unit_desc || !partition->task_offset || !partition->task_unit)
+    if (!partition->win_base || !partition->unit_desc || !partition->task_offset || !partition->task_unit ||
+        !partition->n_units)
         return STRATA_ERR_INVALID_ARG;
     const strata_moe_shape& s = ctx->shape;
     if (s.dispatch_dtype != STRATA_BF16 || (uint32_t)s.H * 2u > windows_max_row_bytes() || s.slot_capacity > 0)

@@ -38,6 +38,27 @@ inline LayoutGeom layout_geom(const strata_moe_shape& s)
     return g;
 }
 
+// rows of the receive buffer: all items plus the worst-case padding of aligned segments
+inline long long recv_rows(const strata_moe_shape& s)
+{
+    if (s.slot_capacity > 0) return (long long)s.E * s.R * s.slot_capacity;
+    const long long pad = s.segment_align > 1 ? s.segment_align - 1 : 0;
+    return (long long)s.R * s.T * s.K + (long long)s.E * pad;
+}
+
+// The clauses of the shape check that the routing layout depends on (everything but H and the
+// dispatch dtype): shared by context creation and by the allocation-free layout entry.
+inline strata_status check_layout_shape(const strata_moe_shape& s)
+{
+    if (s.R <= 0 || s.T <= 0 || s.E <= 0 || s.K <= 0) return STRATA_ERR_SHAPE;
+    if (s.E % s.R != 0 || s.E > kMaxExperts || s.K > kMaxTopK) return STRATA_ERR_SHAPE;
+    if (s.segment_align < 0 || s.segment_align > 65536) return STRATA_ERR_SHAPE;
+    if ((s.flags & ~STRATA_FLAG_ALLOW_UNROUTED) != 0) return STRATA_ERR_SHAPE;
+    if (s.slot_capacity < 0 || (s.slot_capacity > 0 && s.segment_align > 1)) return STRATA_ERR_SHAPE;
+    if (recv_rows(s) >= (1ll << 31) || (long long)s.R * s.T * s.K >= (1ll << 31)) return STRATA_ERR_SHAPE;
+    return STRATA_OK;
+}
+
 // Dynamic work distribution.  CTAs (or warps) claim the next unit with one atomicAdd on a counter in
 // the workspace; nothing ever waits.  Units are claimed in order, so the CTAs running at any moment
 // work on neighbouring tokens, and a CTA that happens to get less memory bandwidth simply claims

@@ -431,16 +431,16 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_cluster_kernel(LayoutPa
         const bool leader = valid && lane == __ffs(peers) - 1;
         if (leader) mine[e] += __popc(peers);
         if (p.src_expert_count) {
-            const int r = valid ? i / p.items_per_rank : -1;
-            // lane 0 of a round is valid whenever any lane is (runs are contiguous); ranks rise with the lane
-            const int r_lo = __shfl_sync(0xffffffffu, r, 0);
-            const int r_lo_valid = r_lo < 0 ? r : r_lo;
-            const unsigned all_same = __all_sync(0xffffffffu, r == r_lo || !valid);
+            // Source rank relative to the rank of the round's first item: defined for every lane whether or
+            // not its id is valid, and in [0, 31] because a round holds 32 consecutive items.
+            const int r0 = (first + q * 32) / p.items_per_rank;
+            const int rel = i / p.items_per_rank - r0;
+            const unsigned all_same = __all_sync(0xffffffffu, rel == 0 || !valid);
             if (all_same) {
-                if (leader) atomicAdd(&src_cnt[r * E + e], __popc(peers));
+                if (leader) atomicAdd(&src_cnt[r0 * E + e], __popc(peers));
             } else {
-                const unsigned peers2 = peers & same_key_lanes(r - r_lo_valid, 5);
-                if (valid && lane == __ffs(peers2) - 1) atomicAdd(&src_cnt[r * E + e], __popc(peers2));
+                const unsigned peers2 = peers & same_key_lanes(rel, 5);
+                if (valid && lane == __ffs(peers2) - 1) atomicAdd(&src_cnt[(r0 + rel) * E + e], __popc(peers2));
             }
         }
         __syncwarp();
@@ -816,13 +816,8 @@ extern "C" strata_status strata_moe_layout_noalloc(const strata_moe_shape* shape
         !layout->dst_row)
         return STRATA_ERR_INVALID_ARG;
     const strata_moe_shape& s = *shape;
-    if (s.R <= 0 || s.T <= 0 || s.E <= 0 || s.K <= 0) return STRATA_ERR_SHAPE;
-    if (s.E % s.R != 0 || s.E > kMaxExperts || s.K > kMaxTopK) return STRATA_ERR_SHAPE;
-    if (s.segment_align < 0 || s.segment_align > 65536) return STRATA_ERR_SHAPE;
-    if (s.slot_capacity < 0 || (s.slot_capacity > 0 && s.segment_align > 1)) return STRATA_ERR_SHAPE;
-    if ((long long)s.E * s.R * s.slot_capacity >= (1ll << 31)) return STRATA_ERR_SHAPE;
-    if ((long long)s.R * s.T * s.K + (long long)s.E * (s.segment_align > 1 ? s.segment_align - 1 : 0) >= (1ll << 31))
-        return STRATA_ERR_SHAPE;
+    const strata_status shape_rc = check_layout_shape(s);
+    if (shape_rc != STRATA_OK) return shape_rc;
     const LayoutGeom g = layout_geom(s);
     const size_t need = (size_t)kWsHeaderBytes + (size_t)g.n_tiles * s.E * sizeof(int);
     if (need > kStaticScratchBytes) return STRATA_ERR_CAPACITY;     // beyond the fixed array: use a workspace

@@ -482,8 +482,9 @@ struct WindowsParams {
     const int32_t* src_of_row;
     const unsigned char* x;
     unsigned char* recv;
+    const int32_t* n_units;
     long long capacity_rows, n_tok;
-    int E, e_loc, K, H;
+    int R, E, e_loc, K, H;
     int* status;
     TraceBuf trace;
 };
@@ -531,6 +532,7 @@ __global__ void __launch_bounds__(32) dispatch_windows_kernel(WindowsParams p)
     int q = p.task_offset[core];
     const int q_end = p.task_offset[core + 1];
     int r = 0, e = 0, e_end = 0, first = 0, rows_left = 0;
+    const int n_units_total = *p.n_units;
     bool ok = true;
 
     while (ok) {
@@ -541,10 +543,21 @@ __global__ void __launch_bounds__(32) dispatch_windows_kernel(WindowsParams p)
                 if (rows_left == 0) {
                     if (q >= q_end) break;
                     const int j = p.task_unit[q++];
+                    if (j < 0 || j >= n_units_total) {          // a task list that names no unit of this partition
+                        report_status(p.status, STRATA_ERR_INVALID_ARG);
+                        q = q_end;
+                        break;
+                    }
                     r = p.unit_desc[j * 4 + 0];
                     const int d = p.unit_desc[j * 4 + 1];
                     first = p.unit_desc[j * 4 + 2];
                     rows_left = p.unit_desc[j * 4 + 3];
+                    if (r < 0 || r >= p.R || d < 0 || d >= p.R || first < 0 || rows_left < 0) {
+                        report_status(p.status, STRATA_ERR_INVALID_ARG);
+                        rows_left = 0;
+                        q = q_end;
+                        break;
+                    }
                     e = d * p.e_loc;
                     e_end = e + p.e_loc;
                 }
@@ -573,8 +586,9 @@ __global__ void __launch_bounds__(32) dispatch_windows_kernel(WindowsParams p)
         __syncwarp();
         const int my_row = lane < n ? s_row[lane] : -1;
         const bool row_ok = my_row >= 0 && my_row < p.capacity_rows;
-        long long my_tok = row_ok ? (long long)p.src_of_row[my_row] / p.K : -1;
-        if (lane < n && (!row_ok || my_tok < 0 || my_tok >= p.n_tok)) {
+        const int my_src = row_ok ? p.src_of_row[my_row] : -1;      // -1: a padding or empty row has no source item
+        long long my_tok = my_src >= 0 ? (long long)my_src / p.K : -1;
+        if (lane < n && (my_tok < 0 || my_tok >= p.n_tok)) {
             report_status(p.status, STRATA_ERR_BAD_ROW);
             my_tok = -1;
         }
@@ -663,10 +677,12 @@ cudaError_t launch_dispatch_windows(const strata_moe_shape& s, const strata_moe_
     p.task_offset = part.task_offset;
     p.task_unit = part.task_unit;
     p.src_of_row = L.src_of_row;
+    p.n_units = part.n_units;
     p.x = static_cast<const unsigned char*>(x);
     p.recv = static_cast<unsigned char*>(recv);
     p.capacity_rows = (long long)capacity_rows;
     p.n_tok = (long long)s.R * s.T;
+    p.R = s.R;
     p.E = s.E;
     p.e_loc = s.E / s.R;
     p.K = s.K;

@@ -519,6 +519,43 @@ def test_aligned_segments_and_unrouted_slots(kw, align, frac):
     ctx.close()
 
 
+def _layout_only(R, T, K, E, ids):
+    ref = oracle.layout(ids, E, allow_unrouted=True)
+    ctx = B.MoEContext(R, T, 64, E, K, allow_unrouted=True)
+    lay = ctx.layout(to_dev(ids))
+    torch.cuda.synchronize()
+    assert ctx.device_status() == B.STRATA_OK
+    for key in ("expert_count", "expert_offset", "rank_count", "rank_offset", "src_expert_count", "dst_row"):
+        assert np.array_equal(getattr(lay, key).cpu().numpy(), ref[key]), key
+    ctx.close()
+
+
+def test_unrouted_first_lane_of_a_round_that_straddles_two_source_ranks():
+    """A 32-item round whose first item is not routed and whose items belong to two source ranks: the
+    per-source-rank counts must still split at the rank boundary (48 items per rank, item 32 = -1)."""
+    R, T, K, E = 2, 24, 2, 4
+    ids = np.ones((R, T, K), np.int32)
+    ids.reshape(-1)[32] = -1
+    ref = oracle.layout(ids, E, allow_unrouted=True)
+    assert ref["src_expert_count"][:, 1].tolist() == [47, 48]
+    _layout_only(R, T, K, E, ids)
+
+
+@pytest.mark.parametrize("kw", [dict(R=3, T=21, K=3, E=6), dict(R=8, T=37, K=5, E=16), dict(R=16, T=129, K=7, E=64),
+                                dict(R=5, T=1, K=1, E=5), dict(R=32, T=3, K=1, E=32)],
+                         ids=lambda kw: "R{R}T{T}K{K}E{E}".format(**kw))
+def test_unrouted_at_every_round_start_with_ranks_off_the_round_grid(kw):
+    """T*K is not a multiple of 32, so rounds straddle ranks; every 32nd item (each round's first lane,
+    whatever the run length) is forced to -1, and a random fifth of the rest too."""
+    R, T, K, E = kw["R"], kw["T"], kw["K"], kw["E"]
+    rng = np.random.default_rng(R * 1000 + T)
+    ids = rng.integers(0, E, size=(R, T, K), dtype=np.int32)
+    flat = ids.reshape(-1)
+    flat[rng.random(flat.shape) < 0.2] = -1
+    flat[::32] = -1
+    _layout_only(R, T, K, E, ids)
+
+
 def test_minus_one_is_an_error_without_the_flag():
     cfg = wl.shrink(wl.CONFIGS["tiny"], H=64)
     ids = wl.gen_topk_ids(cfg)

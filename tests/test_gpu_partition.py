@@ -118,3 +118,38 @@ def test_host_errors():
         == B.STRATA_ERR_INVALID_ARG
     torch.cuda.synchronize()
     ctx.close()
+
+
+def test_window_dispatch_survives_inconsistent_lists():
+    """Lists that do not belong together are reported on the device and nothing is read or written out of
+    bounds: a receive row without a source item (src_of_row = -1, with K > 1) is skipped with BAD_ROW instead
+    of being filled with token 0, and a task list naming a unit that does not exist raises INVALID_ARG."""
+    cfg = wl.shrink(wl.CONFIGS["tiny"], seed=78, R=4, T=64, H=256, E=16, K=4)
+    inp = wl.generate(cfg)
+    ctx = B.MoEContext(cfg.R, cfg.T, cfg.H, cfg.E, cfg.K)
+    lay = ctx.layout(to_dev(inp["ids"]))
+    part = ctx.partition(lay, B.make_policy([(10, 64, 16, 2)]), 8)
+    N = cfg.n_items
+    whole = torch.full((N + 6, cfg.H), SENTINEL16, dtype=torch.int16, device=DEV)
+    recv = whole[3:3 + N]
+    ctx.register(whole)
+    x = to_dev(inp["x"])
+    want = oracle.dispatch_bf16(oracle.layout(inp["ids"], cfg.E)["dst_row"], inp["x"], nthreads=2)
+
+    hole = 37
+    lay.src_of_row[hole] = -1
+    ctx.dispatch_windows(lay, part, x, recv)
+    assert ctx.device_status() == B.STRATA_ERR_BAD_ROW
+    got = whole.cpu().numpy().view(np.uint16)
+    keep = np.arange(N) != hole
+    assert np.array_equal(got[3:3 + N][keep], want[keep]) and np.all(got[3 + hole] == SENTINEL16)
+    assert np.all(got[:3] == SENTINEL16) and np.all(got[3 + N:] == SENTINEL16)
+
+    lay2 = ctx.layout(to_dev(inp["ids"]))
+    part.task_unit[0] = 1 << 20
+    ctx.dispatch_windows(lay2, part, x, recv)
+    assert ctx.device_status() == B.STRATA_ERR_INVALID_ARG
+    part.task_unit[0] = -5
+    ctx.dispatch_windows(lay2, part, x, recv)
+    assert ctx.device_status() == B.STRATA_ERR_INVALID_ARG
+    ctx.close()
