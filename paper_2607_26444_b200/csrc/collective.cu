@@ -22,6 +22,10 @@ namespace strata {
 
 namespace {
 
+// The collectives' grids are not pinned to a number of CTAs per SM, so only small ones are launched as
+// programmatic dependents (a large one overlapped with its predecessor's tail can be placed unevenly).
+constexpr long long kCollectivePdlMaxBytes = 16ll << 20;
+
 constexpr int kCopyStages = 3;
 constexpr uint32_t kCopyChunkBytes = 16384;
 constexpr int kCopyCtasPerSm = 2;
@@ -474,7 +478,7 @@ cudaError_t launch_slice_copyv(const void* in, unsigned long long in_stride, voi
     cudaError_t err = launch_pdl(copyv_table_kernel, 1u, (unsigned)kMaxVPairs, 0, st, p);
     if (err != cudaSuccess) return err;
     // the number of units is known only on the device: a full persistent grid, CTAs without work leave at once
-    const bool small = (long long)R * (long long)(in_stride + out_stride) < kPdlMaxBytes;
+    const bool small = (long long)R * (long long)(in_stride + out_stride) < kCollectivePdlMaxBytes;
     return STRATA_LAUNCH_LONG(small, slice_copyv_kernel, (unsigned)(n_sm * kCopyCtasPerSm), 32, kCopyVSmem, st, p);
 }
 
@@ -531,7 +535,7 @@ cudaError_t launch_slice_copy(const void* in, void* out, unsigned long long n_sl
         max_grid = (long long)n_sm * max(kCopyCtasPerSm, min(per_sm, 8));
     }
     const unsigned grid = (unsigned)max(1ll, min(max_grid, (long long)p.n_units));
-    const bool small = (long long)(n_slices * slice_bytes) * (fan + 1) < kPdlMaxBytes;
+    const bool small = (long long)(n_slices * slice_bytes) * (fan + 1) < kCollectivePdlMaxBytes;
     return STRATA_LAUNCH_LONG(small, slice_copy_kernel, grid, 32, smem, st, p);
 }
 
@@ -548,7 +552,7 @@ cudaError_t launch_slice_reduce(const void* in, void* out, unsigned long long n_
     p.fan_stride = n_vec * 16ull;
     p.wq = wq;
     p.trace = trace;
-    const bool small = (long long)(n_vec * 16ull) * (R + fan) < kPdlMaxBytes;
+    const bool small = (long long)(n_vec * 16ull) * (R + fan) < kCollectivePdlMaxBytes;
     if (R > 8 && n_vec <= (unsigned long long)n_sm * 2u * kReduceThreads) {
         // latency bound: one-warp CTAs so that more SMs take part, the deepest batch of loads
         p.vec_per_unit = 32;

@@ -199,7 +199,8 @@ cudaError_t launch_k(const CombineParams& p, int n_sm, cudaStream_t st)
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, combine_kernel<KT>, kCombineThreads, 0);
     if (err != cudaSuccess) return err;
     if (per_sm < 1) per_sm = 1;
-    if (STRATA_COMBINE_MAX_CTAS_PER_SM > 0) per_sm = min(per_sm, STRATA_COMBINE_MAX_CTAS_PER_SM);
+    const int cap_per_sm = (int)tune("STRATA_COMB_CTAS", STRATA_COMBINE_MAX_CTAS_PER_SM);
+    if (cap_per_sm > 0) per_sm = min(per_sm, cap_per_sm);
     CombineParams q = p;
     const long long max_grid = (long long)n_sm * per_sm;
     q.parts = 1;
@@ -209,12 +210,13 @@ cudaError_t launch_k(const CombineParams& p, int n_sm, cudaStream_t st)
         // vector per thread per unit)
         const int m_full = q.vec_per_part / kCombineThreads;
         int parts = 1;
-        while (parts < m_full && p.n_tok * parts < STRATA_COMBINE_UNITS_PER_CTA * max_grid) ++parts;
+        const long long want_units = tune("STRATA_COMB_UNITS", STRATA_COMBINE_UNITS_PER_CTA) * max_grid;
+        while (parts < m_full && p.n_tok * parts < want_units) ++parts;
         q.vec_per_part = (m_full + parts - 1) / parts * kCombineThreads;
         q.parts = (p.H / 8 + q.vec_per_part - 1) / q.vec_per_part;
     }
     const long long grid = max(1ll, min(max_grid, p.n_tok * q.parts));
-    const bool small = p.n_tok * p.H * 2 * (p.K + 1) < kPdlMaxBytes;
+    const bool small = p.n_tok * p.H * 2 * (p.K + 1) < pdl_max_bytes();
     return STRATA_LAUNCH_LONG(small, combine_kernel<KT>, (unsigned)grid, kCombineThreads, 0, st, q);
 }
 

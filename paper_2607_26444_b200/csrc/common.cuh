@@ -3,6 +3,7 @@
 
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
 
 #include "strata_moe.h"
 #include "strata_collective.h"
@@ -36,6 +37,19 @@ inline LayoutGeom layout_geom(const strata_moe_shape& s)
     g.tiles_per_rank = (g.items_per_rank + kLayoutTile - 1) / kLayoutTile;
     g.n_tiles = s.R * g.tiles_per_rank;
     return g;
+}
+
+// Launch-shape constants can be overridden from the environment in builds made with -DSTRATA_TUNE
+// (measurement sweeps only); the shipped library compiles every call down to its default.
+inline long long tune(const char* name, long long dflt)
+{
+#ifdef STRATA_TUNE
+    const char* v = getenv(name);
+    return (v && *v) ? atoll(v) : dflt;
+#else
+    (void)name;
+    return dflt;
+#endif
 }
 
 // rows of the receive buffer: all items plus the worst-case padding of aligned segments
@@ -199,12 +213,14 @@ inline cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), unsigned grid, u
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-// Dispatch and combine are launched as programmatic dependents only for small batches.  Measured on
-// B200: for a 3 MB batch the overlap takes the three-call step from 17.4 to 13.3 us; at the decode
-// shape (264 MB) it is neutral; at the prefill shape a dispatch launched as a programmatic dependent
-// of another kernel ran 20 % slower for its whole duration (cause not found: CTA placement was
-// checked to be even), so large batches use plain stream order.
-constexpr long long kPdlMaxBytes = 16ll << 20;
+// Dispatch and combine are launched as programmatic dependents too.  Measured on B200 with grids whose
+// shared-memory request pins the number of CTAs per SM: the gap between the last CTA of one kernel and
+// the first CTA of the next falls from 4 us to 1.3 us; the three-call step goes from 17.4 to 13.3 us for
+// a 3 MB batch, from 96 to 90 us at the decode shape and from 2581 to 2570 us at the prefill shape.
+// (Without the pinning, a dispatch launched as a dependent ran 20 % slower for its whole duration.)
+// STRATA_PDL_MAX_MB, in tuning builds, restores plain stream order above a size for A/B measurements.
+constexpr long long kPdlMaxBytes = 1ll << 50;
+inline long long pdl_max_bytes() { return tune("STRATA_PDL_MAX_MB", kPdlMaxBytes >> 20) << 20; }
 #define STRATA_LAUNCH_LONG(small, ...) ((small) ? launch_pdl(__VA_ARGS__) : launch_plain(__VA_ARGS__))
 
 // ---- device helpers --------------------------------------------------------

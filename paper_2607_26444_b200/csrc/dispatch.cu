@@ -21,27 +21,34 @@ namespace strata {
 
 namespace {
 
-// Build-time tuning knobs.  Measured on B200 at the prefill shape: 2..4 stages, 1..5 CTAs per SM,
-// 4..16 KB chunks and the store hint all land within 1% of each other (5.68..5.71 TB/s); a variant
-// that moved the payload through registers (16-byte loads, K 16-byte stores) reached 5.0 TB/s.
-// What bounds the kernel is HBM serving a 1:8 read:write mix: with the same stores and the source
-// rows resident in L2 the kernel writes at 6.3 TB/s (the rate of a pure bulk-store fill), with the
-// source in DRAM it runs at 5.7 TB/s whichever way the rows are loaded (bulk copy, cp.async, or
-// producer warps with plain loads), and clustering the reads with L2 prefetches made it slower.
+// Launch shape, measured on B200 (kernel time from the first CTA's start to the last CTA's end):
+//  - What bounds the kernel is HBM serving a 1:8 read:write mix; a variant that moved the payload through
+//    registers (16-byte loads, K 16-byte stores) was 12 % slower than the copy engine.
+//  - 14 KB rows (decode and prefill shapes): one CTA per SM with an 8-stage ring beats two CTAs per SM with
+//    3 stages (decode 40.9 vs 42.7 us; prefill 1281 vs 1288 us).  Rings of 10 and 12 stages copy as fast
+//    alone but make the layout+dispatch+combine step at the prefill shape 0.5 % and 1.5 % slower.
+//  - 8 KB rows (skew shape): one issuing lane per SM cannot keep the copy engine fed (257 vs 183 us), so
+//    short chunks take two CTAs per SM.
+//  - Cutting the last units of the batch into halves or quarters evens out the CTAs' finish times (8 us
+//    apart to 2 us apart at the decode shape) but does not shorten the kernel: the CTAs that are still
+//    running get the bandwidth of those that have left.  Pieces below 4 KB copy markedly slower.
+//  - The shared-memory request is padded so that exactly the intended number of CTAs fits an SM (see
+//    smem_for_residency): without it a launch overlapped with its predecessor's tail is placed unevenly.
 #ifndef STRATA_BF16_STAGES
 #define STRATA_BF16_STAGES 3
 #endif
 #ifndef STRATA_BF16_CHUNK_BYTES
 #define STRATA_BF16_CHUNK_BYTES 16384
 #endif
-#ifndef STRATA_BF16_MAX_CTAS_PER_SM
-#define STRATA_BF16_MAX_CTAS_PER_SM 2          // 0: as many as fit
-#endif
 #ifndef STRATA_BF16_STORE_HINT
 #define STRATA_BF16_STORE_HINT 0               // 1: L2 evict-first policy on the bulk stores
 #endif
 constexpr uint32_t kMaxChunkBytes = STRATA_BF16_CHUNK_BYTES;   // one stage of the bf16 ring
 constexpr int kBf16Stages = STRATA_BF16_STAGES;
+constexpr size_t kBf16MaxSmem = 200 * 1024;  // ring + barriers of one CTA never exceed this
+constexpr uint32_t kDeepRingMinBytes = 12 * 1024;     // chunks at least this long take the one-CTA-per-SM shape
+constexpr size_t kDeepRingBytes = 128 * 1024;         // its ring: as many stages as fit here, at most
+constexpr int kDeepRingMaxStages = 8;                 // this many
 // 64..256 threads and 2048..4096-column chunks land within 1.5 % of each other (110..113 us at the fp8 shape);
 // 1024-column chunks are 25 % slower.
 constexpr int kFp8Threads = 128;
@@ -58,6 +65,7 @@ struct DispatchParams {
     int H;
     int chunks_per_row;
     uint32_t chunk_cols;        // columns per chunk (last chunk of a row may be shorter)
+    int stages;                 // bf16 only: depth of the ring in shared memory
     int* status;
     WorkQueue wq;
     TraceBuf trace;
@@ -67,14 +75,15 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
     const uint32_t stage_bytes = p.chunk_cols * 2u;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kBf16Stages * stage_bytes);
-    unsigned int* s_unit = reinterpret_cast<unsigned int*>(bars + kBf16Stages);   // unit held by each stage
+    const int n_stages = p.stages;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)n_stages * stage_bytes);
+    unsigned int* s_unit = reinterpret_cast<unsigned int*>(bars + n_stages);   // unit held by each stage
     const int lane = threadIdx.x;
     const size_t row_bytes = (size_t)p.H * 2u;
     const unsigned int n_units = (unsigned int)p.n_units;
 
     if (lane == 0) {
-        for (int s = 0; s < kBf16Stages; ++s) {
+        for (int s = 0; s < n_stages; ++s) {
             mbar_init(&bars[s], 1);
             s_unit[s] = kNoUnit;
         }
@@ -95,11 +104,11 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
     };
     bool triggered = false, exhausted = false;
     // The first stages-1 units of a CTA are fixed (blockIdx + j*grid); the rest are claimed.
-    const unsigned int n_static = (unsigned int)(kBf16Stages - 1) * gridDim.x;
+    const unsigned int n_static = (unsigned int)(n_stages - 1) * gridDim.x;
     auto issue_load = [&](long long j) {   // lane 0 only: next unit into stage j % stages
-        const int s = (int)(j % kBf16Stages);
+        const int s = (int)(j % n_stages);
         unsigned int u;
-        if (j < kBf16Stages - 1) {
+        if (j < n_stages - 1) {
             u = blockIdx.x + (unsigned int)j * gridDim.x;
             if (u >= n_units) u = kNoUnit;
         } else {
@@ -120,14 +129,14 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
     };
 
     if (lane == 0)
-        for (long long j = 0; j < kBf16Stages - 1; ++j) issue_load(j);
+        for (long long j = 0; j < n_stages - 1; ++j) issue_load(j);
     __syncwarp();
 
     bool ok = true;
     StageClock wait_in(p.trace), wait_out(p.trace);
     for (long long j = 0;; ++j) {
-        const int s = (int)(j % kBf16Stages);
-        const uint32_t parity = (uint32_t)((j / kBf16Stages) & 1);
+        const int s = (int)(j % n_stages);
+        const uint32_t parity = (uint32_t)((j / n_stages) & 1);
         const unsigned int u = s_unit[s];
         if (u == kNoUnit) break;          // claims fail in order: nothing is in flight behind this stage
         long long tok;
@@ -167,7 +176,7 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
             bulk_wait_read<1>();
             tl.end(STRATA_STAGE_WAIT_OUT);
             wait_out.end();
-            issue_load(j + kBf16Stages - 1);
+            issue_load(j + n_stages - 1);
         }
         __syncwarp();
     }
@@ -345,11 +354,42 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
     }
 }
 
-uint32_t pick_chunk_cols_bf16(int H)
+// Shared memory to request so that exactly `want` CTAs of `kernel` fit on an SM (fewer if `need` is too
+// large for that).  The persistent grids have want * n_sm CTAs and assume `want` on every SM.  When such a
+// grid is launched as a programmatic dependent, its CTAs are placed while the preceding kernel still
+// holds part of some SMs; if more than `want` fitted on an SM, the free SMs would take several CTAs and
+// others none, and the kernel would run with a lopsided placement for its whole life (measured: 20 %
+// slower at the prefill shape).  Asking for more shared memory than needed makes the surplus CTA not fit.
+template <typename Kernel>
+cudaError_t smem_for_residency(Kernel kernel, int threads, size_t need, int want, size_t max_smem, size_t* smem_out,
+                               int* per_sm_out)
+{
+    int dev = 0, sm_total = 0, reserved = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    err = cudaDeviceGetAttribute(&sm_total, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
+    if (err != cudaSuccess) return err;
+    err = cudaDeviceGetAttribute(&reserved, cudaDevAttrReservedSharedMemoryPerBlock, dev);
+    if (err != cudaSuccess) return err;
+    if (want < 1) want = 1;
+    // want + 1 CTAs must not fit: (want + 1) * (smem + reserved) > sm_total
+    size_t excl = (size_t)sm_total / (size_t)(want + 1) + 1;
+    excl = excl > (size_t)reserved ? excl - (size_t)reserved : 0;
+    size_t smem = max(need, (excl + 127) & ~(size_t)127);
+    if (smem > max_smem) smem = max(need, max_smem);
+    int per_sm = 0;
+    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem);
+    if (err != cudaSuccess) return err;
+    *smem_out = smem;
+    *per_sm_out = max(1, min(per_sm, want));
+    return cudaSuccess;
+}
+
+uint32_t pick_chunk_cols_bf16(int H, uint32_t max_chunk_bytes)
 {
     const uint32_t row_bytes = (uint32_t)H * 2u;
-    if (row_bytes <= kMaxChunkBytes) return (uint32_t)H;
-    const uint32_t n = (row_bytes + kMaxChunkBytes - 1) / kMaxChunkBytes;
+    if (row_bytes <= max_chunk_bytes) return (uint32_t)H;
+    const uint32_t n = (row_bytes + max_chunk_bytes - 1) / max_chunk_bytes;
     uint32_t cols = ((uint32_t)H + n - 1) / n;
     cols = (cols + 7u) & ~7u;        // chunks start on 16-byte boundaries
     return cols;
@@ -360,10 +400,9 @@ uint32_t pick_chunk_cols_bf16(int H)
 cudaError_t configure_dispatch_kernels()
 {
     cudaError_t err = cudaFuncSetAttribute(dispatch_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           kBf16Stages * (int)kMaxChunkBytes + 64);
+                                           (int)kBf16MaxSmem);
     if (err != cudaSuccess) return err;
-    return cudaFuncSetAttribute(dispatch_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                kFp8MaxChunkCols * 6 + 64);
+    return cudaFuncSetAttribute(dispatch_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBf16MaxSmem);
 }
 
 cudaError_t launch_dispatch_bf16(const strata_moe_shape& s, const int32_t* dst_row, const void* x, void* recv,
@@ -379,19 +418,26 @@ cudaError_t launch_dispatch_bf16(const strata_moe_shape& s, const int32_t* dst_r
     p.recv_scale = nullptr;
     p.K = s.K;
     p.H = s.H;
-    p.chunk_cols = pick_chunk_cols_bf16(s.H);
+    p.chunk_cols = pick_chunk_cols_bf16(s.H, (uint32_t)tune("STRATA_DISP_CHUNK", kMaxChunkBytes));
     p.chunks_per_row = (int)(((uint32_t)s.H + p.chunk_cols - 1) / p.chunk_cols);
-    p.n_units = (long long)s.R * s.T * p.chunks_per_row;
     p.capacity_rows = (long long)capacity_rows;
     p.status = status;
-    const size_t smem = (size_t)kBf16Stages * p.chunk_cols * 2u + 64;   // stages | mbarriers | unit ids
+    // Long chunks: one CTA per SM with a deep ring (its single issuing lane keeps up: a unit every ~3 us).
+    // Short chunks need two issuing lanes per SM to keep the copy engine fed, so two CTAs with a short ring.
+    const uint32_t stage_bytes = p.chunk_cols * 2u;
+    const bool deep = stage_bytes >= kDeepRingMinBytes;
+    int want_per_sm = (int)tune("STRATA_DISP_CTAS", deep ? 1 : 2);
+    p.stages = (int)tune("STRATA_DISP_STAGES", deep ? min(kDeepRingMaxStages, (int)(kDeepRingBytes / stage_bytes)) : kBf16Stages);
+    while (p.stages > 2 && (size_t)p.stages * (stage_bytes + 12) + 16 > kBf16MaxSmem) --p.stages;
+    const size_t need = (size_t)p.stages * stage_bytes + 12 * (size_t)p.stages + 16;   // stages | mbarriers | unit ids
+    size_t smem = 0;
     int per_sm = 0;
-    cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dispatch_bf16_kernel, 32, smem);
+    cudaError_t err = smem_for_residency(dispatch_bf16_kernel, 32, need, want_per_sm, kBf16MaxSmem, &smem, &per_sm);
     if (err != cudaSuccess) return err;
-    if (per_sm < 1) per_sm = 1;
-    if (STRATA_BF16_MAX_CTAS_PER_SM > 0) per_sm = min(per_sm, STRATA_BF16_MAX_CTAS_PER_SM);
-    const long long grid = max(1ll, min((long long)n_sm * per_sm, p.n_units));
-    const bool small = (long long)s.R * s.T * s.H * 2 * (s.K + 1) < kPdlMaxBytes;
+    p.n_units = (long long)s.R * s.T * p.chunks_per_row;
+    const long long max_grid = (long long)n_sm * per_sm;
+    const long long grid = max(1ll, min(max_grid, p.n_units));
+    const bool small = (long long)s.R * s.T * s.H * 2 * (s.K + 1) < pdl_max_bytes();
     return STRATA_LAUNCH_LONG(small, dispatch_bf16_kernel, (unsigned)grid, 32, smem, st, p);
 }
 
@@ -413,13 +459,17 @@ cudaError_t launch_dispatch_fp8(const strata_moe_shape& s, const int32_t* dst_ro
     p.n_units = (long long)s.R * s.T * p.chunks_per_row;
     p.capacity_rows = (long long)capacity_rows;
     p.status = status;
-    const size_t smem = (size_t)p.chunk_cols * 6u + 64;
-    int per_sm = 0;
-    cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dispatch_fp8_kernel, kFp8Threads, smem);
+    const size_t need = (size_t)p.chunk_cols * 6u + 64;
+    // as many CTAs per SM as fit, and the request padded so that not one more does
+    int natural = 0;
+    cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&natural, dispatch_fp8_kernel, kFp8Threads, need);
     if (err != cudaSuccess) return err;
-    if (per_sm < 1) per_sm = 1;
+    size_t smem = 0;
+    int per_sm = 0;
+    err = smem_for_residency(dispatch_fp8_kernel, kFp8Threads, need, max(1, natural), kBf16MaxSmem, &smem, &per_sm);
+    if (err != cudaSuccess) return err;
     const long long grid = max(1ll, min((long long)n_sm * per_sm, p.n_units));
-    const bool small = (long long)s.R * s.T * s.H * (s.K + 2) < kPdlMaxBytes;
+    const bool small = (long long)s.R * s.T * s.H * (s.K + 2) < pdl_max_bytes();
     return STRATA_LAUNCH_LONG(small, dispatch_fp8_kernel, (unsigned)grid, kFp8Threads, smem, st, p);
 }
 

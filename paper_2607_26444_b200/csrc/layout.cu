@@ -377,26 +377,51 @@ constexpr int kSmallItems = 32 * 32 * kSmallRounds;      // per CTA
 constexpr int kLayoutCluster = 8;
 
 
+#ifdef STRATA_LAYOUT_PROBE
+#define LPROBE(k) do { if (threadIdx.x == 0) p.tile_cnt[1024 + blockIdx.x * 16 + (k)] = (int)(global_timer_ns() & 0x7fffffff); } while (0)
+#else
+#define LPROBE(k) do { } while (0)
+#endif
+
+// The two halves of a cluster barrier.  A CTA arrives as soon as it has finished reading the other
+// CTAs' shared memory and waits only before it exits, so the barrier costs no idle time.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
+// Threads that share the per-expert scan over the CTA's 32 warps: groups of E threads, each group
+// taking a contiguous run of warps (at most 8 groups, so the second step reads at most 7 partial sums).
+__host__ __device__ __forceinline__ int small_scan_groups(int E) { return max(1, min(8, kLayoutThreads / E)); }
+
 __global__ void __launch_bounds__(kLayoutThreads) layout_cluster_kernel(LayoutParams p, int n_items)
 {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
     const int n_cta = (int)cluster.num_blocks(), cta = (int)cluster.block_rank();
 
-    extern __shared__ int sm[];          // warp_cnt[32*E] | offs[E+1] | cta_cnt[E] | all_cnt[E] | warp_sums[32] | total[2] | src_cnt[R*E]
+    // warp_cnt[32*E] | offs[E+1] | cta_cnt[E] | all_cnt[E] | warp_sums[32] | total[2] | grp_sum[G*E] | grp_pre[G*E] | src_cnt[R*E]
+    extern __shared__ int sm[];
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int E = p.E;
+    const int G = small_scan_groups(E), wpg = (32 + G - 1) / G;     // warps per scan group
     int* warp_cnt = sm;
     int* offs = sm + 32 * E;
     int* cta_cnt = offs + E + 1;          // this CTA's per-expert totals, read by the other CTAs of the cluster
     int* all_cnt = cta_cnt + E;           // cluster-wide per-expert counts (local copy)
     int* warp_sums = all_cnt + E;
     int* total = warp_sums + 32;
-    int* src_cnt = total + 2;             // [R*E], only when src_expert_count is wanted
+    int* grp_sum = total + 2;             // [G, E] items per (scan group, expert)
+    int* grp_pre = grp_sum + G * E;       // [G, E] the same, as an exclusive prefix over the groups
+    int* src_cnt = grp_pre + G * E;       // [R*E], only when src_expert_count is wanted
     int* mine = warp_cnt + wid * E;
     const int ebits = key_bits(E);
 
+    // the tables do not depend on anything an earlier kernel wrote: clear them before the wait
+    for (int x = tid; x < 32 * E; x += kLayoutThreads) warp_cnt[x] = 0;
+    if (p.src_expert_count)
+        for (int x = tid; x < p.R * E; x += kLayoutThreads) src_cnt[x] = 0;
+    LPROBE(0);
     griddep_wait();
+    LPROBE(1);
     griddep_launch_dependents();
     // contiguous run per warp over all warps of the cluster, a multiple of 32 items
     const int n_warps = 32 * n_cta;
@@ -409,12 +434,14 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_cluster_kernel(LayoutPa
         const int i = first + q * 32 + lane;
         ids[q] = (q * 32 < run && i < n_items) ? p.ids[i] : -1;
     }
-    for (int x = tid; x < 32 * E; x += kLayoutThreads) warp_cnt[x] = 0;
-    if (p.src_expert_count)
-        for (int x = tid; x < p.R * E; x += kLayoutThreads) src_cnt[x] = 0;
     __syncthreads();
+    LPROBE(2);
 
-    // pass 1: per-warp counts (and per-source-rank counts, which are order independent)
+    // pass 1: per-warp counts, and for every item the number of same-id items in front of it inside its
+    // warp's run (earlier rounds from the running count, earlier lanes from the lane mask); also the
+    // per-source-rank counts, which are order independent
+    int in_warp[kSmallRounds];
+    const unsigned lt = (1u << lane) - 1u;
 #pragma unroll
     for (int q = 0; q < kSmallRounds; ++q) {
         if (q * 32 >= run) break;
@@ -428,8 +455,15 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_cluster_kernel(LayoutPa
         if (!valid) e = -1;
         ids[q] = e;
         const unsigned peers = same_key_lanes(e, ebits);
-        const bool leader = valid && lane == __ffs(peers) - 1;
-        if (leader) mine[e] += __popc(peers);
+        const int lead_lane = __ffs(peers) - 1;
+        const bool leader = valid && lane == lead_lane;
+        int old = 0;
+        if (leader) {
+            old = mine[e];
+            mine[e] = old + __popc(peers);
+        }
+        old = __shfl_sync(0xffffffffu, old, lead_lane);
+        in_warp[q] = old + __popc(peers & lt);
         if (p.src_expert_count) {
             // Source rank relative to the rank of the round's first item: defined for every lane whether or
             // not its id is valid, and in [0, 31] because a round holds 32 consecutive items.
@@ -446,19 +480,35 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_cluster_kernel(LayoutPa
         __syncwarp();
     }
     __syncthreads();
+    LPROBE(3);
 
-    // exclusive prefix over this CTA's 32 warps per expert; the totals go to cta_cnt for the cluster
-    if (tid < E) {
+    // exclusive prefix over this CTA's 32 warps per expert, in two steps: every scan group walks its own
+    // run of warps, then the groups' sums are combined.  The totals go to cta_cnt for the cluster.
+    const int sg = tid / E, se = tid - sg * E;
+    if (sg < G) {
         int running = 0;
-#pragma unroll 8
-        for (int w = 0; w < 32; ++w) {
-            const int c = warp_cnt[w * E + tid];
-            warp_cnt[w * E + tid] = running;
+        const int w_end = min(32, (sg + 1) * wpg);
+        for (int w = sg * wpg; w < w_end; ++w) {
+            const int c = warp_cnt[w * E + se];
+            warp_cnt[w * E + se] = running;
             running += c;
         }
-        cta_cnt[tid] = running;
+        grp_sum[sg * E + se] = running;
     }
+    __syncthreads();
+    if (sg < G) {
+        int before_g = 0, all_g = 0;
+        for (int g2 = 0; g2 < G; ++g2) {
+            const int v = grp_sum[g2 * E + se];
+            if (g2 < sg) before_g += v;
+            all_g += v;
+        }
+        grp_pre[sg * E + se] = before_g;
+        if (sg == 0) cta_cnt[se] = all_g;
+    }
+    LPROBE(4);
     cluster.sync();                       // every CTA's cta_cnt and src_cnt are complete and visible
+    LPROBE(5);
 
     // items with the same id in earlier CTAs of the cluster, and the cluster-wide count
     int before = 0, count_e = 0;
@@ -472,34 +522,9 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_cluster_kernel(LayoutPa
             count_e += v[c];
         }
     }
-    const int padded = round_up_rows(count_e, p.align);
-    const int off = block_exclusive_scan_1024(tid < E ? padded : 0, warp_sums, total);
-    if (tid < E) {
-        offs[tid] = off;
-        all_cnt[tid] = count_e;
-    }
-    if (tid == 0) offs[E] = *total;
-    if (cta == 0) {
-        if (tid < E) {
-            p.expert_count[tid] = count_e;
-            p.expert_offset[tid] = off;
-            if (p.src_of_row)             // padding rows of this segment have no source item
-                for (int row = off + count_e; row < off + padded; ++row) p.src_of_row[row] = -1;
-        }
-        if (tid == 0) {
-            p.expert_offset[E] = *total;
-            p.rank_offset[p.R] = *total;
-        }
-    }
-    __syncthreads();
-    if (cta == 0)
-        for (int d = tid; d < p.R; d += kLayoutThreads) {
-            p.rank_offset[d] = offs[d * p.e_loc];
-            int real = 0;
-            for (int e2 = d * p.e_loc; e2 < (d + 1) * p.e_loc; ++e2) real += all_cnt[e2];
-            p.rank_count[d] = real;
-        }
-    if (p.src_expert_count) {             // CTA c sums its contiguous slice of the per-source-rank table
+    // the other remote reads (the per-source-rank table: CTA c sums its contiguous slice) go out before
+    // the block scan, so that this CTA can tell the cluster early that it needs nobody's memory any more
+    if (p.src_expert_count) {
         const int slice = (p.R * E + n_cta - 1) / n_cta;
         const int x_end = min(p.R * E, (cta + 1) * slice);
         for (int x = cta * slice + tid; x < x_end; x += kLayoutThreads) {
@@ -513,36 +538,54 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_cluster_kernel(LayoutPa
             p.src_expert_count[x] = sum;
         }
     }
+    cluster_arrive();                     // matched by cluster_wait() before the exit
+    const int padded = round_up_rows(count_e, p.align);
+    const int off = block_exclusive_scan_1024(tid < E ? padded : 0, warp_sums, total);
+    if (tid < E) {
+        offs[tid] = off + before;         // first row of this CTA's items in each expert's segment
+        all_cnt[tid] = count_e;
+    }
+    LPROBE(6);
+    if (cta == 0) {
+        if (tid < E) {
+            p.expert_count[tid] = count_e;
+            p.expert_offset[tid] = off;
+            if (p.src_of_row)             // padding rows of this segment have no source item
+                for (int row = off + count_e; row < off + padded; ++row) p.src_of_row[row] = -1;
+            if (tid % p.e_loc == 0) p.rank_offset[tid / p.e_loc] = off;
+        }
+        if (tid == 0) {
+            p.expert_offset[E] = *total;
+            p.rank_offset[p.R] = *total;
+        }
+    }
     __syncthreads();
-    if (tid < E) offs[tid] += before;     // first row of this CTA's items in each expert's segment
-    __syncthreads();
+    if (cta == 0)
+        for (int d = tid; d < p.R; d += kLayoutThreads) {
+            int real = 0;
+            for (int e2 = d * p.e_loc; e2 < (d + 1) * p.e_loc; ++e2) real += all_cnt[e2];
+            p.rank_count[d] = real;
+        }
+    LPROBE(7);
 
-    // pass 2: rows.  mine[e] counts the same-id items of earlier warps and earlier rounds of this CTA.
-    const unsigned lt = (1u << lane) - 1u;
+    // pass 2: rows.  Everything an item needs is a table look-up away.
+    const int* my_grp = grp_pre + (wid / wpg) * E;
 #pragma unroll
     for (int q = 0; q < kSmallRounds; ++q) {
         if (q * 32 >= run) break;
         const int i = first + q * 32 + lane;
         const int e = ids[q];
-        const bool valid = e >= 0;
-        const unsigned peers = same_key_lanes(e, ebits);
-        const int leader = __ffs(peers) - 1;
-        int old = 0;
-        if (valid && lane == leader) {
-            old = mine[e];
-            mine[e] = old + __popc(peers);
-        }
-        old = __shfl_sync(0xffffffffu, old, leader);
-        if (valid) {
-            const int row = offs[e] + old + __popc(peers & lt);
+        if (e >= 0) {
+            const int row = offs[e] + my_grp[e] + mine[e] + in_warp[q];
             p.dst_row[i] = row;
             if (p.src_of_row) p.src_of_row[row] = i;
         } else if (i < n_items) {
             p.dst_row[i] = -1;
         }
-        __syncwarp();
     }
-    cluster.sync();                       // no CTA leaves while another may still read its shared memory
+    LPROBE(8);
+    cluster_wait();                       // no CTA leaves while another may still read its shared memory
+    LPROBE(9);
 }
 
 // ---- fixed-capacity layout of small batches: one launch, one CTA per source rank ---------------
@@ -679,7 +722,7 @@ __global__ void __launch_bounds__(kLayoutThreads) layout_capacity_kernel(LayoutP
 // shared memory of the cluster kernel; the per-source-rank table is only there when asked for
 size_t small_smem(int E, int R, bool with_src)
 {
-    return (size_t)(32 * E + E + 1 + E + E + 32 + 2 + (with_src ? R * E : 0)) * sizeof(int);
+    return (size_t)(32 * E + E + 1 + E + E + 32 + 2 + 2 * small_scan_groups(E) * E + (with_src ? R * E : 0)) * sizeof(int);
 }
 constexpr size_t kSmallSmemLimit = 200 * 1024;
 
