@@ -38,14 +38,28 @@ UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch at the prefill shape.  Captured with
-# ncu --set full on the same recipe at T=512 tokens/rank (1/8 of the tokens) and scaled by 8, since
-# traffic grows in proportion to the tokens (profiles/*_prefill_T512.md); None = no capture yet.
-NCU_TRAFFIC_BYTES = {
-    "dispatch_bf16_kernel": 8 * (117_720_832 + 879_663_104),
-    "dispatch_fp8_kernel": None,      # captured at its own full size (fp8 config): 134.8 MB read + 494.1 MB written
-    "combine_kernel": 8 * (940_060_928 + 98_199_296),
+# dram__bytes_read.sum and dram__bytes_write.sum per launch, captured with ncu on the prefill recipe shrunk to
+# T=512 and to T=1024 tokens/rank (the full launch is too large to capture under the profiler).  Reads grow in
+# proportion to T.  Writes are the algorithmic bytes minus a constant: the lines still dirty in the 126 MB L2
+# when the kernel ends (dispatch 63 MB, combine 15 MB at both sizes), so the traffic of a full launch is the
+# straight line through the two captures taken at T=4096, not 8 x the smaller capture
+# (profiles/dram_traffic_prefill_T512_T1024.md).
+NCU_CAPTURES = {
+    # kernel: {tokens per rank: (bytes read, bytes written)}, means of the two captured launches
+    "dispatch_bf16_kernel": {512: (117_736_064, 876_647_296), 1024: (235_501_568, 1_815_977_728)},
+    "combine_kernel": {512: (940_062_976, 103_737_856), 1024: (1_880_134_016, 219_123_840)},
 }
+
+
+def ncu_traffic_bytes(kernel: str, tokens_per_rank: int):
+    """DRAM bytes (read + written) of one launch at the prefill recipe with T = tokens_per_rank, on the line
+    through the two captures; None for a kernel without captures."""
+    cap = NCU_CAPTURES.get(kernel)
+    if not cap:
+        return None
+    (t1, (r1, w1)), (t2, (r2, w2)) = sorted(cap.items())
+    b1, b2 = r1 + w1, r2 + w2
+    return int(round(b1 + (b2 - b1) * (tokens_per_rank - t1) / (t2 - t1)))
 
 
 def measured_peak():
@@ -137,19 +151,22 @@ def oracle_sample_config(cfg: wl.MoEConfig, tokens_per_rank: int) -> wl.MoEConfi
     return wl.shrink(cfg, T=min(cfg.T, tokens_per_rank))
 
 
-def time_oracle(cfg: wl.MoEConfig, inp, reps: int):
-    """Times oracle layout+dispatch+combine (as it stands) on the given inputs, all host cores."""
+def time_oracle(cfg: wl.MoEConfig, inp, reps: int, keep=None):
+    """Times oracle layout+dispatch+combine (as it stands) on the given inputs, all host cores.
+    keep: a dict that receives the last pass's dst_row, recv and out (for a comparison with the GPU's)."""
     import oracle
     cores = oracle.max_threads()
     best = None
-    for _ in range(reps):
+    for i in range(reps):
         t0 = time.perf_counter()
         lay = oracle.layout(inp["ids"], cfg.E)
         recv = oracle.dispatch_bf16(lay["dst_row"], inp["x"], nthreads=cores)
-        oracle.combine(lay["dst_row"], recv, inp["w"], nthreads=cores)
+        out = oracle.combine(lay["dst_row"], recv, inp["w"], nthreads=cores)
         dt = time.perf_counter() - t0
         best = dt if best is None else min(best, dt)
-        del recv
+        if keep is not None and i == reps - 1:
+            keep.update(dst_row=lay["dst_row"], recv=recv, out=out)
+        del recv, out
     nbytes = cfg.dispatch_bytes() + cfg.combine_bytes()
     sample = (f"the whole workload (R={cfg.R} T={cfg.T} H={cfg.H} E={cfg.E} K={cfg.K}, seed {cfg.seed}); "
               f"layout+dispatch+combine, best of {reps}, OpenMP over tokens")
@@ -749,7 +766,7 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
         return
 
     peak, peak_src = measured_peak()
-    traffic_ok = args.workload == "prefill" and not args.tokens_per_rank   # the captures are scaled to this shape
+    traffic_ok = args.workload == "prefill"          # the captures are of this recipe
     disp_name = "dispatch_bf16_kernel" if cfg.dispatch_dtype == wl.BF16 else "dispatch_fp8_kernel"
     kernels = {
         disp_name: {"bytes": disp_bytes, "ms": disp_ms},
@@ -764,17 +781,60 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
                 "peak_source": f"{peak_src} (MEASURED_PEAKS.json hbm_gbs)" if peak_src == "measured"
                 else "fallback (recipe figure)",
                 "unit": "GB/s", "frac": kernels[dom]["frac"],
-                "traffic": NCU_TRAFFIC_BYTES.get(dom) if traffic_ok else None,
+                "traffic": ncu_traffic_bytes(dom, cfg.T) if traffic_ok else None,
+                "traffic_source": "ncu dram__bytes read+write captured at T=512 and T=1024 tokens/rank, linear in T, "
+                                  "taken at this T" if traffic_ok else None,
                 "algorithmic_bytes_per_launch": kernels[dom]["bytes"],
+                "frac_of_nominal_8TBs": round(kernels[dom]["frac_of_nominal_8TBs"], 4),
+                "note": ("frac above 1: the denominator is a measured torch copy (1:1 read:write), and this kernel "
+                         "outruns it") if kernels[dom]["frac"] > 1 else None,
                 "kernels": {k: {"achieved": round(v["achieved"], 1), "frac": round(v["frac"], 4),
                                 "frac_of_nominal_8TBs": round(v["frac_of_nominal_8TBs"], 4),
                                 "avg_ms": round(v["ms"], 4),
-                                "traffic": NCU_TRAFFIC_BYTES.get(k) if traffic_ok else None}
+                                "traffic": ncu_traffic_bytes(k, cfg.T) if traffic_ok else None}
                             for k, v in kernels.items()},
                 "layout_avg_ms": round(lay_ms, 4)}
 
+    # ---- the oracle on the host cores: timed as a baseline, and its results compared with what the
+    #      timed GPU steps left in their buffers (same inputs) ----
+    cpu, oracle_check = None, None
+    if not args.no_cpu:
+        kept = {}
+        gbs, dt, cores, sample = time_oracle(cfg, host_inp, reps=2, keep=kept)
+        cpu = {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+               "seconds": round(dt, 3)}
+        if cfg.dispatch_dtype == wl.BF16:
+            got_out = case.out.cpu().numpy().view(np.uint16)
+            a, b = got_out.astype(np.int32), kept["out"].reshape(got_out.shape).astype(np.int32)
+            a = np.where(a & 0x8000, -(a & 0x7FFF), a & 0x7FFF)
+            b = np.where(b & 0x8000, -(b & 0x7FFF), b & 0x7FFF)
+            rows = np.arange(0, cfg.n_items, max(1, cfg.n_items // 8192))
+            got_rows = case.recv[torch.from_numpy(rows).to(case.dev)].cpu().numpy().view(np.uint16)
+            oracle_check = {
+                "dst_row_equal": bool(np.array_equal(case.lay.dst_row.cpu().numpy(), kept["dst_row"])),
+                "recv_rows_equal": bool(np.array_equal(got_rows, kept["recv"][rows])), "recv_rows_compared": int(rows.size),
+                "combine_max_ulp": int(np.abs(a - b).max()), "combine_elements_compared": int(a.size)}
+            if not (oracle_check["dst_row_equal"] and oracle_check["recv_rows_equal"]
+                    and oracle_check["combine_max_ulp"] <= 1):
+                raise RuntimeError(f"the timed buffers differ from the oracle: {oracle_check}")
+            del a, b, got_out, got_rows
+        kept.clear()
+        # one thread, on a sixteenth of the tokens (same recipe)
+        import oracle
+        scfg = oracle_sample_config(cfg, max(1, cfg.T // 16))
+        sinp = wl.generate(scfg)
+        t0 = time.perf_counter()
+        lay1 = oracle.layout(sinp["ids"], scfg.E)
+        recv1 = oracle.dispatch_bf16(lay1["dst_row"], sinp["x"], nthreads=1)
+        oracle.combine(lay1["dst_row"], recv1, sinp["w"], nthreads=1)
+        dt1 = time.perf_counter() - t0
+        del recv1
+        cpu["single_thread"] = {"value": (scfg.dispatch_bytes() + scfg.combine_bytes()) / dt1 / 1e9, "unit": UNIT,
+                                "sample": f"T={scfg.T} of {cfg.T} tokens/rank, one pass", "seconds": round(dt1, 3)}
+
     # ---- the other shapes: per-call microseconds (not bench lines, context for the metric) ----
-    other = {}
+    # The second half of the metric is the time per call at the decode shape: it gets a block of its own.
+    other, decode_us = {}, None
     if not args.no_other:
         del case
         torch.cuda.empty_cache()
@@ -788,57 +848,42 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
                 "layout_us": round(us["layout"]["median_us"], 2),
                 "dispatch_us": round(us["dispatch"]["median_us"], 2),
                 "combine_us": round(us["combine"]["median_us"], 2),
-                "layout+dispatch_us": round(us["layout+dispatch"]["median_us"], 2),
                 "step_us": round(us["step"]["median_us"], 2),
-                "step_cuda_graph_us": round(us["step_graph"]["median_us"], 2),
-                "dispatch_GBs": round(db / us["dispatch"]["median_us"] / 1e3, 1),
-                "combine_GBs": round(cb / us["combine"]["median_us"] / 1e3, 1),
-                "min_p95_us": {k: [round(v["min_us"], 2), round(v["p95_us"], 2)] for k, v in us.items()},
-                "back_to_back_us": {k: round(v["back_to_back_us"], 2) for k, v in us.items() if "back_to_back_us" in v},
-                "iters": 30,
+                "step_back_to_back_us": round(us["step"]["back_to_back_us"], 2),
             }
+            if name == "decode":
+                b2b = {k: round(v["back_to_back_us"], 2) for k, v in us.items() if "back_to_back_us" in v}
+                decode_us = {
+                    "layout": other[name]["layout_us"], "dispatch": other[name]["dispatch_us"],
+                    "combine": other[name]["combine_us"], "step": other[name]["step_us"],
+                    "step_cuda_graph": round(us["step_graph"]["median_us"], 2),
+                    "back_to_back": {"layout": b2b["layout"], "dispatch": b2b["dispatch"], "combine": b2b["combine"],
+                                     "step": b2b["step"]},
+                    "of_measured_peak": {"dispatch": round(db / us["dispatch"]["median_us"] / 1e3 / peak, 3),
+                                         "combine": round(cb / us["combine"]["median_us"] / 1e3 / peak, 3),
+                                         "dispatch_back_to_back": round(db / b2b["dispatch"] / 1e3 / peak, 3),
+                                         "combine_back_to_back": round(cb / b2b["combine"] / 1e3 / peak, 3)},
+                    "both_copies_at_measured_peak_us": round((db + cb) / peak / 1e3, 1),
+                    "how": "median of 30 calls, each between two CUDA events; back_to_back: 30 calls between one "
+                           "pair of events; step = layout + dispatch + combine",
+                }
             if name == "skew":
                 # load balance under Zipf routing: per-CTA finish-time spread, and the same shape with
                 # uniform routing for comparison
-                other[name]["cta_finish_spread"] = cta_finish_spread(dc)
+                sp = cta_finish_spread(dc)
+                other[name]["cta_finish_spread"] = {"dispatch": sp["dispatch"], "combine": sp["combine"]}
                 del dc
                 torch.cuda.empty_cache()
                 uc = DeviceCase(wl.shrink(c, routing="uniform"), local_rank)
                 uu = per_call_us(uc)
                 other["skew_shape_uniform_routing"] = {
-                    "dispatch_GBs": round(db / uu["dispatch"]["median_us"] / 1e3, 1),
-                    "combine_GBs": round(cb / uu["combine"]["median_us"] / 1e3, 1),
-                    "cta_finish_spread": cta_finish_spread(uc),
+                    "dispatch_us": round(uu["dispatch"]["median_us"], 2),
+                    "combine_us": round(uu["combine"]["median_us"], 2),
                 }
                 dc = uc
             del dc
             torch.cuda.empty_cache()
 
-    if not args.no_other:
-        other["paper_window_partitioning"] = {
-            "skew": window_partitioning_report(wl.CONFIGS["skew"], local_rank, unit_rows=64),
-            "prefill": window_partitioning_report(wl.CONFIGS["prefill"], local_rank, unit_rows=128),
-        }
-        torch.cuda.empty_cache()
-        other["full_mesh_collectives"] = collectives_report(local_rank)
-
-    cpu = None
-    if not args.no_cpu:
-        gbs, dt, cores, sample = time_oracle(cfg, host_inp, reps=2)
-        cpu = {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
-               "seconds": round(dt, 3)}
-        # one thread, on a sixteenth of the tokens (same recipe)
-        import oracle
-        scfg = oracle_sample_config(cfg, max(1, cfg.T // 16))
-        sinp = wl.generate(scfg)
-        t0 = time.perf_counter()
-        lay1 = oracle.layout(sinp["ids"], scfg.E)
-        recv1 = oracle.dispatch_bf16(lay1["dst_row"], sinp["x"], nthreads=1)
-        oracle.combine(lay1["dst_row"], recv1, sinp["w"], nthreads=1)
-        dt1 = time.perf_counter() - t0
-        del recv1
-        cpu["single_thread"] = {"value": (scfg.dispatch_bytes() + scfg.combine_bytes()) / dt1 / 1e9, "unit": UNIT,
-                                "sample": f"T={scfg.T} of {cfg.T} tokens/rank, one pass", "seconds": round(dt1, 3)}
     sampler.stop()
 
     line = {
@@ -854,9 +899,10 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
                    "parallelism": "replicas only" if world > 1 else "1 GPU, 16 ranks emulated in HBM"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(n1 - n0), "roofline": roofline,
         "verified": "after the timed steps: device status clean, out == x, sampled receive rows == source rows",
+        "oracle_check": oracle_check,
         "pct_of_8TBs": {"dispatch": round(100 * kernels[disp_name]["frac_of_nominal_8TBs"], 2),
                         "combine": round(100 * kernels["combine_kernel"]["frac_of_nominal_8TBs"], 2)},
-        "other_configs": other, "cpu_baseline": cpu,
+        "decode_us": decode_us, "other_configs": other, "cpu_baseline": cpu,
     }
     print(json.dumps(line), flush=True)
     if world > 1:
@@ -885,6 +931,8 @@ def main():
                     help="print only the interference report: dispatch+combine beside a library GEMM on another stream")
     ap.add_argument("--collectives", action="store_true",
                     help="print only the report on the full-mesh collectives (one JSON object; not the bench line)")
+    ap.add_argument("--partition-report", action="store_true",
+                    help="print only the report on the paper's window partitioning at the skew and prefill shapes")
     ap.add_argument("--collective-kib", type=int, nargs="+", default=[64, 1024, 16384], help="payload per rank, KiB")
     ap.add_argument("--collective-iters", type=int, default=10)
     ap.add_argument("--collective-ops", nargs="+", default=list(COLLECTIVE_OPS), choices=COLLECTIVE_OPS)
@@ -918,6 +966,12 @@ def main():
     if args.overlap:
         if rank == 0:
             print(json.dumps(overlap_report(wl.CONFIGS[args.workload], local_rank)), flush=True)
+        return
+    if args.partition_report:
+        if rank == 0:
+            print(json.dumps({
+                "skew": window_partitioning_report(wl.CONFIGS["skew"], local_rank, unit_rows=64),
+                "prefill": window_partitioning_report(wl.CONFIGS["prefill"], local_rank, unit_rows=128)}), flush=True)
         return
     if args.collectives:
         if rank == 0:

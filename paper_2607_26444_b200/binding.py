@@ -13,7 +13,8 @@ import os
 from typing import Optional, Tuple
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libstrata_moe.so")
+# STRATA_MOE_LIB names another build of the same library (the test-hooks variant in the time-out test)
+LIB_PATH = os.environ.get("STRATA_MOE_LIB") or os.path.join(_HERE, "libstrata_moe.so")
 
 STRATA_OK = 0
 STRATA_ERR_INVALID_ARG = 1

@@ -28,27 +28,46 @@ def _deps():
     return out
 
 
-def stale() -> bool:
-    if not os.path.exists(LIB):
+# The same sources with the test hooks compiled in and a short limit on every bounded device wait: used
+# only by the test of the time-out path (tests/test_gpu_timeout.py), never by the product path.
+TEST_HOOKS_LIB = os.path.join(HERE, "libstrata_moe_testhooks.so")
+TEST_HOOKS_DEFINES = ["-DSTRATA_TEST_HOOKS", "-DSTRATA_WAIT_LIMIT=2000"]
+
+
+def stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     return any(os.path.getmtime(d) > t for d in _deps())
+
+
+def _compile(lib: str, defines, verbose: bool) -> str:
+    cmd = [_nvcc(), *NVCC_FLAGS, *defines, "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-shared",
+           *[os.path.join(CSRC, s) for s in SOURCES], "-o", lib + ".tmp"]
+    if verbose:
+        cmd.insert(1, "-Xptxas")
+        cmd.insert(2, "-v")
+        print(" ".join(cmd), file=sys.stderr)
+    subprocess.run(cmd, check=True)
+    os.replace(lib + ".tmp", lib)
+    return lib
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
     """Compile csrc/*.cu into libstrata_moe.so next to this file; returns its path."""
     if not force and not stale():
         return LIB
-    cmd = [_nvcc(), *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-shared",
-           *[os.path.join(CSRC, s) for s in SOURCES], "-o", LIB + ".tmp"]
-    if verbose:
-        cmd.insert(1, "-Xptxas")
-        cmd.insert(2, "-v")
-        print(" ".join(cmd), file=sys.stderr)
-    subprocess.run(cmd, check=True)
-    os.replace(LIB + ".tmp", LIB)
-    return LIB
+    return _compile(LIB, [], verbose)
+
+
+def build_test_hooks(force: bool = False) -> str:
+    """Compile the test-hooks variant (see TEST_HOOKS_LIB); returns its path."""
+    if not force and not stale(TEST_HOOKS_LIB):
+        return TEST_HOOKS_LIB
+    return _compile(TEST_HOOKS_LIB, TEST_HOOKS_DEFINES, False)
 
 
 if __name__ == "__main__":
     print(build(force=True, verbose="-v" in sys.argv))
+    if "--test-hooks" in sys.argv:
+        print(build_test_hooks(force=True))

@@ -338,10 +338,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within the iteration limit.
+// Bounded wait: false if the phase did not complete within the iteration limit (each try suspends the
+// thread for up to a hardware-defined time, so the default limit is seconds; test builds shorten it).
+#ifndef STRATA_WAIT_LIMIT
+#define STRATA_WAIT_LIMIT (1u << 22)
+#endif
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity)
 {
-    for (uint32_t it = 0; it < (1u << 22); ++it)
+    for (uint32_t it = 0; it < (uint32_t)(STRATA_WAIT_LIMIT); ++it)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }

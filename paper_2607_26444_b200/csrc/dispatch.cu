@@ -17,9 +17,20 @@
 //       coalesced stores.
 #include "common.cuh"
 
+#ifdef STRATA_TEST_HOOKS
+#include <atomic>
+#endif
+
 namespace strata {
 
 namespace {
+
+#ifdef STRATA_TEST_HOOKS
+// Test builds only: the next dispatch launch makes CTA 0 expect 16 bytes more than its first copy delivers,
+// so that its bounded wait runs out and the error path (status word, recovery by strata_device_status) runs
+// without any fault, trap or unbounded spin.
+std::atomic<int> g_inject_short_copy{0};
+#endif
 
 // Launch shape, measured on B200 (kernel time from the first CTA's start to the last CTA's end):
 //  - What bounds the kernel is HBM serving a 1:8 read:write mix; a variant that moved the payload through
@@ -32,6 +43,10 @@ namespace {
 //  - Cutting the last units of the batch into halves or quarters evens out the CTAs' finish times (8 us
 //    apart to 2 us apart at the decode shape) but does not shorten the kernel: the CTAs that are still
 //    running get the bandwidth of those that have left.  Pieces below 4 KB copy markedly slower.
+//  - The issuing lane is not the limiter.  A version that took its three memory round trips per unit off its
+//    path (destination rows loaded one unit early, the claim's result first read one iteration later, more
+//    store groups left in flight) issued faster but in bursts: the copy engine pushed back for 1..2 us at a
+//    time, the units per CTA spread from 13..15 to 12..17, and the kernel ran 1..2 us longer.
 //  - The shared-memory request is padded so that exactly the intended number of CTAs fits an SM (see
 //    smem_for_residency): without it a launch overlapped with its predecessor's tail is placed unevenly.
 #ifndef STRATA_BF16_STAGES
@@ -66,6 +81,7 @@ struct DispatchParams {
     int chunks_per_row;
     uint32_t chunk_cols;        // columns per chunk (last chunk of a row may be shorter)
     int stages;                 // bf16 only: depth of the ring in shared memory
+    int test_flags;             // always 0 in the shipped library
     int* status;
     WorkQueue wq;
     TraceBuf trace;
@@ -123,7 +139,11 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
         long long tok;
         uint32_t col0, bytes;
         decode(u, tok, col0, bytes);
-        mbar_expect_tx(&bars[s], bytes);
+        uint32_t expect = bytes;
+#ifdef STRATA_TEST_HOOKS
+        if ((p.test_flags & 1) && blockIdx.x == 0 && j == 0) expect += 16;
+#endif
+        mbar_expect_tx(&bars[s], expect);
         bulk_g2s(smem + (size_t)s * stage_bytes, p.x + (size_t)tok * row_bytes + (size_t)col0 * 2u, bytes, &bars[s],
                  pol);
     };
@@ -134,7 +154,8 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
 
     bool ok = true;
     StageClock wait_in(p.trace), wait_out(p.trace);
-    for (long long j = 0;; ++j) {
+    long long j = 0;
+    for (;; ++j) {
         const int s = (int)(j % n_stages);
         const uint32_t parity = (uint32_t)((j / n_stages) & 1);
         const unsigned int u = s_unit[s];
@@ -179,6 +200,14 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
             issue_load(j + n_stages - 1);
         }
         __syncwarp();
+    }
+    if (!ok) {
+        // A wait ran out.  The loads issued behind the unit that gave up may still be on their way: wait for
+        // them, again with a limit, so that nothing is written into this CTA's shared memory after it has left.
+        for (long long jj = j + 1; jj < j + n_stages - 1; ++jj) {
+            const int s2 = (int)(jj % n_stages);
+            if (s_unit[s2] != kNoUnit) mbar_wait_bounded(&bars[s2], (uint32_t)((jj / n_stages) & 1));
+        }
     }
     if (lane == 0) {
         if (!ok) report_status(p.status, STRATA_ERR_TIMEOUT);
@@ -260,7 +289,11 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
         long long tok;
         uint32_t col0, cols;
         decode(u, tok, col0, cols);
-        mbar_expect_tx(&bars[s], cols * 2u);
+        uint32_t expect = cols * 2u;
+#ifdef STRATA_TEST_HOOKS
+        if ((p.test_flags & 1) && blockIdx.x == 0 && j == 0) expect += 16;
+#endif
+        mbar_expect_tx(&bars[s], expect);
         bulk_g2s(in_stage(s), p.x + (size_t)tok * in_row_bytes + (size_t)col0 * 2u, cols * 2u, &bars[s], pol);
     };
     if (tid == 0) {
@@ -270,7 +303,8 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
     __syncthreads();
 
     bool ok = true;
-    for (long long j = 0;; ++j) {
+    long long j = 0;
+    for (;; ++j) {
         const int s = (int)(j & 1);
         const uint32_t parity = (uint32_t)((j >> 1) & 1);
         const unsigned int u = s_unit[s];
@@ -345,6 +379,8 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
         __syncthreads();                            // s_rows, s_scale and s_unit[s] are rewritten next
         tl.end(STRATA_STAGE_WORK);
     }
+    if (!ok && s_unit[(j + 1) & 1] != kNoUnit)      // the other stage's load may still be on its way
+        mbar_wait_bounded(&bars[(j + 1) & 1], (uint32_t)(((j + 1) >> 1) & 1));
     if (tid == 0) {
         if (!ok) report_status(p.status, STRATA_ERR_TIMEOUT);
         bulk_wait_read<0>();
@@ -435,6 +471,9 @@ cudaError_t launch_dispatch_bf16(const strata_moe_shape& s, const int32_t* dst_r
     cudaError_t err = smem_for_residency(dispatch_bf16_kernel, 32, need, want_per_sm, kBf16MaxSmem, &smem, &per_sm);
     if (err != cudaSuccess) return err;
     p.n_units = (long long)s.R * s.T * p.chunks_per_row;
+#ifdef STRATA_TEST_HOOKS
+    p.test_flags = g_inject_short_copy.exchange(0);
+#endif
     const long long max_grid = (long long)n_sm * per_sm;
     const long long grid = max(1ll, min(max_grid, p.n_units));
     const bool small = (long long)s.R * s.T * s.H * 2 * (s.K + 1) < pdl_max_bytes();
@@ -457,6 +496,9 @@ cudaError_t launch_dispatch_fp8(const strata_moe_shape& s, const int32_t* dst_ro
     p.chunk_cols = (uint32_t)min(s.H, kFp8MaxChunkCols);
     p.chunks_per_row = (int)(((uint32_t)s.H + p.chunk_cols - 1) / p.chunk_cols);
     p.n_units = (long long)s.R * s.T * p.chunks_per_row;
+#ifdef STRATA_TEST_HOOKS
+    p.test_flags = g_inject_short_copy.exchange(0);
+#endif
     p.capacity_rows = (long long)capacity_rows;
     p.status = status;
     const size_t need = (size_t)p.chunk_cols * 6u + 64;
@@ -474,3 +516,8 @@ cudaError_t launch_dispatch_fp8(const strata_moe_shape& s, const int32_t* dst_ro
 }
 
 }  // namespace strata
+
+#ifdef STRATA_TEST_HOOKS
+// Test builds only (not declared in the public header): arms the one-shot short-copy injection above.
+extern "C" void strata_test_inject_short_copy(int on) { strata::g_inject_short_copy.store(on ? 1 : 0); }
+#endif

@@ -50,6 +50,26 @@ def test_gpu_arm_line_on_a_small_workload():
 
 
 @pytest.mark.gpu
+def test_default_line_carries_the_decode_block_and_stays_short():
+    """Everything but the main workload is as in the default run (decode block, the other shapes), the main
+    workload is the tiny one so that the test is quick; the line must stay short enough to be kept whole."""
+    d = run_bench("--workload", "tiny", "--steps", "5", "--warmup", "3", "--no-cpu", "--no-e2e")
+    dec = d["decode_us"]
+    for k in ("layout", "dispatch", "combine", "step", "step_cuda_graph"):
+        assert 0 < dec[k] < 1000, k
+    assert set(dec["back_to_back"]) == {"layout", "dispatch", "combine", "step"}
+    assert 0.3 < dec["of_measured_peak"]["dispatch"] < 1.3 and 0.3 < dec["of_measured_peak"]["combine"] < 1.3
+    assert dec["step"] >= dec["back_to_back"]["step"] * 0.9
+    assert set(d["other_configs"]) == {"tiny", "decode", "skew", "fp8", "skew_shape_uniform_routing"}
+    for name in ("tiny", "decode", "skew", "fp8"):
+        assert {"layout_us", "dispatch_us", "combine_us", "step_us", "step_back_to_back_us"} <= set(d["other_configs"][name])
+    assert len(json.dumps(d)) < 6000
+    assert set(d["roofline"]["kernels"]) == {"dispatch_bf16_kernel", "combine_kernel"}
+    for k in d["roofline"]["kernels"].values():
+        assert k["avg_ms"] > 0 and k["achieved"] > 0
+
+
+@pytest.mark.gpu
 def test_collectives_report_mode():
     d = run_bench("--collectives", "--collective-kib", "64", "256", "--collective-iters", "3")
     assert d["R"] == 32 and set(d["sizes"]) == {"64KiB_per_rank", "256KiB_per_rank"}
