@@ -53,6 +53,8 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).argtypes = [i32, i64, vp, vp]
         L.oracle_broadcast.restype = None
         L.oracle_broadcast.argtypes = [i32, i32, i64, vp, vp]
+        L.oracle_expert_affine.restype = None
+        L.oracle_expert_affine.argtypes = [i32, i32, vp, vp, vp, vp, vp]
         L.oracle_mask_ragged.restype = None
         L.oracle_mask_ragged.argtypes = [i32, i32, i32, vp, vp]
         L.oracle_row_experts.restype = None
@@ -136,6 +138,19 @@ def row_experts(lay: Dict[str, np.ndarray], R: int, slot_capacity: int = 0) -> n
     lib().oracle_row_experts(R, E, int(slot_capacity), _p(_c(lay["expert_count"], np.int32)),
                              _p(_c(lay["expert_offset"], np.int32)), _p(_c(lay["src_expert_count"], np.int32)),
                              n_rows, _p(out))
+    return out
+
+
+def expert_affine(lay: Dict[str, np.ndarray], recv: np.ndarray, scale: np.ndarray, bias: np.ndarray) -> np.ndarray:
+    """A copy of recv uint16 [rows,H] in which every occupied row of expert e's segment has become
+    bf16(fma(f32(row), scale[e], bias[e])); padding rows keep their contents."""
+    out = _c(recv, np.uint16).copy()
+    E = lay["expert_count"].shape[0]
+    scale, bias = _c(scale, np.float32), _c(bias, np.float32)
+    assert scale.shape == (E,) and bias.shape == (E,)
+    assert out.shape[0] >= int(lay["expert_offset"][E])
+    lib().oracle_expert_affine(E, out.shape[1], _p(_c(lay["expert_count"], np.int32)),
+                               _p(_c(lay["expert_offset"], np.int32)), _p(scale), _p(bias), _p(out))
     return out
 
 

@@ -34,6 +34,10 @@
  * cap, and equality of window-major with token-major dispatch.
  * The row -> expert map: the worked examples and "a row's expert is the id of
  * the item src_of_row names".
+ * The in-place expert stand-in (tests/test_oracle_expert.py): exact rational
+ * arithmetic with one rounding, a single-rounding probe, powers of two per
+ * expert, identity constants, untouched padding rows, and an independent
+ * numpy product for bias 0.
  * For the full-mesh collectives (tests/test_oracle_collectives.py): counter
  * patterns with closed-form results, the involution of all-to-all, exact
  * integer sums, a hand-worked order-sensitive sum, all-reduce = reduce-scatter
@@ -575,6 +579,28 @@ void oracle_row_experts(int32_t R, int32_t E, int32_t C, const int32_t *expert_c
             for (int32_t j = 0; j < expert_count[e]; ++j) row_expert[(int64_t)expert_offset[e] + j] = e;
         }
     }
+}
+
+/* ------------------------------------------------------------------ */
+/* Expert stand-in that consumes the receive buffer where dispatch left */
+/* it (paper Sec. 2.2 / 8.1: the receive buffer is the input of the     */
+/* expert computation, no staging copy in between).  The paper's expert */
+/* is a grouped GEMM, which is outside this path; the stand-in keeps    */
+/* what matters here, namely that every occupied row is transformed     */
+/* with the constants of the expert that owns its segment, in place:    */
+/*   recv[row][c] = bf16_rne( fma( f32(recv[row][c]), scale[e], bias[e] ) ) */
+/* for the rows offset[e] .. offset[e]+count[e]-1 of every expert e, one */
+/* binary32 fused multiply-add and one rounding to bf16.  Padding rows  */
+/* of aligned segments are not touched.                                 */
+/* ------------------------------------------------------------------ */
+void oracle_expert_affine(int32_t E, int32_t H, const int32_t *expert_count, const int32_t *expert_offset,
+                          const float *scale, const float *bias, uint16_t *recv)
+{
+    for (int32_t e = 0; e < E; ++e)
+        for (int32_t j = 0; j < expert_count[e]; ++j) {
+            uint16_t *row = recv + ((size_t)expert_offset[e] + (size_t)j) * (size_t)H;
+            for (int32_t c = 0; c < H; ++c) row[c] = f32_to_bf16_rne(fmaf(bf16_to_f32(row[c]), scale[e], bias[e]));
+        }
 }
 
 /* ------------------------------------------------------------------ */
