@@ -292,6 +292,22 @@ strata_status strata_moe_combine(strata_ctx *ctx, const strata_moe_layout_t *lay
  * (STRATA_ERR_SHAPE otherwise).  One launch. */
 strata_status strata_moe_mask_ragged(strata_ctx *ctx, const int32_t *tokens_per_rank, int32_t *topk_ids, void *stream);
 
+/* In-place consumer of the receive buffer (paper Sec. 2.2 / 8.1: the receive buffer is the input of the expert
+ * computation, no staging copy).  The paper's expert is a grouped GEMM, which this library does not contain;
+ * this call is the hand-over part of such a consumer with a per-expert affine map standing in for the GEMM.
+ * It walks recv in tiles of tile_rows rows; every tile finds the expert e that owns it and its number of
+ * occupied rows from expert_offset / expert_count as the layout call on the same stream left them, and
+ * rewrites those rows in place:  recv[row][c] = bf16_rne(fma(f32(recv[row][c]), scale[e], bias[e]))
+ * (one binary32 fused multiply-add, one rounding).  Padding rows are not touched.  With it, layout ->
+ * dispatch -> expert -> combine runs on the device with no host step and no copy between the calls.
+ * recv: device bf16 [capacity_rows >= strata_moe_recv_rows, H] inside a registered region; scale, bias:
+ * device float [E].  tile_rows >= 1 must divide the context's segment_align (1 for packed segments), so
+ * that no tile holds rows of two experts (STRATA_ERR_SHAPE otherwise, and for e4m3 or fixed-capacity
+ * contexts).  One launch. */
+strata_status strata_moe_expert_affine_inplace(strata_ctx *ctx, const strata_moe_layout_t *layout, void *recv,
+                                               size_t capacity_rows, const float *scale, const float *bias,
+                                               int32_t tile_rows, void *stream);
+
 /* Row -> expert map of the receive buffer (production variant; the paper names no such array): the per-row
  * group index a grouped expert GEMM needs to read the receive buffer in place, completing the zero-copy
  * hand-over (with segment_align set to the GEMM's tile height, every tile of rows belongs to one expert or

@@ -41,7 +41,7 @@ EXPORTS = [
     "strata_moe_partition_max_units", "strata_moe_partition", "strata_moe_dispatch_windows",
     "strata_moe_recv_rows",
     "strata_ctx_set_timeline", "strata_timeline_decode", "strata_ctx_set_sm_budget", "strata_moe_row_experts",
-    "strata_moe_mask_ragged",
+    "strata_moe_mask_ragged", "strata_moe_expert_affine_inplace",
     "strata_allgather", "strata_alltoall", "strata_broadcast", "strata_reducescatter", "strata_allreduce",
     "strata_p2p", "strata_alltoallv",
 ]
@@ -144,6 +144,7 @@ def lib() -> ctypes.CDLL:
         "strata_ctx_set_sm_budget": [vp, i32],
         "strata_moe_row_experts": [vp, P(strata_moe_layout_t), vp, sz, vp],
         "strata_moe_mask_ragged": [vp, vp, vp, vp],
+        "strata_moe_expert_affine_inplace": [vp, P(strata_moe_layout_t), vp, sz, vp, vp, i32, vp],
         "strata_ctx_set_timeline": [vp, vp, sz, sz],
         "strata_timeline_decode": [vp, sz, sz, vp, sz, P(sz), P(sz)],
         "strata_allgather": [vp, i32, vp, vp, sz, vp],
@@ -293,6 +294,12 @@ def strata_moe_row_experts(ctx, layout: strata_moe_layout_t, row_expert: int, ca
 
 def strata_moe_mask_ragged(ctx, tokens_per_rank: int, topk_ids: int, stream: int) -> int:
     return lib().strata_moe_mask_ragged(ctx, tokens_per_rank, topk_ids, stream)
+
+
+def strata_moe_expert_affine_inplace(ctx, layout: strata_moe_layout_t, recv: int, capacity_rows: int, scale: int,
+                                     bias: int, tile_rows: int, stream: int) -> int:
+    return lib().strata_moe_expert_affine_inplace(ctx, ctypes.byref(layout), recv, capacity_rows, scale, bias,
+                                                  tile_rows, stream)
 
 
 def strata_ctx_set_sm_budget(ctx, n_sm: int) -> int:
@@ -479,6 +486,12 @@ class MoEContext:
         """Marks, in place, the slots of the tokens t >= tokens_per_rank[r] as not routed (-1)."""
         _check(strata_moe_mask_ragged(self.h, tokens_per_rank.data_ptr(), ids.data_ptr(), self._stream()),
                "strata_moe_mask_ragged")
+
+    def expert_affine_inplace(self, layout: Layout, recv, scale, bias, tile_rows: int = 1) -> None:
+        """recv[row] = bf16(fma(recv[row], scale[e], bias[e])) for every occupied row, in place, tile by tile."""
+        _check(strata_moe_expert_affine_inplace(self.h, layout.c, recv.data_ptr(), recv.shape[0], scale.data_ptr(),
+                                                bias.data_ptr(), tile_rows, self._stream()),
+               "strata_moe_expert_affine_inplace")
 
     def row_experts(self, layout: Layout, out=None):
         """int32 [recv_rows]: the expert of every occupied receive row, -1 for padding and empty rows."""

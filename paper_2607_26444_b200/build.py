@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libstrata_moe.so")
-SOURCES = ["api.cu", "layout.cu", "dispatch.cu", "combine.cu", "partition.cu", "collective.cu", "rowmap.cu"]
+SOURCES = ["api.cu", "layout.cu", "dispatch.cu", "combine.cu", "partition.cu", "collective.cu", "rowmap.cu", "expert.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "-cudart", "static"]
 

@@ -448,6 +448,36 @@ strata_status strata_moe_combine(strata_ctx* ctx, const strata_moe_layout_t* lay
     return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
 }
 
+strata_status strata_moe_expert_affine_inplace(strata_ctx* ctx, const strata_moe_layout_t* layout, void* recv,
+                                               size_t capacity_rows, const float* scale, const float* bias,
+                                               int32_t tile_rows, void* stream)
+{
+    if (!ctx || !layout || !recv || !scale || !bias) return STRATA_ERR_INVALID_ARG;
+    if (!layout->expert_count || !layout->expert_offset) return STRATA_ERR_INVALID_ARG;
+    const strata_moe_shape& s = ctx->shape;
+    if (s.dispatch_dtype != STRATA_BF16 || s.slot_capacity > 0) return STRATA_ERR_SHAPE;
+    const int align = s.segment_align > 1 ? s.segment_align : 1;
+    if (tile_rows < 1 || align % tile_rows != 0) return STRATA_ERR_SHAPE;    // a tile must never hold two experts
+    if (!aligned16(recv)) return STRATA_ERR_ALIGNMENT;
+    const size_t n_rows = (size_t)recv_rows(s);
+    if (capacity_rows < n_rows) return STRATA_ERR_CAPACITY;
+    {
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        if (!region_contains(ctx, recv, capacity_rows * (size_t)s.H * 2)) return STRATA_ERR_NOT_REGISTERED;
+    }
+    if (ctx->device < 0) return STRATA_ERR_CUDA;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return STRATA_ERR_CUDA;
+    cudaError_t err = launch_expert_affine(s, *layout, recv, (long long)n_rows, scale, bias, tile_rows, ctx->n_sm,
+                                           static_cast<cudaStream_t>(stream));
+    {
+        std::lock_guard<std::mutex> lk(ctx->mu);
+        ctx->launches += 1;
+    }
+    if (err != cudaSuccess) cudaGetLastError();
+    return err == cudaSuccess ? STRATA_OK : STRATA_ERR_CUDA;
+}
+
 strata_status strata_moe_mask_ragged(strata_ctx* ctx, const int32_t* tokens_per_rank, int32_t* topk_ids, void* stream)
 {
     if (!ctx || !tokens_per_rank || !topk_ids) return STRATA_ERR_INVALID_ARG;

@@ -134,6 +134,8 @@ cudaError_t launch_mask_ragged(const strata_moe_shape& s, const int32_t* tokens_
                                cudaStream_t st);
 cudaError_t launch_row_experts(const strata_moe_shape& s, const strata_moe_layout_t& L, int32_t* row_expert,
                                long long n_rows, cudaStream_t st);
+cudaError_t launch_expert_affine(const strata_moe_shape& s, const strata_moe_layout_t& L, void* recv, long long n_rows,
+                                 const float* scale, const float* bias, int tile_rows, int n_sm, cudaStream_t st);
 int partition_max_units_supported();
 int partition_max_cores_supported();
 uint32_t windows_max_row_bytes();
