@@ -246,6 +246,8 @@ class DeviceCase:
         inp = inp or wl.generate(cfg)
         self.inp = inp
         self.ctx = B.MoEContext(cfg.R, cfg.T, cfg.H, cfg.E, cfg.K, cfg.dispatch_dtype, device=dev_index)
+        # x exists before routing starts (here: before the first step), so dispatch may read it while the layout runs
+        self.ctx.x_early(True)
         self.ids = torch.from_numpy(inp["ids"]).to(dev)
         self.x = torch.from_numpy(inp["x"].view(np.int16)).to(dev)
         self.w = torch.from_numpy(inp["w"]).to(dev)
@@ -894,7 +896,8 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
                                f"E={cfg.E}, K={cfg.K} {cfg.routing} distinct experts, softmax gates, "
                                + ("identity experts (combine reads recv)" if cfg.dispatch_dtype == wl.BF16
                                   else "e4m3 dispatch, bf16 expert outputs"),
-                   "step": "strata_moe_layout + strata_moe_dispatch + strata_moe_combine",
+                   "step": "strata_moe_layout + strata_moe_dispatch + strata_moe_combine (x_early promise on: x is "
+                           "complete before the layout call)",
                    "bytes_per_step": step_bytes, "l2": "inputs larger than L2 (8.4 GB working set), no flush",
                    "parallelism": "replicas only" if world > 1 else "1 GPU, 16 ranks emulated in HBM"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(n1 - n0), "roofline": roofline,

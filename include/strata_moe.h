@@ -139,6 +139,18 @@ strata_status strata_ctx_launch_count(strata_ctx *ctx, uint64_t *count);
  * affected. */
 strata_status strata_ctx_set_sm_budget(strata_ctx *ctx, int32_t n_sm);
 
+/* A promise about the caller's stream order that lets dispatch start earlier (paper Sec. 5.2 / 6.2 want the
+ * transfer issued as soon as its operands exist; the paper defines no such call).  In an MoE layer the hidden
+ * states x exist before routing starts, while dispatch is enqueued right behind the layout call.  on != 0
+ * promises, for every later strata_moe_dispatch on this context: the x passed to it is complete before the
+ * operation that directly precedes that dispatch call in its stream STARTS, and nothing writes x until the
+ * dispatch has finished.  Dispatch, which is launched so that its prologue overlaps the preceding kernel, then
+ * loads its first rows of x while that kernel (normally the layout) is still running; only its stores wait for
+ * the layout.  Measured at the decode shape: 1.5 us off a 90 us step.  Off (0) by default: without the promise
+ * dispatch reads x only after everything before it in the stream has finished.  A broken promise yields stale
+ * rows, never an out-of-bounds access.  strata_moe_roundtrip_host never uses it. */
+strata_status strata_ctx_set_x_early(strata_ctx *ctx, int32_t on);
+
 /* Per-CTA stage probes (after the paper's in-kernel profiler, Sec. 6.4: probes at stage boundaries
  * writing a cycle counter into a per-core slice of a trace buffer).  dptr: device array of
  * 4*capacity_ctas uint64, owned by the caller; while set, CTA b (b < capacity_ctas) of every

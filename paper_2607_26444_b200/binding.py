@@ -41,7 +41,7 @@ EXPORTS = [
     "strata_moe_partition_max_units", "strata_moe_partition", "strata_moe_dispatch_windows",
     "strata_moe_recv_rows",
     "strata_ctx_set_timeline", "strata_timeline_decode", "strata_ctx_set_sm_budget", "strata_moe_row_experts",
-    "strata_moe_mask_ragged", "strata_moe_expert_affine_inplace",
+    "strata_moe_mask_ragged", "strata_moe_expert_affine_inplace", "strata_ctx_set_x_early",
     "strata_allgather", "strata_alltoall", "strata_broadcast", "strata_reducescatter", "strata_allreduce",
     "strata_p2p", "strata_alltoallv",
 ]
@@ -142,6 +142,7 @@ def lib() -> ctypes.CDLL:
                                  P(strata_partition_t), sz, vp],
         "strata_moe_dispatch_windows": [vp, P(strata_moe_layout_t), P(strata_partition_t), i32, vp, vp, sz, vp],
         "strata_ctx_set_sm_budget": [vp, i32],
+        "strata_ctx_set_x_early": [vp, i32],
         "strata_moe_row_experts": [vp, P(strata_moe_layout_t), vp, sz, vp],
         "strata_moe_mask_ragged": [vp, vp, vp, vp],
         "strata_moe_expert_affine_inplace": [vp, P(strata_moe_layout_t), vp, sz, vp, vp, i32, vp],
@@ -300,6 +301,10 @@ def strata_moe_expert_affine_inplace(ctx, layout: strata_moe_layout_t, recv: int
                                      bias: int, tile_rows: int, stream: int) -> int:
     return lib().strata_moe_expert_affine_inplace(ctx, ctypes.byref(layout), recv, capacity_rows, scale, bias,
                                                   tile_rows, stream)
+
+
+def strata_ctx_set_x_early(ctx, on: int) -> int:
+    return lib().strata_ctx_set_x_early(ctx, int(on))
 
 
 def strata_ctx_set_sm_budget(ctx, n_sm: int) -> int:
@@ -519,6 +524,10 @@ class MoEContext:
     def trace_off(self) -> None:
         _check(strata_ctx_set_trace(self.h, None, 0), "strata_ctx_set_trace")
         self._trace = None
+
+    def x_early(self, on: bool = True) -> None:
+        """Promise that x is complete before the call preceding each dispatch starts (see the header)."""
+        _check(strata_ctx_set_x_early(self.h, 1 if on else 0), "strata_ctx_set_x_early")
 
     def sm_budget(self, n_sm: int) -> None:
         """Sizes the persistent grids for n_sm SMs (0: the whole GPU)."""

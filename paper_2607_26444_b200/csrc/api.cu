@@ -26,6 +26,7 @@ struct strata_ctx {
     int device;
     int n_sm;             // SMs the persistent kernels size their grids for (the device's, or the caller's budget)
     int n_sm_device;
+    int x_early;          // the caller's promise about x (strata_ctx_set_x_early)
     int* ws;              // device workspace (header + tile counts)
     size_t ws_bytes;
     uint64_t next_region;
@@ -153,6 +154,7 @@ strata_status strata_ctx_create(strata_ctx** out, const strata_moe_shape* shape,
     c->device = device;
     c->n_sm = n_sm;
     c->n_sm_device = n_sm;
+    c->x_early = 0;
     c->ws = nullptr;
     c->ws_bytes = 0;
     c->next_region = 1;
@@ -232,6 +234,14 @@ strata_status strata_ctx_set_sm_budget(strata_ctx* ctx, int32_t n_sm)
     if (!ctx || n_sm < 0) return STRATA_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lk(ctx->mu);
     ctx->n_sm = (n_sm == 0 || n_sm > ctx->n_sm_device) ? ctx->n_sm_device : n_sm;
+    return STRATA_OK;
+}
+
+strata_status strata_ctx_set_x_early(strata_ctx* ctx, int32_t on)
+{
+    if (!ctx) return STRATA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(ctx->mu);
+    ctx->x_early = on ? 1 : 0;
     return STRATA_OK;
 }
 
@@ -418,9 +428,9 @@ strata_status strata_moe_dispatch(strata_ctx* ctx, const strata_moe_layout_t* la
     if (!g.ok) return STRATA_ERR_CUDA;
     cudaError_t err =
         fp8 ? launch_dispatch_fp8(s, layout->dst_row, x, recv, recv_scale, capacity_rows, ctx->ws, dispatch_queue(ctx),
-                                  ctx->n_sm, ctx->trace, static_cast<cudaStream_t>(stream))
+                                  ctx->n_sm, ctx->trace, ctx->x_early != 0, static_cast<cudaStream_t>(stream))
             : launch_dispatch_bf16(s, layout->dst_row, x, recv, capacity_rows, ctx->ws, dispatch_queue(ctx), ctx->n_sm,
-                                   ctx->trace, static_cast<cudaStream_t>(stream));
+                                   ctx->trace, ctx->x_early != 0, static_cast<cudaStream_t>(stream));
     {
         std::lock_guard<std::mutex> lk(ctx->mu);
         ctx->launches += 1;
@@ -872,7 +882,7 @@ strata_status strata_moe_roundtrip_host(strata_ctx* ctx, const strata_moe_device
             cq = combine_queue(ctx);
         }
         cudaError_t err = launch_dispatch_bf16(sub, dev->layout.dst_row + a * s.K, dx + a * row_bytes, dev->recv, n_recv,
-                                               ctx->ws, dq, ctx->n_sm, TraceBuf{nullptr, 0, nullptr, 0, 0}, st);
+                                               ctx->ws, dq, ctx->n_sm, TraceBuf{nullptr, 0, nullptr, 0, 0}, false, st);
         if (err == cudaSuccess)
             err = launch_combine(sub, dev->layout.dst_row + a * s.K, dev->recv, n_recv, dev->w + a * s.K,
                                  dout + a * row_bytes, ctx->ws, cq, ctx->n_sm, TraceBuf{nullptr, 0, nullptr, 0, 0}, st);

@@ -103,12 +103,14 @@ struct TraceBuf {
 // ---- launchers (defined next to their kernels) -----------------------------
 cudaError_t launch_layout(const strata_moe_shape& s, const int32_t* ids, const strata_moe_layout_t& L,
                           int* ws_header, int* tile_cnt, cudaStream_t st, int* n_launches);
+// x_early: the caller promised that x is complete before the kernel preceding dispatch in the stream starts,
+// so the first rows may be loaded before that kernel has finished (see strata_ctx_set_x_early)
 cudaError_t launch_dispatch_bf16(const strata_moe_shape& s, const int32_t* dst_row, const void* x, void* recv,
                                  size_t capacity_rows, int* status, WorkQueue wq, int n_sm, TraceBuf trace,
-                                 cudaStream_t st);
+                                 bool x_early, cudaStream_t st);
 cudaError_t launch_dispatch_fp8(const strata_moe_shape& s, const int32_t* dst_row, const void* x, void* recv_q,
                                 float* recv_scale, size_t capacity_rows, int* status, WorkQueue wq, int n_sm,
-                                TraceBuf trace, cudaStream_t st);
+                                TraceBuf trace, bool x_early, cudaStream_t st);
 cudaError_t launch_combine(const strata_moe_shape& s, const int32_t* dst_row, const void* y, size_t y_rows,
                            const float* w, void* out, int* status, WorkQueue wq, int n_sm, TraceBuf trace,
                            cudaStream_t st);

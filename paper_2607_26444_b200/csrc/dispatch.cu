@@ -82,6 +82,7 @@ struct DispatchParams {
     uint32_t chunk_cols;        // columns per chunk (last chunk of a row may be shorter)
     int stages;                 // bf16 only: depth of the ring in shared memory
     int test_flags;             // always 0 in the shipped library
+    int x_early;                // the first loads of x may go out before the preceding kernel has finished
     int* status;
     WorkQueue wq;
     TraceBuf trace;
@@ -107,10 +108,6 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
     }
     __syncwarp();
     const uint64_t pol = policy_evict_first();
-    griddep_wait();                       // x and dst_row belong to earlier kernels in the stream
-    if (lane == 0) trace_begin(p.trace);
-    Timeline tl(p.trace, STRATA_KERNEL_DISPATCH_BF16, lane == 0);
-    tl.begin(STRATA_STAGE_KERNEL);
 
     auto decode = [&](unsigned int u, long long& tok, uint32_t& col0, uint32_t& bytes) {
         tok = u / (unsigned int)p.chunks_per_row;
@@ -118,7 +115,7 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
         col0 = ch * p.chunk_cols;
         bytes = min(p.chunk_cols, (uint32_t)p.H - col0) * 2u;
     };
-    bool triggered = false, exhausted = false;
+    bool triggered = false, exhausted = false, waited = false;
     // The first stages-1 units of a CTA are fixed (blockIdx + j*grid); the rest are claimed.
     const unsigned int n_static = (unsigned int)(n_stages - 1) * gridDim.x;
     auto issue_load = [&](long long j) {   // lane 0 only: next unit into stage j % stages
@@ -132,8 +129,12 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
         }
         s_unit[s] = u;
         if (u == kNoUnit) {
-            if (!triggered) griddep_launch_dependents();   // queue empty: the next kernel may be scheduled
-            triggered = true;
+            // queue empty: the next kernel may be scheduled (never before this kernel's own wait: a dependent
+            // must not start before our predecessor has finished)
+            if (waited && !triggered) {
+                griddep_launch_dependents();
+                triggered = true;
+            }
             return;
         }
         long long tok;
@@ -148,8 +149,24 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
                  pol);
     };
 
-    if (lane == 0)
+    // The first stages-1 units are fixed, so their loads need nothing from the layout: when the caller has
+    // promised that x was complete before the preceding kernel started, they go out before the wait and are
+    // in shared memory by the time the layout is done.  dst_row and the claim counter are touched after it.
+    if (p.x_early && lane == 0)
         for (long long j = 0; j < n_stages - 1; ++j) issue_load(j);
+    griddep_wait();                       // dst_row (and, without the promise, x) belong to earlier kernels in the stream
+    if (lane == 0) trace_begin(p.trace);
+    Timeline tl(p.trace, STRATA_KERNEL_DISPATCH_BF16, lane == 0);
+    tl.begin(STRATA_STAGE_KERNEL);
+    waited = true;
+    if (lane == 0) {
+        if (!p.x_early)
+            for (long long j = 0; j < n_stages - 1; ++j) issue_load(j);
+        else if (s_unit[(n_stages - 2) % n_stages] == kNoUnit) {   // fewer fixed units than stages: nothing left to claim
+            griddep_launch_dependents();
+            triggered = true;
+        }
+    }
     __syncwarp();
 
     bool ok = true;
@@ -258,10 +275,6 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
     }
     __syncthreads();
     const uint64_t pol = policy_evict_first();
-    griddep_wait();
-    if (tid == 0) trace_begin(p.trace);
-    Timeline tl(p.trace, STRATA_KERNEL_DISPATCH_FP8, tid == 0);
-    tl.begin(STRATA_STAGE_KERNEL);
 
     auto decode = [&](unsigned int u, long long& tok, uint32_t& col0, uint32_t& cols) {
         tok = u / (unsigned int)p.chunks_per_row;
@@ -269,7 +282,7 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
         col0 = ch * p.chunk_cols;
         cols = min(p.chunk_cols, (uint32_t)p.H - col0);
     };
-    bool triggered = false, exhausted = false;
+    bool triggered = false, exhausted = false, waited = false;
     const unsigned int n_static = 2u * gridDim.x;   // the first two units of a CTA are fixed
     auto issue_load = [&](long long j) {   // thread 0 only
         const int s = (int)(j & 1);
@@ -282,8 +295,10 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
         }
         s_unit[s] = u;
         if (u == kNoUnit) {
-            if (!triggered) griddep_launch_dependents();   // queue empty: the next kernel may be scheduled
-            triggered = true;
+            if (waited && !triggered) {                    // queue empty: the next kernel may be scheduled
+                griddep_launch_dependents();
+                triggered = true;
+            }
             return;
         }
         long long tok;
@@ -296,9 +311,23 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
         mbar_expect_tx(&bars[s], expect);
         bulk_g2s(in_stage(s), p.x + (size_t)tok * in_row_bytes + (size_t)col0 * 2u, cols * 2u, &bars[s], pol);
     };
-    if (tid == 0) {
+    if (p.x_early && tid == 0) {          // the two fixed units need nothing from the layout (see the bf16 kernel)
         issue_load(0);
         issue_load(1);
+    }
+    griddep_wait();
+    if (tid == 0) trace_begin(p.trace);
+    Timeline tl(p.trace, STRATA_KERNEL_DISPATCH_FP8, tid == 0);
+    tl.begin(STRATA_STAGE_KERNEL);
+    waited = true;
+    if (tid == 0) {
+        if (!p.x_early) {
+            issue_load(0);
+            issue_load(1);
+        } else if (s_unit[1] == kNoUnit) {
+            griddep_launch_dependents();
+            triggered = true;
+        }
     }
     __syncthreads();
 
@@ -443,9 +472,10 @@ cudaError_t configure_dispatch_kernels()
 
 cudaError_t launch_dispatch_bf16(const strata_moe_shape& s, const int32_t* dst_row, const void* x, void* recv,
                                  size_t capacity_rows, int* status, WorkQueue wq, int n_sm, TraceBuf trace,
-                                 cudaStream_t st)
+                                 bool x_early, cudaStream_t st)
 {
     DispatchParams p{};
+    p.x_early = x_early ? 1 : 0;
     p.trace = trace;
     p.wq = wq;
     p.dst_row = dst_row;
@@ -482,9 +512,10 @@ cudaError_t launch_dispatch_bf16(const strata_moe_shape& s, const int32_t* dst_r
 
 cudaError_t launch_dispatch_fp8(const strata_moe_shape& s, const int32_t* dst_row, const void* x, void* recv_q,
                                 float* recv_scale, size_t capacity_rows, int* status, WorkQueue wq, int n_sm,
-                                TraceBuf trace, cudaStream_t st)
+                                TraceBuf trace, bool x_early, cudaStream_t st)
 {
     DispatchParams p{};
+    p.x_early = x_early ? 1 : 0;
     p.trace = trace;
     p.wq = wq;
     p.dst_row = dst_row;

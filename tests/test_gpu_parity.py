@@ -54,7 +54,7 @@ def guarded(n_rows: int, width: int, dtype, fill):
     return whole, whole[GUARD:GUARD + n_rows]
 
 
-def run_full_case(cfg: wl.MoEConfig, inp=None, threads=8):
+def run_full_case(cfg: wl.MoEConfig, inp=None, threads=8, x_early=False):
     """Whole path on one config, every output compared with the oracle element by element."""
     inp = inp or wl.generate(cfg)
     ref_lay = oracle.layout(inp["ids"], cfg.E)
@@ -62,6 +62,8 @@ def run_full_case(cfg: wl.MoEConfig, inp=None, threads=8):
     fp8 = cfg.dispatch_dtype == wl.FP8_E4M3_B128
 
     ctx = make_ctx(cfg)
+    if x_early:
+        ctx.x_early(True)
     ids_d, x_d, w_d = to_dev(inp["ids"]), to_dev(inp["x"]), to_dev(inp["w"])
     lay = ctx.layout(ids_d)
     assert_layout_equal(lay, ref_lay)
@@ -123,6 +125,55 @@ def test_skew_full():
 
 def test_fp8_full():
     run_full_case(wl.CONFIGS["fp8"])
+
+
+@pytest.mark.parametrize("name", ["tiny", "decode", "skew", "fp8"])
+def test_full_configs_with_the_early_x_promise(name):
+    """The same comparisons with dispatch allowed to load its first rows before the layout has finished."""
+    run_full_case(wl.CONFIGS[name], x_early=True)
+
+
+@pytest.mark.parametrize("kw", [dict(R=1, T=3, H=64, E=2, K=1), dict(R=2, T=100, H=16384, E=4, K=3),
+                                dict(R=4, T=300, H=1920, E=32, K=8)],
+                         ids=lambda kw: "R{R}T{T}H{H}E{E}K{K}".format(**kw))
+@pytest.mark.parametrize("fp8", [False, True], ids=["bf16", "e4m3"])
+def test_early_x_promise_over_several_steps_with_x_rewritten_before_each_layout(kw, fp8):
+    """Three steps in one stream; before each layout call a copy kernel rewrites x (the promise holds: x is
+    complete before the call preceding dispatch starts).  Fewer units than ring stages in the first shape."""
+    if fp8 and kw["H"] % 128:
+        pytest.skip("e4m3 dispatch needs H % 128 == 0")
+    cfg = wl.shrink(wl.CONFIGS["fp8" if fp8 else "tiny"], seed=606, **kw)
+    ctx = make_ctx(cfg)
+    ctx.x_early(True)
+    N, H = cfg.n_items, cfg.H
+    recv = torch.zeros((N, H), dtype=torch.uint8 if fp8 else torch.int16, device=DEV)
+    scale = torch.zeros((N, H // 128), dtype=torch.float32, device=DEV) if fp8 else None
+    ctx.register(recv)
+    if fp8:
+        ctx.register(scale)
+    x_d = torch.zeros((cfg.n_tok, H), dtype=torch.int16, device=DEV)
+    ids_d = torch.zeros((cfg.R, cfg.T, cfg.K), dtype=torch.int32, device=DEV)
+    lay = ctx.new_layout()
+    inputs = [wl.generate(wl.shrink(cfg, seed=700 + i)) for i in range(3)]
+    staged = [(to_dev(i["ids"]), to_dev(i["x"]).view(cfg.n_tok, H)) for i in inputs]
+    got = []
+    for ids_s, x_s in staged:                      # everything is enqueued before anything is read back
+        ids_d.copy_(ids_s)
+        x_d.copy_(x_s)
+        ctx.layout(ids_d, lay)
+        ctx.dispatch(lay, x_d, recv, scale)
+        got.append((recv.clone(), scale.clone() if fp8 else None))
+    torch.cuda.synchronize()
+    assert ctx.device_status() == B.STRATA_OK
+    for inp, (r, sc) in zip(inputs, got):
+        ref = oracle.layout(inp["ids"], cfg.E)
+        if fp8:
+            q, s_ = oracle.dispatch_fp8(ref["dst_row"], inp["x"], nthreads=4)
+            assert np.array_equal(r.cpu().numpy(), q)
+            assert np.array_equal(sc.cpu().numpy().view(np.uint32), s_.view(np.uint32))
+        else:
+            assert np.array_equal(u16(r), oracle.dispatch_bf16(ref["dst_row"], inp["x"], nthreads=4))
+    ctx.close()
 
 
 def test_prefill_full_size_sampled():
