@@ -45,7 +45,7 @@ def lib() -> ctypes.CDLL:
         L.oracle_e4m3_encode.restype = ctypes.c_uint8
         L.oracle_e4m3_encode.argtypes = [ctypes.c_float]
         L.oracle_partition.restype = i64
-        L.oracle_partition.argtypes = [i32, i32, i64, i32, vp, vp, vp, i32, i32, i32, i64, vp, vp, vp, vp, vp, vp]
+        L.oracle_partition.argtypes = [i32, i32, i64, i32, vp, vp, vp, i32, i32, i32, i64, vp, vp, vp, vp, vp, vp, vp]
         L.oracle_dispatch_windows.restype = None
         L.oracle_dispatch_windows.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         for name in ("oracle_allgather", "oracle_alltoall", "oracle_reducescatter", "oracle_allreduce"):
@@ -233,17 +233,20 @@ def partition(lay: Dict[str, np.ndarray], row_bytes: int, n_cores: int, tiers, g
         "unit_cost": np.zeros(max_units, np.int64),
         "task_offset": np.zeros(n_cores + 1, np.int32),
         "task_unit": np.zeros(max_units, np.int32),
+        "task_stripe": np.zeros(max_units, np.int32),
         "core_load": np.zeros(n_cores, np.int64),
     }
     U = lib().oracle_partition(R, E, row_bytes, n_cores, _p(sec), _p(off), _p(t), len(t), g0, g1, max_units,
                                _p(out["win_base"]), _p(out["unit_desc"]), _p(out["unit_cost"]),
-                               _p(out["task_offset"]), _p(out["task_unit"]), _p(out["core_load"]))
+                               _p(out["task_offset"]), _p(out["task_unit"]), _p(out["task_stripe"]),
+                               _p(out["core_load"]))
     if U < 0:
-        raise ValueError("more units than max_units")
+        raise ValueError("more units than max_units" if U == -1 else "a tier's cap, unit size or bandwidth is below 1")
     out["n_units"] = int(U)
     out["unit_desc"] = out["unit_desc"][:U]
     out["unit_cost"] = out["unit_cost"][:U]
     out["task_unit"] = out["task_unit"][:U]
+    out["task_stripe"] = out["task_stripe"][:U]
     return out
 
 

@@ -404,16 +404,21 @@ void oracle_combine(int64_t n_tok, int32_t K, int32_t H,
 /*    in integer cost units.                                            */
 /*  list scheduling (Sec. 6.2, App. B "LPT-style"): units sorted by     */
 /*    cost, largest first (ties: lower unit id first); each unit goes   */
-/*    to the least-loaded core (ties: lower core id) among the cores    */
-/*    whose next issue stripe still has room for the unit's destination */
-/*    rank, F[stripe][d] < H_t; a core's stripe index is the number of  */
-/*    units it already holds.  If no core is feasible the cap is        */
-/*    relaxed for that unit (this build's reading: the paper does not   */
-/*    say what happens then).                                           */
+/*    to the least-loaded core (ties: lower core id) and, on that core, */
+/*    into the earliest issue stripe after the core's previous unit     */
+/*    that still has room for the unit's destination rank,              */
+/*    F[stripe][d] < H_t.  This build's reading of Sec. 6.2: a core     */
+/*    issues AT MOST one unit per stripe (x_{c,k,j} in {0,1}), so it    */
+/*    may leave a stripe empty, and the number of stripes is not        */
+/*    bounded; the cap F_{k,p} <= H_t can then always be met by moving  */
+/*    a unit to a later stripe and never forces a unit onto a more      */
+/*    loaded core.  The predicted loads L_c are those of plain LPT; the */
+/*    cap shows in the stripe indices only (task_stripe).               */
 /* Tiers (stand-in for the fabric's die / node / inter-node levels):    */
 /*   tier(r,d) = 0 if r/g0 == d/g0, else 1 if r/g1 == d/g1, else 2,     */
 /*   clamped to n_tiers-1.                                              */
-/* Returns the number of units, or -1 if it exceeds max_units.          */
+/* Returns the number of units, -1 if it exceeds max_units, -2 for a    */
+/* tier with a cap, unit size or bandwidth below 1.                     */
 /* ------------------------------------------------------------------ */
 typedef struct {
     int64_t alpha;        /* fixed cost of one unit                    */
@@ -439,9 +444,12 @@ int64_t oracle_partition(int32_t R, int32_t E, int64_t row_bytes, int32_t n_core
                          int64_t *unit_cost,                /* [max_units]    */
                          int32_t *task_offset,              /* [n_cores+1]    */
                          int32_t *task_unit,                /* [max_units]    */
+                         int32_t *task_stripe,              /* [max_units] issue stripe of every entry of task_unit */
                          int64_t *core_load)                /* [n_cores]      */
 {
     const int32_t E_loc = E / R;
+    for (int32_t t = 0; t < n_tiers; ++t)
+        if (tiers[t].fanout_cap < 1 || tiers[t].unit_rows < 1 || tiers[t].beta < 1) return -2;   /* not a policy */
     /* level 2: base row of every expert window */
     for (int32_t e = 0; e < E; ++e) {
         int32_t row = expert_offset[e];
@@ -478,32 +486,41 @@ int64_t oracle_partition(int32_t R, int32_t E, int64_t row_bytes, int32_t n_core
         }
         order[k] = (int32_t)j;
     }
-    /* list scheduling under the stripe-level fan-out cap */
-    int32_t *len = (int32_t *)calloc((size_t)n_cores, sizeof(int32_t));
-    int32_t *fan = (int32_t *)calloc((size_t)(U > 0 ? U : 1) * R, sizeof(int32_t));   /* F[stripe][d] */
+    /* list scheduling; the stripe-level fan-out cap decides the stripe, not the core */
+    int32_t *len = (int32_t *)calloc((size_t)n_cores, sizeof(int32_t));       /* units a core holds       */
+    int32_t *next = (int32_t *)calloc((size_t)n_cores, sizeof(int32_t));      /* first stripe it may use  */
+    int32_t *fan = (int32_t *)calloc((size_t)(U > 0 ? U : 1) * R, sizeof(int32_t));   /* F[stripe][d]: a stripe below the
+                                                                                 highest one in use is never empty, so U rows do */
     int32_t *core_of = (int32_t *)malloc((size_t)(U > 0 ? U : 1) * sizeof(int32_t));
+    int32_t *pos_of = (int32_t *)malloc((size_t)(U > 0 ? U : 1) * sizeof(int32_t));
     int32_t *stripe_of = (int32_t *)malloc((size_t)(U > 0 ? U : 1) * sizeof(int32_t));
     for (int32_t c = 0; c < n_cores; ++c) core_load[c] = 0;
     for (int64_t o = 0; o < U; ++o) {
         const int32_t j = order[o];
         const int32_t r = unit_desc[j * 4 + 0], d = unit_desc[j * 4 + 1];
         const int32_t cap = tiers[tier_of(r, d, g0, g1, n_tiers)].fanout_cap;
-        int32_t best = -1, best_any = 0;
-        for (int32_t c = 0; c < n_cores; ++c) {
-            if (core_load[c] < core_load[best_any]) best_any = c;
-            if (fan[(int64_t)len[c] * R + d] < cap && (best < 0 || core_load[c] < core_load[best])) best = c;
-        }
-        if (best < 0) best = best_any;
+        int32_t best = 0;
+        for (int32_t c = 1; c < n_cores; ++c)
+            if (core_load[c] < core_load[best]) best = c;
+        int32_t k = next[best];
+        while (fan[(int64_t)k * R + d] >= cap) ++k;
+        fan[(int64_t)k * R + d] += 1;
+        next[best] = k + 1;
         core_of[j] = best;
-        stripe_of[j] = len[best];
-        fan[(int64_t)len[best] * R + d] += 1;
+        pos_of[j] = len[best];
+        stripe_of[j] = k;
         len[best] += 1;
         core_load[best] += unit_cost[j];
     }
     /* per-core task lists in issue order */
     task_offset[0] = 0;
     for (int32_t c = 0; c < n_cores; ++c) task_offset[c + 1] = task_offset[c] + len[c];
-    for (int64_t j = 0; j < U; ++j) task_unit[task_offset[core_of[j]] + stripe_of[j]] = (int32_t)j;
+    for (int64_t j = 0; j < U; ++j) {
+        task_unit[task_offset[core_of[j]] + pos_of[j]] = (int32_t)j;
+        task_stripe[task_offset[core_of[j]] + pos_of[j]] = stripe_of[j];
+    }
+    free(next);
+    free(pos_of);
     free(order);
     free(len);
     free(fan);

@@ -39,15 +39,16 @@ def parse_golden():
             line = line.split("#")[0].strip()
             if not line:
                 continue
-            name, cores, cap, units, loads, opt = [s.strip() for s in line.split("|")]
+            name, cores, cap, units, loads, opt, stripes = [s.strip() for s in line.split("|")]
             us = [(int(u.split("@")[0]), int(u.split("@")[1])) for u in units.split()]
-            rows.append((name, int(cores), int(cap), us, [int(v) for v in loads.split()], int(opt)))
+            rows.append((name, int(cores), int(cap), us, [int(v) for v in loads.split()], int(opt),
+                         [[int(v) for v in core.split()] for core in stripes.split(";")]))
     return rows
 
 
 @pytest.mark.parametrize("case", parse_golden(), ids=lambda c: c[0])
 def test_hand_worked_schedules(case):
-    name, cores, cap, units, loads, opt = case
+    name, cores, cap, units, loads, opt, stripes = case
     R = 8
     lay = units_to_layout(units, R)
     # cost = rows exactly: alpha 0, beta = row_bytes, one unit per peer window
@@ -56,7 +57,9 @@ def test_hand_worked_schedules(case):
     assert part["unit_cost"].tolist() == [u[0] for u in units]
     assert part["unit_desc"][:, 1].tolist() == [u[1] for u in units]
     assert part["core_load"].tolist() == loads
-    assert max(loads) <= (4 / 3 - 1 / (3 * cores)) * opt + 1e-9 or cap < cores   # classical bound when uncapped
+    got = [part["task_stripe"][part["task_offset"][c]:part["task_offset"][c + 1]].tolist() for c in range(cores)]
+    assert got == stripes
+    assert max(loads) <= (4 / 3 - 1 / (3 * cores)) * opt + 1e-9      # the cap never costs makespan: classical bound
 
 
 def brute_force_optimum(costs, C):
@@ -87,15 +90,16 @@ def test_lpt_bound_against_brute_force_optimum(seed):
 
 
 def schedule_tables(part, R):
-    """(core, stripe) of every unit and the fan-out table F[stripe][dest] rebuilt from the task lists."""
+    """How often every unit is scheduled, and the fan-out table F[stripe][dest] rebuilt from the task lists and
+    their stripes; also checks that a core's stripes strictly increase (at most one unit per core and stripe)."""
     C = part["task_offset"].size - 1
     U = part["n_units"]
     seen = np.zeros(U, np.int32)
-    max_len = int(np.diff(part["task_offset"]).max()) if U else 0
-    F = np.zeros((max_len, R), np.int32)
+    F = np.zeros((int(part["task_stripe"].max()) + 1 if U else 0, R), np.int32)
     for c in range(C):
-        lst = part["task_unit"][part["task_offset"][c]:part["task_offset"][c + 1]]
-        for k, j in enumerate(lst):
+        lo, hi = part["task_offset"][c], part["task_offset"][c + 1]
+        assert np.all(np.diff(part["task_stripe"][lo:hi]) > 0)
+        for j, k in zip(part["task_unit"][lo:hi], part["task_stripe"][lo:hi]):
             seen[j] += 1
             F[k, part["unit_desc"][j, 1]] += 1
     return seen, F
@@ -145,11 +149,23 @@ def test_structure_on_a_routed_batch():
     for c in range(C):
         lst = part["task_unit"][part["task_offset"][c]:part["task_offset"][c + 1]]
         assert np.all(np.diff(part["unit_cost"][lst]) <= 0)
-    # balance: without a binding cap, list scheduling keeps every core within one largest unit of the lightest
+    # balance: list scheduling keeps every core within one largest unit of the lightest, and the cap changes
+    # no core's list (it only moves units to later stripes)
     free = oracle.partition(lay, row_bytes, C, [(a, b, s, 10 ** 6) for a, b, s, _ in tiers], g0=2, g1=4)
     assert free["core_load"].max() - free["core_load"].min() <= free["unit_cost"].max()
-    assert free["core_load"].sum() == part["core_load"].sum()
-    assert free["core_load"].max() <= part["core_load"].max()          # the cap can only cost makespan here
+    assert np.array_equal(free["core_load"], part["core_load"]) and np.array_equal(free["task_unit"], part["task_unit"])
+    assert np.array_equal(free["task_stripe"], np.concatenate([np.arange(n) for n in np.diff(free["task_offset"])]))
+    # the cap holds unit by unit: replayed in list-scheduling order (largest cost first, ties by id), a unit
+    # never enters a stripe that already holds H_t units for its destination, H_t the cap of the unit's tier
+    stripe_of = np.zeros(U, np.int64)
+    stripe_of[part["task_unit"]] = part["task_stripe"]
+    F2 = np.zeros((int(part["task_stripe"].max()) + 1, cfg.R), np.int32)
+    assert F2.shape == F.shape
+    for j in sorted(range(U), key=lambda u: (-int(part["unit_cost"][u]), u)):
+        r, d = part["unit_desc"][j, 0], part["unit_desc"][j, 1]
+        assert F2[stripe_of[j], d] < tiers[tier(r, d)][3]
+        F2[stripe_of[j], d] += 1
+    assert F.max() <= max(t[3] for t in tiers) and (part["task_stripe"] != free["task_stripe"]).any()
     # window-major dispatch writes exactly what token-major dispatch writes, every row once
     got = oracle.dispatch_windows(lay, part, inp["x"], cfg.K)
     assert np.array_equal(got, oracle.dispatch_bf16(lay["dst_row"], inp["x"]))
