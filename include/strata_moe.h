@@ -341,9 +341,12 @@ strata_status strata_moe_row_experts(strata_ctx *ctx, const strata_moe_layout_t 
  *                   tier(r,d) = 0 if r/g0 == d/g0, else 1 if r/g1 == d/g1, else 2 (clamped to n_tiers-1);
  *   unit cost       tau = alpha + ceil(bytes / beta), integers;
  *   policy          LPT-style list scheduling: units by decreasing cost (ties: lower unit id) onto the
- *                   least-loaded core (ties: lower core id) among the cores whose next issue stripe
- *                   (= number of units the core already holds) has fewer than fanout_cap units for the
- *                   unit's destination rank; if no core qualifies the cap is waived for that unit.
+ *                   least-loaded core (ties: lower core id), and on that core into the earliest issue
+ *                   stripe after the core's previous unit that holds fewer than fanout_cap units for the
+ *                   unit's destination rank.  Reading of Sec. 6.2 used: a core issues at most one unit per
+ *                   stripe and may leave a stripe empty, and stripes are not limited in number, so the cap
+ *                   F[stripe][dest] <= H_t is always met by a later stripe and never moves a unit to a
+ *                   busier core: the lists and loads are those of plain LPT, the cap shows in task_stripe.
  * Unit ids enumerate (r, d, k) in that order. */
 typedef struct {
     int64_t alpha;        /* fixed cost of a unit, 0 <= alpha < 2^30                      */
@@ -367,6 +370,8 @@ typedef struct {            /* all device pointers, caller-owned */
     int32_t *task_unit;     /* [max_units]      unit ids, core-major, in issue order                   */
     int64_t *core_load;     /* [n_cores]        predicted load of each core                            */
     int32_t *scratch;       /* [max_units*(R+2)] working memory of the policy kernel                   */
+    int32_t *task_stripe;   /* [max_units]      issue stripe of every entry of task_unit (strictly          */
+                            /*                  increasing inside a core's list)                            */
 } strata_partition_t;
 
 /* Upper bound of the unit count for a shape and policy (host arithmetic only):

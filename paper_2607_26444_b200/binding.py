@@ -83,7 +83,7 @@ class strata_partition_policy(ctypes.Structure):
 class strata_partition_t(ctypes.Structure):
     _fields_ = [("win_base", ctypes.c_void_p), ("unit_desc", ctypes.c_void_p), ("unit_cost", ctypes.c_void_p),
                 ("n_units", ctypes.c_void_p), ("task_offset", ctypes.c_void_p), ("task_unit", ctypes.c_void_p),
-                ("core_load", ctypes.c_void_p), ("scratch", ctypes.c_void_p)]
+                ("core_load", ctypes.c_void_p), ("scratch", ctypes.c_void_p), ("task_stripe", ctypes.c_void_p)]
 
 
 def make_policy(tiers, g0: int = 1, g1: int = 1) -> strata_partition_policy:
@@ -398,9 +398,10 @@ class Partition:
         self.task_unit = torch.zeros(max_units, **i32)
         self.core_load = torch.zeros(n_cores, **i64)
         self.scratch = torch.zeros(max_units * (R + 2), **i32)
+        self.task_stripe = torch.zeros(max_units, **i32)
         self.c = strata_partition_t(self.win_base.data_ptr(), self.unit_desc.data_ptr(), self.unit_cost.data_ptr(),
                                     self.n_units.data_ptr(), self.task_offset.data_ptr(), self.task_unit.data_ptr(),
-                                    self.core_load.data_ptr(), self.scratch.data_ptr())
+                                    self.core_load.data_ptr(), self.scratch.data_ptr(), self.task_stripe.data_ptr())
 
 
 class MoEContext:

@@ -565,6 +565,7 @@ strata_status strata_moe_partition(strata_ctx* ctx, const strata_moe_layout_t* l
 {
     if (!ctx || !layout || !out) return STRATA_ERR_INVALID_ARG;
     if (!layout->src_expert_count || !layout->expert_offset) return STRATA_ERR_INVALID_ARG;
+    if (!out->task_stripe) return STRATA_ERR_INVALID_ARG;
     if (!out->win_base || !out->unit_desc || !out->unit_cost || !out->n_units || !out->task_offset ||
         !out->task_unit || !out->core_load || !out->scratch)
         return STRATA_ERR_INVALID_ARG;

@@ -5,12 +5,16 @@
 //   level 3  peer-window partitioning: the expert windows of (source r -> destination rank d),
 //            concatenated in expert order, are cut into transfer units of at most S_t rows, t the tier
 //            of (r,d); cost tau = alpha_t + ceil(bytes / beta_t);
-//   policy   LPT-style list scheduling: units by decreasing cost onto the least-loaded core whose next
-//            issue stripe still has room for the unit's destination rank (fan-out cap H_t); the output
-//            is one task list per core, which the window-major dispatch kernel simply follows.
+//   policy   LPT-style list scheduling: units by decreasing cost onto the least-loaded core, and on that core
+//            into the earliest issue stripe after its previous unit that still has room for the unit's
+//            destination rank (fan-out cap H_t; a core issues at most one unit per stripe and may leave a
+//            stripe empty, so the cap moves a unit to a later stripe, never to a busier core); the output is
+//            one task list per core with the stripe of every entry.  The window-major dispatch kernel simply
+//            follows the lists (CTAs do not synchronise per stripe on one GPU).
 // The policy is generated ON the GPU by one CTA (no host round trip): a bitonic sort of the units and a
-// greedy loop run by one warp, whose "least-loaded feasible core" step is a warp-wide arg-min; where the
-// fan-out cap cannot bind, runs of equal-cost units are handed out in closed-form rounds.
+// greedy loop run by one warp, whose "least-loaded core" step is a warp-wide arg-min, with runs of
+// equal-cost units handed out in closed-form rounds; then, only when a cap can bind (H_t below the number
+// of cores), one sequential pass that gives every unit its stripe.
 #include "common.cuh"
 
 namespace strata {
@@ -32,8 +36,9 @@ struct PartitionParams {
     int32_t* n_units;                  // [1]
     int32_t* task_offset;              // [n_cores+1]
     int32_t* task_unit;                // [max_units]
+    int32_t* task_stripe;              // [max_units]
     long long* core_load;              // [n_cores]
-    int32_t* scratch;                  // [2*max_units + max_units*R]: core_of | stripe_of | fan-out overflow
+    int32_t* scratch;                  // [2*max_units + max_units*R]: core_of | pos_of | fan-out counts beyond shared memory
     int* status;
     int R, E, e_loc, n_cores, max_units, n_tiers, g0, g1;
     long long row_bytes;
@@ -151,7 +156,7 @@ __global__ void __launch_bounds__(kPartThreads) partition_kernel(PartitionParams
     }
     for (int x = tid; x < kFanSmemInts; x += kPartThreads) fan[x] = 0;
     int* core_of = p.scratch;
-    int* stripe_of = p.scratch + p.max_units;
+    int* pos_of = p.scratch + p.max_units;             // position of a unit in its core's list
     int* fan_global = p.scratch + 2 * p.max_units;     // stripes beyond shared memory
     const int smem_stripes = kFanSmemInts / R;
     for (int x = tid; x < U * R; x += kPartThreads) fan_global[x] = 0;
@@ -200,23 +205,20 @@ __global__ void __launch_bounds__(kPartThreads) partition_kernel(PartitionParams
     // ---- list scheduling: one warp, one unit per iteration; lane l speaks for cores l, l+32, ... ----
     // The loop is sequential in the units and a lone warp pays full ALU latency on every dependent
     // instruction, so the arithmetic is kept narrow: while every core's load fits 21 bits the key
-    // (infeasible | load | core) is one 32-bit word and the arg-min is one redux instruction; the
-    // first load that would not fit switches the rest of the run to 64-bit keys.
+    // (load | core) is one 32-bit word and the arg-min is one redux instruction; the first load that
+    // would not fit switches the rest of the run to 64-bit keys.
     if (wid == 0) {
-        // narrow state of a core: load (21 bits) << 11 | list length (11 bits); slots past the last core
-        // (the table is padded to a multiple of 128) hold all ones and can never win
+        // slots past the last core (the table is padded to a multiple of 128) hold all ones and can never win
         unsigned int* st32 = reinterpret_cast<unsigned int*>(scan);        // [kPartMaxCores] (scan[] is free here)
         const int padded = (p.n_cores + 127) / 128 * 128;
         for (int c = lane; c < padded; c += 32) st32[c] = c < p.n_cores ? 0u : 0xffffffffu;
         __syncwarp();
         int o = 0;
-        // A stripe holds at most one unit per core, so a cap of n_cores or more can never bind.  Then no
-        // fan-out table is consulted, a core's key changes only when the core wins, and every lane keeps
-        // its own cores' keys in registers (up to 384 cores; beyond, the lane minimum): a unit costs one min
-        // tree, one redux and the winner's update, about 0.2 us instead of 0.47 us per unit measured on B200.
-        bool cap_free = true;
-        for (int t = 0; t < p.n_tiers; ++t) cap_free = cap_free && p.cap[t] >= p.n_cores;
-        if (cap_free) {
+        // The core of a unit does not depend on the fan-out cap, so no fan-out table is consulted here: a
+        // core's key changes only when the core wins, and every lane keeps its own cores' keys in registers
+        // (up to 384 cores; beyond, the lane minimum): a unit costs one min tree, one redux and the winner's
+        // update, about 0.2 us per unit measured on B200.
+        {
             // here st32[c] is the key itself, load << 10 | core, and the list lengths live in len[]
             for (int c = lane; c < padded; c += 32) {
                 st32[c] = c < p.n_cores ? (unsigned)c : 0xffffffffu;
@@ -296,7 +298,7 @@ __global__ void __launch_bounds__(kPartThreads) partition_kernel(PartitionParams
                                     const int j = (int)((keys[o + rank] >> 2) & 0x1fffu);
                                     const int kk = len[core];
                                     core_of[j] = core;
-                                    stripe_of[j] = kk;
+                                    pos_of[j] = kk;
                                     len[core] = kk + 1;
                                     k[i] += cost << 10;
                                 }
@@ -316,7 +318,7 @@ __global__ void __launch_bounds__(kPartThreads) partition_kernel(PartitionParams
                             if (i == slot) k[i] = nk;
                         const int kk = len[win];
                         core_of[j] = win;
-                        stripe_of[j] = kk;
+                        pos_of[j] = kk;
                         len[win] = kk + 1;
                     }
                     ++o;
@@ -338,7 +340,7 @@ __global__ void __launch_bounds__(kPartThreads) partition_kernel(PartitionParams
                 if (lane == (win & 31)) {
                     const int kk = len[win];
                     core_of[j] = win;
-                    stripe_of[j] = kk;
+                    pos_of[j] = kk;
                     len[win] = kk + 1;
                     st32[win] = (new_load << 10) | (unsigned)win;
                     my_min = lane_min();
@@ -348,65 +350,16 @@ __global__ void __launch_bounds__(kPartThreads) partition_kernel(PartitionParams
             __syncwarp();
             for (int c = lane; c < p.n_cores; c += 32) load[c] = (long long)(st32[c] >> 10);
         }
-        for (; o < U && !cap_free; ++o) {
-            const unsigned long long m = keys[o];
-            const unsigned int cost = (unsigned int)min(m >> 27, (unsigned long long)0x7fffffffu);
-            const int d = (int)((m >> 15) & 0xfffu), j = (int)((m >> 2) & 0x1fffu);
-            const int cap = (m & 3u) == 0 ? p.cap[0] : (m & 3u) == 1 ? p.cap[1] : p.cap[2];
-            const int* fan_d = fan + d;
-            unsigned int best = 0xffffffffu;
-            for (int c0 = lane; c0 < padded; c0 += 128) {
-                unsigned int st[4];
-                int f[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) st[u] = st32[c0 + 32 * u];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) f[u] = fan_d[min((int)(st[u] & 2047u), smem_stripes - 1) * R];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    unsigned int key = ((st[u] >> 1) & 0x7ffffc00u) | (unsigned)(c0 + 32 * u);
-                    if (f[u] >= cap) key |= 0x80000000u;                        // infeasible cores sort last
-                    best = min(best, st[u] == 0xffffffffu ? 0xffffffffu : key);
-                }
-            }
-            best = __reduce_min_sync(0xffffffffu, best);
-            const int win = (int)(best & 1023u);    // if every core was infeasible this is the least loaded overall
-            const unsigned int sw = st32[win];
-            const unsigned int new_load = (sw >> 11) + cost, kk = sw & 2047u;
-            // leave the narrow mode before anything stops fitting: load in 21 bits, list length in 11
-            // bits and inside the shared-memory part of the fan-out table
-            if (new_load >= (1u << 21) || kk + 1 >= 2047u || (int)kk + 1 >= smem_stripes) break;
-            if (lane == (win & 31)) {
-                fan[kk * R + d] += 1;
-                core_of[j] = win;
-                stripe_of[j] = (int)kk;
-                st32[win] = (new_load << 11) | (kk + 1);
-            }
-            __syncwarp();
-        }
-        if (!cap_free)
-            for (int c = lane; c < p.n_cores; c += 32) {
-                len[c] = (int)(st32[c] & 2047u);
-                load[c] = (long long)(st32[c] >> 11);
-            }
-
         __syncwarp();
         const int cores_per_lane_w = (p.n_cores + 31) / 32;
         for (; o < U; ++o) {                        // wide keys: load << 10 | core in 64 bits (load < 2^53)
             const unsigned long long m = keys[o];
             const long long cost = (long long)(m >> 27);
-            const int d = (int)((m >> 15) & 0xfffu), j = (int)((m >> 2) & 0x1fffu);
-            const int cap = (m & 3u) == 0 ? p.cap[0] : (m & 3u) == 1 ? p.cap[1] : p.cap[2];
+            const int j = (int)((m >> 2) & 0x1fffu);
             unsigned long long best = ~0ull;
             for (int i = 0; i < cores_per_lane_w; ++i) {
                 const int c = lane + 32 * i;
-                if (c < p.n_cores) {
-                    const int kk = len[c];
-                    const int f = kk < smem_stripes ? fan[kk * R + d] : fan_global[(size_t)kk * R + d];
-                    unsigned long long key = ((unsigned long long)load[c] << 10) | (unsigned)c;
-                    if (f >= cap) key |= 1ull << 63;
-                    best = min(best, key);
-                }
+                if (c < p.n_cores) best = min(best, ((unsigned long long)load[c] << 10) | (unsigned)c);
             }
 #pragma unroll
             for (int dlt = 16; dlt > 0; dlt >>= 1) {
@@ -417,10 +370,8 @@ __global__ void __launch_bounds__(kPartThreads) partition_kernel(PartitionParams
             const int win = (int)(best & 1023u);
             if (lane == (win & 31)) {
                 const int kk = len[win];
-                if (kk < smem_stripes) fan[kk * R + d] += 1;
-                else fan_global[(size_t)kk * R + d] += 1;
                 core_of[j] = win;
-                stripe_of[j] = kk;
+                pos_of[j] = kk;
                 len[win] = kk + 1;
                 load[win] += cost;
             }
@@ -462,7 +413,51 @@ __global__ void __launch_bounds__(kPartThreads) partition_kernel(PartitionParams
             *p.n_units = U;
         }
         __syncthreads();
-        for (int j = tid; j < U; j += kPartThreads) p.task_unit[scan[34 + core_of[j]] + stripe_of[j]] = j;
+        for (int j = tid; j < U; j += kPartThreads) p.task_unit[scan[34 + core_of[j]] + pos_of[j]] = j;
+    }
+
+    // ---- issue stripes ----
+    // A stripe holds at most one unit per core, so a cap of n_cores or more can never bind: the stripe of a
+    // unit is then its position in the list.
+    bool cap_binds = false;
+    for (int t = 0; t < p.n_tiers; ++t) cap_binds = cap_binds || p.cap[t] < p.n_cores;
+    if (!cap_binds) {
+        for (int j = tid; j < U; j += kPartThreads) p.task_stripe[scan[34 + core_of[j]] + pos_of[j]] = pos_of[j];
+        return;
+    }
+    // Otherwise the stripes follow from one pass over the units in list-scheduling order (keys[] still holds
+    // it): a unit takes the earliest stripe at or after its core's next free one in which fewer than H_t units
+    // target its destination.  The walk is sequential (F[stripe][d] and the cores' next stripes evolve with
+    // every unit), so one lane does it; the other lanes fetch the next 32 units' cores and list slots.  A
+    // stripe below the highest one in use is never empty, so no stripe index reaches U.
+    __syncthreads();
+    if (wid != 0) return;
+    for (int c = lane; c < p.n_cores; c += 32) len[c] = 0;     // from here on: the first stripe the core may use
+    __syncwarp();
+    for (int o0 = 0; o0 < U; o0 += 32) {
+        const int o = o0 + lane;
+        const unsigned long long m = o < U ? keys[o] : 0ull;
+        const int j = (int)((m >> 2) & 0x1fffu);
+        const int my_d = (int)((m >> 15) & 0xfffu);
+        const int my_cap = (m & 3u) == 0 ? p.cap[0] : (m & 3u) == 1 ? p.cap[1] : p.cap[2];
+        const int my_core = o < U ? core_of[j] : 0;
+        const int my_slot = o < U ? scan[34 + my_core] + pos_of[j] : 0;
+        const int n = min(32, U - o0);
+        for (int i = 0; i < n; ++i) {
+            const int core = __shfl_sync(0xffffffffu, my_core, i), d = __shfl_sync(0xffffffffu, my_d, i);
+            const int cap = __shfl_sync(0xffffffffu, my_cap, i), slot = __shfl_sync(0xffffffffu, my_slot, i);
+            if (lane == 0) {
+                int k = len[core];
+                for (;; ++k) {
+                    const int f = k < smem_stripes ? fan[k * R + d] : fan_global[(size_t)k * R + d];
+                    if (f < cap) break;
+                }
+                if (k < smem_stripes) fan[k * R + d] += 1;
+                else fan_global[(size_t)k * R + d] += 1;
+                len[core] = k + 1;
+                p.task_stripe[slot] = k;
+            }
+        }
     }
 }
 
@@ -645,6 +640,7 @@ cudaError_t launch_partition(const strata_moe_shape& s, const strata_moe_layout_
     p.n_units = out.n_units;
     p.task_offset = out.task_offset;
     p.task_unit = out.task_unit;
+    p.task_stripe = out.task_stripe;
     p.core_load = reinterpret_cast<long long*>(out.core_load);
     p.scratch = out.scratch;
     p.status = status;

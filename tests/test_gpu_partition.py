@@ -62,6 +62,7 @@ def test_policy_and_window_dispatch_match_the_oracle(case):
     assert np.array_equal(part.unit_cost.cpu().numpy()[:U], ref["unit_cost"])
     assert np.array_equal(part.task_offset.cpu().numpy(), ref["task_offset"])
     assert np.array_equal(part.task_unit.cpu().numpy()[:U], ref["task_unit"])
+    assert np.array_equal(part.task_stripe.cpu().numpy()[:U], ref["task_stripe"])
     assert np.array_equal(part.core_load.cpu().numpy(), ref["core_load"])
 
     # window-major dispatch, with guard rows
