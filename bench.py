@@ -441,6 +441,57 @@ def window_partitioning_report(cfg: wl.MoEConfig, dev_index: int, unit_rows: int
     return out
 
 
+def expert_chain_report(cfg: wl.MoEConfig, dev_index: int, tile_rows: int = 128, iters: int = 30):
+    """layout -> dispatch -> in-place expert stand-in -> combine with segments aligned to tile_rows, all on the
+    device: microseconds per call (30 calls between one pair of events) and the stand-in's effective GB/s
+    (every occupied row read once and written once)."""
+    import torch
+    from paper_2607_26444_b200 import binding as B
+    dev = torch.device("cuda", dev_index)
+    inp = wl.generate(cfg) if cfg.n_tok <= 20000 else None
+    ctx = B.MoEContext(cfg.R, cfg.T, cfg.H, cfg.E, cfg.K, device=dev_index, segment_align=tile_rows)
+    ctx.x_early(True)
+    ids = torch.from_numpy(inp["ids"] if inp else wl.gen_topk_ids(cfg)).to(dev)
+    x = (torch.from_numpy(inp["x"].view(np.int16)).to(dev) if inp
+         else torch.randint(-30000, 30000, (cfg.n_tok, cfg.H), dtype=torch.int16, device=dev))
+    w = torch.from_numpy(inp["w"] if inp else wl.gen_gate_weights(cfg)).to(dev)
+    scale = (1.0 + torch.arange(cfg.E, dtype=torch.float32, device=dev) / cfg.E)
+    bias = 0.01 * torch.arange(cfg.E, dtype=torch.float32, device=dev)
+    recv = torch.zeros((ctx.recv_rows, cfg.H), dtype=torch.int16, device=dev)
+    ctx.register(recv)
+    out = torch.empty((cfg.n_tok, cfg.H), dtype=torch.int16, device=dev)
+    lay = ctx.new_layout(with_optional=False)
+    calls = {
+        "layout": lambda: ctx.layout(ids, lay),
+        "dispatch": lambda: ctx.dispatch(lay, x, recv),
+        "expert": lambda: ctx.expert_affine_inplace(lay, recv, scale, bias, tile_rows),
+        "combine": lambda: ctx.combine(lay, recv, w, out),
+    }
+
+    def chain():
+        for fn in calls.values():
+            fn()
+    calls["chain"] = chain
+    chain()
+    rep = {"workload": cfg.name, "tile_rows": tile_rows, "recv_rows": int(ctx.recv_rows), "us": {}}
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for name, fn in calls.items():
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        torch.cuda._sleep(10_000_000)
+        a.record()
+        for _ in range(iters):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        rep["us"][name] = round(a.elapsed_time(b) * 1e3 / iters, 2)
+    rep["expert_GBs"] = round(2 * cfg.n_items * cfg.H * 2 / rep["us"]["expert"] / 1e3, 1)
+    rep["device_status"] = ctx.device_status()
+    ctx.close()
+    return rep
+
+
 def timeline_report(cfg: wl.MoEConfig, dev_index: int, trace_path: str = "", pinned: bool = False):
     """One step with the in-kernel event timeline on (paper Sec. 6.4): per kernel the CTA count, wall time,
     finish-time spread and the share of CTA time per stage.  Probes cost time: these are not bench numbers."""
@@ -934,6 +985,8 @@ def main():
                     help="print only the interference report: dispatch+combine beside a library GEMM on another stream")
     ap.add_argument("--collectives", action="store_true",
                     help="print only the report on the full-mesh collectives (one JSON object; not the bench line)")
+    ap.add_argument("--expert-chain", action="store_true",
+                    help="print only the timings of layout -> dispatch -> in-place expert stand-in -> combine for --workload")
     ap.add_argument("--partition-report", action="store_true",
                     help="print only the report on the paper's window partitioning at the skew and prefill shapes")
     ap.add_argument("--collective-kib", type=int, nargs="+", default=[64, 1024, 16384], help="payload per rank, KiB")
@@ -969,6 +1022,10 @@ def main():
     if args.overlap:
         if rank == 0:
             print(json.dumps(overlap_report(wl.CONFIGS[args.workload], local_rank)), flush=True)
+        return
+    if args.expert_chain:
+        if rank == 0:
+            print(json.dumps(expert_chain_report(wl.CONFIGS[args.workload], local_rank)), flush=True)
         return
     if args.partition_report:
         if rank == 0:

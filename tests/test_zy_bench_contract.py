@@ -86,3 +86,11 @@ def test_timeline_report_mode(tmp_path):
     assert d["events_dropped"] == 0 and {"dispatch_bf16", "combine"} <= set(d["kernels"])
     assert d["kernels"]["dispatch_bf16"]["stages"]["work"]["intervals"] == 4 * 128       # one per token
     assert d["chrome_trace_events"] > 0 and json.loads(trace.read_text())["traceEvents"]
+
+
+@pytest.mark.gpu
+def test_expert_chain_report_mode():
+    d = run_bench("--expert-chain", "--workload", "decode")
+    assert d["device_status"] == 0 and d["tile_rows"] == 128 and d["recv_rows"] == 16384 + 256 * 127
+    assert set(d["us"]) == {"layout", "dispatch", "expert", "combine", "chain"} and all(v > 0 for v in d["us"].values())
+    assert d["expert_GBs"] > 1000
