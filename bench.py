@@ -468,8 +468,10 @@ def expert_chain_report(cfg: wl.MoEConfig, dev_index: int, tile_rows: int = 128,
         "combine": lambda: ctx.combine(lay, recv, w, out),
     }
 
+    parts = list(calls.values())
+
     def chain():
-        for fn in calls.values():
+        for fn in parts:
             fn()
     calls["chain"] = chain
     chain()
@@ -502,7 +504,7 @@ def timeline_report(cfg: wl.MoEConfig, dev_index: int, trace_path: str = "", pin
         case.step()
     torch.cuda.synchronize()
     units = cfg.n_tok * max(1, -(-cfg.H * 2 // 16384))
-    cap = 16 + 8 * (units // (2 * 148) + 64)                 # 6 events per dispatch unit, with room to spare
+    cap = 16 + 8 * (units // 148 + 64)                       # 6 events per dispatch unit (one CTA per SM at least), with room to spare
     t = case.ctx.timeline(n_ctas=2048, events_per_cta=cap, pinned=pinned)
     case.step()
     spans, dropped = case.ctx.timeline_spans(t)
