@@ -27,6 +27,9 @@ namespace {
 #ifndef STRATA_COMBINE_UNITS_PER_CTA
 #define STRATA_COMBINE_UNITS_PER_CTA 24      // rows are split into column parts until a CTA can expect this many units
 #endif
+#ifndef STRATA_COMBINE_LOAD_HINT
+#define STRATA_COMBINE_LOAD_HINT 0           // 1: the row loads carry an L2 evict-first policy (measured: no effect at any shape)
+#endif
 constexpr int kCombineThreads = STRATA_COMBINE_THREADS;
 
 struct CombineParams {
@@ -73,6 +76,9 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
     const size_t row_bytes = (size_t)p.H * 2u;
     const unsigned int n_units = (unsigned int)(p.n_tok * p.parts);
     __shared__ unsigned int s_next[2];             // the claim made during unit j is read for unit j+1
+#if STRATA_COMBINE_LOAD_HINT
+    const uint64_t pol = policy_evict_first();
+#endif
     griddep_wait();
     if (tid == 0) trace_begin(p.trace);
     Timeline tl(p.trace, STRATA_KERNEL_COMBINE, tid == 0);
@@ -105,7 +111,11 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
             uint4 d[K];
 #pragma unroll
             for (int k = 0; k < K; ++k)
+#if STRATA_COMBINE_LOAD_HINT
+                d[k] = src[k] ? ld_stream16_hint(src[k] + (size_t)v * 16, pol) : make_uint4(0, 0, 0, 0);
+#else
                 d[k] = src[k] ? ld_stream16(src[k] + (size_t)v * 16) : make_uint4(0, 0, 0, 0);
+#endif
             float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int k = 0; k < K; ++k)

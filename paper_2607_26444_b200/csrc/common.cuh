@@ -403,6 +403,15 @@ __device__ __forceinline__ uint4 ld_stream16(const void* p)
                  : "l"(p));
     return v;
 }
+// the same load with an L2 eviction policy (see policy_evict_first)
+__device__ __forceinline__ uint4 ld_stream16_hint(const void* p, uint64_t policy)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p), "l"(policy));
+    return v;
+}
 __device__ __forceinline__ void st_stream16(void* p, uint4 v)
 {
     asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)

@@ -55,15 +55,18 @@ std::atomic<int> g_inject_short_copy{0};
 #ifndef STRATA_BF16_CHUNK_BYTES
 #define STRATA_BF16_CHUNK_BYTES 16384
 #endif
-#ifndef STRATA_BF16_STORE_HINT
-#define STRATA_BF16_STORE_HINT 0               // 1: L2 evict-first policy on the bulk stores
-#endif
 constexpr uint32_t kMaxChunkBytes = STRATA_BF16_CHUNK_BYTES;   // one stage of the bf16 ring
 constexpr int kBf16Stages = STRATA_BF16_STAGES;
 constexpr size_t kBf16MaxSmem = 200 * 1024;  // ring + barriers of one CTA never exceed this
 constexpr uint32_t kDeepRingMinBytes = 12 * 1024;     // chunks at least this long take the one-CTA-per-SM shape
 constexpr size_t kDeepRingBytes = 128 * 1024;         // its ring: as many stages as fit here, at most
 constexpr int kDeepRingMaxStages = 8;                 // this many
+// Receive buffers far larger than L2 (126 MB) are written with an L2 evict-first policy: the kernel itself runs
+// the same, but the kernel that reads the buffer next does not start on an L2 full of normal-priority dirty
+// lines.  Measured: combine right after dispatch 1,270 -> 1,228 us at the prefill shape (7.5 GB); at the skew
+// shape (1.1 GB) neutral; at the decode shape (235 MB) combine loses 3 us, because half of what it reads would
+// still have been in L2.
+constexpr long long kStoreHintMinBytes = 2ll << 30;
 // 64..256 threads and 2048..4096-column chunks land within 1.5 % of each other (110..113 us at the fp8 shape);
 // 1024-column chunks are 25 % slower.
 constexpr int kFp8Threads = 128;
@@ -83,6 +86,7 @@ struct DispatchParams {
     int stages;                 // bf16 only: depth of the ring in shared memory
     int test_flags;             // always 0 in the shipped library
     int x_early;                // the first loads of x may go out before the preceding kernel has finished
+    int store_hint;             // bf16 only: the bulk stores carry an L2 evict-first policy
     int* status;
     WorkQueue wq;
     TraceBuf trace;
@@ -197,12 +201,11 @@ __global__ void __launch_bounds__(32) dispatch_bf16_kernel(DispatchParams p)
         for (int k = 0; k < p.K; ++k) {
             const int row = __shfl_sync(0xffffffffu, my_row, k);
             if (lane == 0 && row >= 0 && row < p.capacity_rows) {
-#if STRATA_BF16_STORE_HINT
-                bulk_s2g_hint(p.recv + (size_t)row * row_bytes + (size_t)col0 * 2u, smem + (size_t)s * stage_bytes,
-                              bytes, pol);
-#else
-                bulk_s2g(p.recv + (size_t)row * row_bytes + (size_t)col0 * 2u, smem + (size_t)s * stage_bytes, bytes);
-#endif
+                if (p.store_hint)
+                    bulk_s2g_hint(p.recv + (size_t)row * row_bytes + (size_t)col0 * 2u, smem + (size_t)s * stage_bytes,
+                                  bytes, pol);
+                else
+                    bulk_s2g(p.recv + (size_t)row * row_bytes + (size_t)col0 * 2u, smem + (size_t)s * stage_bytes, bytes);
             }
         }
         if (lane == 0) {
@@ -501,6 +504,7 @@ cudaError_t launch_dispatch_bf16(const strata_moe_shape& s, const int32_t* dst_r
     cudaError_t err = smem_for_residency(dispatch_bf16_kernel, 32, need, want_per_sm, kBf16MaxSmem, &smem, &per_sm);
     if (err != cudaSuccess) return err;
     p.n_units = (long long)s.R * s.T * p.chunks_per_row;
+    p.store_hint = (long long)s.R * s.T * s.K * s.H * 2 >= (tune("STRATA_DISP_STORE_HINT_MB", kStoreHintMinBytes >> 20) << 20);
 #ifdef STRATA_TEST_HOOKS
     p.test_flags = g_inject_short_copy.exchange(0);
 #endif
