@@ -58,7 +58,10 @@ std::atomic<int> g_inject_short_copy{0};
 constexpr uint32_t kMaxChunkBytes = STRATA_BF16_CHUNK_BYTES;   // one stage of the bf16 ring
 constexpr int kBf16Stages = STRATA_BF16_STAGES;
 constexpr size_t kBf16MaxSmem = 200 * 1024;  // ring + barriers of one CTA never exceed this
-constexpr uint32_t kDeepRingMinBytes = 12 * 1024;     // chunks at least this long take the one-CTA-per-SM shape
+constexpr long long kDeepRingMinUnitBytes = 100 * 1024;   // units (1 + K chunks) at least this long take the one-CTA-per-SM shape
+constexpr long long kUnitBytesInFlightPerSm = 144 * 1024; // what the short-ring CTAs of an SM should have in flight together
+constexpr size_t kShortRingsBytesPerSm = 192 * 1024;      // shared memory their rings may take together
+constexpr int kMaxCtasPerSm = 24;
 constexpr size_t kDeepRingBytes = 128 * 1024;         // its ring: as many stages as fit here, at most
 constexpr int kDeepRingMaxStages = 8;                 // this many
 // Receive buffers far larger than L2 (126 MB) are written with an L2 evict-first policy: the kernel itself runs
@@ -491,11 +494,18 @@ cudaError_t launch_dispatch_bf16(const strata_moe_shape& s, const int32_t* dst_r
     p.chunks_per_row = (int)(((uint32_t)s.H + p.chunk_cols - 1) / p.chunk_cols);
     p.capacity_rows = (long long)capacity_rows;
     p.status = status;
-    // Long chunks: one CTA per SM with a deep ring (its single issuing lane keeps up: a unit every ~3 us).
-    // Short chunks need two issuing lanes per SM to keep the copy engine fed, so two CTAs with a short ring.
+    // A unit (one chunk read, K chunk writes) occupies its issuing lane for about 2.5 us whatever its size
+    // (destination rows, claim and stage hand-over are round trips to memory), so an SM needs enough lanes
+    // working side by side to move its share of the bandwidth: about 144 KB of units in flight per SM.  Units of
+    // 100 KB and more (14 KB rows with top-8) get one CTA per SM with a deep ring; smaller units get
+    // ceil(144 KB / unit) CTAs per SM with a short ring each (measured at 16,384 tokens, top-8: 2 KB rows 2.3 ->
+    // 6.1 TB/s with 8 CTAs per SM, 4 KB rows 4.3 -> 6.4 TB/s with 4; top-2, 4 KB rows 2.1 -> 6.1 TB/s with 12).
     const uint32_t stage_bytes = p.chunk_cols * 2u;
-    const bool deep = stage_bytes >= kDeepRingMinBytes;
-    int want_per_sm = (int)tune("STRATA_DISP_CTAS", deep ? 1 : 2);
+    const long long unit_bytes = (long long)(s.K + 1) * stage_bytes;
+    const bool deep = unit_bytes >= kDeepRingMinUnitBytes;
+    int lanes = (int)((kUnitBytesInFlightPerSm + unit_bytes - 1) / unit_bytes);
+    lanes = max(2, min(kMaxCtasPerSm, min(lanes, (int)(kShortRingsBytesPerSm / ((size_t)kBf16Stages * stage_bytes)))));
+    int want_per_sm = (int)tune("STRATA_DISP_CTAS", deep ? 1 : lanes);
     p.stages = (int)tune("STRATA_DISP_STAGES", deep ? min(kDeepRingMaxStages, (int)(kDeepRingBytes / stage_bytes)) : kBf16Stages);
     while (p.stages > 2 && (size_t)p.stages * (stage_bytes + 12) + 16 > kBf16MaxSmem) --p.stages;
     const size_t need = (size_t)p.stages * stage_bytes + 12 * (size_t)p.stages + 16;   // stages | mbarriers | unit ids
