@@ -15,6 +15,8 @@
 //       the per-128-column amax, scale = amax/448 and the e4m3 codes into an output stage,
 //       and K bulk stores ship the codes; the scales (H/128 floats per row) go out with plain
 //       coalesced stores.
+#include <mutex>
+
 #include "common.cuh"
 
 #ifdef STRATA_TEST_HOOKS
@@ -38,8 +40,8 @@ std::atomic<int> g_inject_short_copy{0};
 //  - 14 KB rows (decode and prefill shapes): one CTA per SM with an 8-stage ring beats two CTAs per SM with
 //    3 stages (decode 40.9 vs 42.7 us; prefill 1281 vs 1288 us).  Rings of 10 and 12 stages copy as fast
 //    alone but make the layout+dispatch+combine step at the prefill shape 0.5 % and 1.5 % slower.
-//  - 8 KB rows (skew shape): one issuing lane per SM cannot keep the copy engine fed (257 vs 183 us), so
-//    short chunks take two CTAs per SM.
+//  - 8 KB rows (skew shape): one issuing lane per SM cannot keep the copy engine fed (257 vs 183 us); the
+//    number of CTAs per SM follows the unit size (see launch_dispatch_bf16).
 //  - Cutting the last units of the batch into halves or quarters evens out the CTAs' finish times (8 us
 //    apart to 2 us apart at the decode shape) but does not shorten the kernel: the CTAs that are still
 //    running get the bandwidth of those that have left.  Pieces below 4 KB copy markedly slower.
@@ -431,6 +433,18 @@ __global__ void __launch_bounds__(kFp8Threads) dispatch_fp8_kernel(DispatchParam
 // holds part of some SMs; if more than `want` fitted on an SM, the free SMs would take several CTAs and
 // others none, and the kernel would run with a lopsided placement for its whole life (measured: 20 %
 // slower at the prefill shape).  Asking for more shared memory than needed makes the surplus CTA not fit.
+// The answer depends only on (device, kernel, threads, need, want), and a context asks the same question on
+// every call: the last few answers are kept, so a call costs a lock instead of four runtime queries.
+struct ResidencyAnswer {
+    const void* kernel;
+    int dev, threads, want;
+    size_t need, max_smem, smem;
+    int per_sm;
+};
+std::mutex g_residency_mu;
+ResidencyAnswer g_residency[8];
+int g_residency_n = 0, g_residency_next = 0;
+
 template <typename Kernel>
 cudaError_t smem_for_residency(Kernel kernel, int threads, size_t need, int want, size_t max_smem, size_t* smem_out,
                                int* per_sm_out)
@@ -438,6 +452,19 @@ cudaError_t smem_for_residency(Kernel kernel, int threads, size_t need, int want
     int dev = 0, sm_total = 0, reserved = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
+    const void* kptr = reinterpret_cast<const void*>(kernel);
+    {
+        std::lock_guard<std::mutex> lk(g_residency_mu);
+        for (int i = 0; i < g_residency_n; ++i) {
+            const ResidencyAnswer& a = g_residency[i];
+            if (a.kernel == kptr && a.dev == dev && a.threads == threads && a.want == want && a.need == need &&
+                a.max_smem == max_smem) {
+                *smem_out = a.smem;
+                *per_sm_out = a.per_sm;
+                return cudaSuccess;
+            }
+        }
+    }
     err = cudaDeviceGetAttribute(&sm_total, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
     if (err != cudaSuccess) return err;
     err = cudaDeviceGetAttribute(&reserved, cudaDevAttrReservedSharedMemoryPerBlock, dev);
@@ -453,6 +480,12 @@ cudaError_t smem_for_residency(Kernel kernel, int threads, size_t need, int want
     if (err != cudaSuccess) return err;
     *smem_out = smem;
     *per_sm_out = max(1, min(per_sm, want));
+    {
+        std::lock_guard<std::mutex> lk(g_residency_mu);
+        g_residency[g_residency_next] = ResidencyAnswer{kptr, dev, threads, want, need, max_smem, *smem_out, *per_sm_out};
+        g_residency_next = (g_residency_next + 1) % 8;
+        if (g_residency_n < 8) ++g_residency_n;
+    }
     return cudaSuccess;
 }
 
