@@ -69,27 +69,35 @@ __global__ void __launch_bounds__(kExpertThreads) expert_affine_kernel(ExpertPar
     const float sc = p.scale[s_expert], bi = p.bias[s_expert];
     const int vpr = p.H / 8;              // 16-byte vectors per row
     const int v0 = part * p.vec_per_part, nv = min(p.vec_per_part, vpr - v0);
-    const long long total = (long long)rows * nv;
-    unsigned char* base = p.recv + (size_t)row0 * (size_t)p.H * 2u;
-    for (long long i0 = threadIdx.x; i0 < total; i0 += (long long)kExpertThreads * kExpertVecPerThread) {
-        uint4 d[kExpertVecPerThread];
-        unsigned char* addr[kExpertVecPerThread];
+    const size_t row_bytes = (size_t)p.H * 2u;
+    unsigned char* base = p.recv + (size_t)row0 * row_bytes + (size_t)v0 * 16u;
+    // Threads form 256 / tpr groups of tpr threads (tpr a power of two, at most the vectors of a row part): a
+    // group takes every (256 / tpr)-th row, a thread of it every tpr-th vector of the row.  Lanes of a warp read
+    // consecutive vectors, and no index needs a division.
+    int tpr_log2 = 0;
+    while ((2 << tpr_log2) <= min(nv, kExpertThreads)) ++tpr_log2;
+    const int tpr = 1 << tpr_log2, groups = kExpertThreads >> tpr_log2;
+    const int my_v = (int)threadIdx.x & (tpr - 1), my_g = (int)threadIdx.x >> tpr_log2;
+    for (int v = my_v; v < nv; v += tpr) {
+        unsigned char* col = base + (size_t)v * 16u;
+        for (int r0 = my_g; r0 < rows; r0 += groups * kExpertVecPerThread) {
+            uint4 d[kExpertVecPerThread];
 #pragma unroll
-        for (int q = 0; q < kExpertVecPerThread; ++q) {
-            const long long i = i0 + (long long)q * kExpertThreads;
-            const int r = (int)(i / nv), v = (int)(i - (long long)r * nv);
-            addr[q] = i < total ? base + ((size_t)r * vpr + (size_t)(v0 + v)) * 16u : nullptr;
-            if (addr[q]) d[q] = *reinterpret_cast<const uint4*>(addr[q]);
-        }
+            for (int q = 0; q < kExpertVecPerThread; ++q) {
+                const int r = r0 + q * groups;
+                if (r < rows) d[q] = *reinterpret_cast<const uint4*>(col + (size_t)r * row_bytes);
+            }
 #pragma unroll
-        for (int q = 0; q < kExpertVecPerThread; ++q) {
-            if (!addr[q]) continue;
-            uint4 o;
-            o.x = affine_pack(d[q].x, sc, bi);
-            o.y = affine_pack(d[q].y, sc, bi);
-            o.z = affine_pack(d[q].z, sc, bi);
-            o.w = affine_pack(d[q].w, sc, bi);
-            *reinterpret_cast<uint4*>(addr[q]) = o;
+            for (int q = 0; q < kExpertVecPerThread; ++q) {
+                const int r = r0 + q * groups;
+                if (r >= rows) continue;
+                uint4 o;
+                o.x = affine_pack(d[q].x, sc, bi);
+                o.y = affine_pack(d[q].y, sc, bi);
+                o.z = affine_pack(d[q].z, sc, bi);
+                o.w = affine_pack(d[q].w, sc, bi);
+                *reinterpret_cast<uint4*>(col + (size_t)r * row_bytes) = o;
+            }
         }
     }
 }
