@@ -1,6 +1,7 @@
 /* The C ABI used from plain C: no Python, no torch.  Runs the hand-worked routing example
  * (R=2 T=2 K=2 E=4; ids r0t0=[2,0] r0t1=[0,3] r1t0=[0,2] r1t1=[3,2]) through layout, dispatch and
- * combine with identity experts, plus a 2-rank all-reduce, and checks the results.
+ * combine with identity experts, a 2-rank all-reduce, and a second step with the early-x promise and the
+ * in-place expert stand-in, and checks the results.
  * Build: gcc c_abi_demo.c -I<include> -I<cuda>/include <libstrata_moe.so> -L<cuda>/lib64 -lcudart */
 #include <cuda_runtime_api.h>
 #include <stdint.h>
@@ -99,8 +100,30 @@ int main(void)
         const uint16_t s = bf16_of_small_int(16 + c + 32 + c);
         CHECK(out[c] == s && out[H + c] == s);
     }
+    /* a second step with dispatch allowed to read x while the layout still runs, and the in-place expert stand-in
+     * doubling every occupied row (x holds small integers, so 2x is exact in bf16): out = 2 x */
+    float two[E], zero[E];
+    for (int e = 0; e < E; ++e) { two[e] = 2.0f; zero[e] = 0.0f; }
+    void *d_scale, *d_bias;
+    CHECK(cudaMalloc(&d_scale, sizeof two) == cudaSuccess && cudaMalloc(&d_bias, sizeof zero) == cudaSuccess);
+    CHECK(cudaMemcpy(d_scale, two, sizeof two, cudaMemcpyHostToDevice) == cudaSuccess);
+    CHECK(cudaMemcpy(d_bias, zero, sizeof zero, cudaMemcpyHostToDevice) == cudaSuccess);
+    CHECK(strata_ctx_set_x_early(ctx, 1) == STRATA_OK);
+    CHECK(strata_moe_layout(ctx, (const int32_t *)d_ids, &lay, NULL) == STRATA_OK);
+    CHECK(strata_moe_dispatch(ctx, &lay, d_x, d_recv, NULL, N, NULL) == STRATA_OK);
+    CHECK(strata_moe_expert_affine_inplace(ctx, &lay, d_recv, N, (const float *)d_scale, (const float *)d_bias, 2, NULL)
+          == STRATA_ERR_SHAPE);                      /* packed segments: a tile is one row */
+    CHECK(strata_moe_expert_affine_inplace(ctx, &lay, d_recv, N, (const float *)d_scale, (const float *)d_bias, 1, NULL)
+          == STRATA_OK);
+    CHECK(strata_moe_combine(ctx, &lay, d_recv, N, (const float *)d_w, d_out, NULL) == STRATA_OK);
+    CHECK(strata_device_status(ctx, NULL, &dev) == STRATA_OK && dev == STRATA_OK);
+    CHECK(cudaMemcpy(out, d_out, sizeof out, cudaMemcpyDeviceToHost) == cudaSuccess);
+    for (int n = 0; n < NTOK; ++n)
+        for (int c = 0; c < H; ++c) CHECK(out[n * H + c] == bf16_of_small_int(2 * (16 * (n + 1) + c)));
+    cudaFree(d_scale); cudaFree(d_bias);
+
     uint64_t launches = 0;
-    CHECK(strata_ctx_launch_count(ctx, &launches) == STRATA_OK && launches == 4);
+    CHECK(strata_ctx_launch_count(ctx, &launches) == STRATA_OK && launches == 8);
     CHECK(strata_ctx_destroy(ctx) == STRATA_OK);
     cudaFree(ws); cudaFree(d_ids); cudaFree(d_x); cudaFree(d_w); cudaFree(d_recv); cudaFree(d_out); cudaFree(d_meta);
     printf("PASS %s\n", strata_status_string(STRATA_OK));
