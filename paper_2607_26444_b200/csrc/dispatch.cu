@@ -60,7 +60,10 @@ std::atomic<int> g_inject_short_copy{0};
 constexpr uint32_t kMaxChunkBytes = STRATA_BF16_CHUNK_BYTES;   // one stage of the bf16 ring
 constexpr int kBf16Stages = STRATA_BF16_STAGES;
 constexpr size_t kBf16MaxSmem = 200 * 1024;  // ring + barriers of one CTA never exceed this
-constexpr long long kDeepRingMinUnitBytes = 100 * 1024;   // units (1 + K chunks) at least this long take the one-CTA-per-SM shape
+constexpr long long kDeepRingMinUnitBytes = 100 * 1024;   // units (1 + K chunks) at least this long, made of chunks of at
+constexpr uint32_t kDeepRingMinChunkBytes = 12 * 1024;    // least this size, take the one-CTA-per-SM shape (8 KB rows with
+                                                          // top-12 make a 106 KB unit but 13 copies per unit: one lane
+                                                          // per SM reached 5.2 TB/s there, two reach 6.5)
 constexpr long long kUnitBytesInFlightPerSm = 144 * 1024; // what the short-ring CTAs of an SM should have in flight together
 constexpr size_t kShortRingsBytesPerSm = 192 * 1024;      // shared memory their rings may take together
 constexpr int kMaxCtasPerSm = 24;
@@ -73,7 +76,9 @@ constexpr int kDeepRingMaxStages = 8;                 // this many
 // still have been in L2.
 constexpr long long kStoreHintMinBytes = 2ll << 30;
 // 64..256 threads and 2048..4096-column chunks land within 1.5 % of each other (110..113 us at the fp8 shape);
-// 1024-column chunks are 25 % slower.
+// 1024-column chunks are 25 % slower.  Requesting the work claim one unit early (so that the CTA does not sit
+// between two barriers during the atomic's round trip) helps small units a little (top-2: 4.2 -> 4.3 TB/s) and
+// costs 2 % at the fp8 shape and with 7,168 columns: not taken, as in the bf16 kernel.
 constexpr int kFp8Threads = 128;
 constexpr int kFp8MaxChunkCols = 4096;       // 8 KB in, 4 KB out per stage
 
@@ -535,7 +540,7 @@ cudaError_t launch_dispatch_bf16(const strata_moe_shape& s, const int32_t* dst_r
     // 6.1 TB/s with 8 CTAs per SM, 4 KB rows 4.3 -> 6.4 TB/s with 4; top-2, 4 KB rows 2.1 -> 6.1 TB/s with 12).
     const uint32_t stage_bytes = p.chunk_cols * 2u;
     const long long unit_bytes = (long long)(s.K + 1) * stage_bytes;
-    const bool deep = unit_bytes >= kDeepRingMinUnitBytes;
+    const bool deep = unit_bytes >= kDeepRingMinUnitBytes && stage_bytes >= kDeepRingMinChunkBytes;
     int lanes = (int)((kUnitBytesInFlightPerSm + unit_bytes - 1) / unit_bytes);
     lanes = max(2, min(kMaxCtasPerSm, min(lanes, (int)(kShortRingsBytesPerSm / ((size_t)kBf16Stages * stage_bytes)))));
     int want_per_sm = (int)tune("STRATA_DISP_CTAS", deep ? 1 : lanes);
