@@ -3,9 +3,10 @@
 //
 // Work split: a unit is one token (or one column chunk of a token when a row is larger than
 // a stage): 1 row read + K row writes whatever the expert popularity is.  A persistent grid claims
-// units in order from a counter in the workspace, two units ahead of the one being stored, so the
-// claim latency is hidden, CTAs running together work on neighbouring rows, and no CTA is left
-// with a fixed share it cannot finish in time.
+// units in order from a counter in the workspace, a ring's depth ahead of the one being stored, so
+// CTAs running together work on neighbouring rows and no CTA is left with a fixed share it cannot
+// finish in time.  Under the caller's promise that x is complete before the preceding kernel starts
+// (strata_ctx_set_x_early) the first ring of rows is loaded before the wait on that kernel.
 //
 // bf16: each CTA is a single warp that runs the SM's bulk-copy engine as a small DMA program
 //       (the on-SM counterpart of the paper's device-issued SDMA descriptors, Sec. 6.3):
