@@ -928,10 +928,11 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
                 b2b = {k: round(v["back_to_back_us"], 2) for k, v in us.items() if "back_to_back_us" in v}
                 decode_us = {
                     "layout": other[name]["layout_us"], "dispatch": other[name]["dispatch_us"],
-                    "combine": other[name]["combine_us"], "step": other[name]["step_us"],
+                    "combine": other[name]["combine_us"],
+                    "layout+dispatch": round(us["layout+dispatch"]["median_us"], 2), "step": other[name]["step_us"],
                     "step_cuda_graph": round(us["step_graph"]["median_us"], 2),
                     "back_to_back": {"layout": b2b["layout"], "dispatch": b2b["dispatch"], "combine": b2b["combine"],
-                                     "step": b2b["step"]},
+                                     "layout+dispatch": b2b["layout+dispatch"], "step": b2b["step"]},
                     "of_measured_peak": {"dispatch": round(db / us["dispatch"]["median_us"] / 1e3 / peak, 3),
                                          "combine": round(cb / us["combine"]["median_us"] / 1e3 / peak, 3),
                                          "dispatch_back_to_back": round(db / b2b["dispatch"] / 1e3 / peak, 3),

@@ -55,9 +55,9 @@ def test_default_line_carries_the_decode_block_and_stays_short():
     workload is the tiny one so that the test is quick; the line must stay short enough to be kept whole."""
     d = run_bench("--workload", "tiny", "--steps", "5", "--warmup", "3", "--no-cpu", "--no-e2e")
     dec = d["decode_us"]
-    for k in ("layout", "dispatch", "combine", "step", "step_cuda_graph"):
+    for k in ("layout", "dispatch", "combine", "layout+dispatch", "step", "step_cuda_graph"):
         assert 0 < dec[k] < 1000, k
-    assert set(dec["back_to_back"]) == {"layout", "dispatch", "combine", "step"}
+    assert set(dec["back_to_back"]) == {"layout", "dispatch", "combine", "layout+dispatch", "step"}
     assert 0.3 < dec["of_measured_peak"]["dispatch"] < 1.3 and 0.3 < dec["of_measured_peak"]["combine"] < 1.3
     assert dec["step"] >= dec["back_to_back"]["step"] * 0.9
     assert set(d["other_configs"]) == {"tiny", "decode", "skew", "fp8", "skew_shape_uniform_routing"}
