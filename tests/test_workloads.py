@@ -60,3 +60,18 @@ def test_bf16_round_trip_helpers():
 
 def test_expert_of_row():
     assert wl.expert_of_row(np.array([0, 3, 3, 6, 8]), 8).tolist() == [0, 0, 0, 2, 2, 2, 3, 3]
+
+
+def test_bench_traffic_extrapolation_stays_close_to_the_algorithmic_bytes():
+    """The DRAM traffic bench.py reports for a full prefill launch is the straight line through two captures;
+    it must reproduce both captures and land within 2 % of the algorithmic bytes at full size (a kernel that
+    re-read rows or read lines for ownership would show up as a ratio well above 1)."""
+    import bench
+    cfg = wl.CONFIGS["prefill"]
+    for kernel, alg in (("dispatch_bf16_kernel", cfg.dispatch_bytes()), ("combine_kernel", cfg.combine_bytes())):
+        cap = bench.NCU_CAPTURES[kernel]
+        for t, (rd, wr) in cap.items():
+            assert bench.ncu_traffic_bytes(kernel, t) == rd + wr
+        full = bench.ncu_traffic_bytes(kernel, cfg.T)
+        assert 0.98 <= full / alg <= 1.02, (kernel, full / alg)
+    assert bench.ncu_traffic_bytes("dispatch_fp8_kernel", 256) is None
