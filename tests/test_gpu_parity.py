@@ -620,12 +620,15 @@ def test_minus_one_is_an_error_without_the_flag():
 @pytest.mark.parametrize("kw", [dict(R=4, T=300, H=512, E=16, K=4),          # cluster layout, claimed units
                                 dict(R=8, T=1200, H=256, E=32, K=4)],         # tiled layout (38,400 items)
                          ids=lambda kw: "R{R}T{T}H{H}E{E}K{K}".format(**kw))
-def test_cuda_graph_replay(kw):
+@pytest.mark.parametrize("x_early", [False, True], ids=["default", "x_early"])
+def test_cuda_graph_replay(kw, x_early):
     """layout -> dispatch -> combine captured once in a CUDA graph and replayed on new inputs: every
     piece of state the kernels hand from one launch to the next (ticket, work-claim counters) is
-    restored by the kernels themselves, so a replay computes the same as a fresh call."""
+    restored by the kernels themselves, so a replay computes the same as a fresh call.  With the early-x
+    promise the replays keep it: x is rewritten before the graph (hence before its layout) starts."""
     cfg = wl.shrink(wl.CONFIGS["decode"], seed=1, **kw)
     ctx = make_ctx(cfg)
+    ctx.x_early(x_early)
     first = wl.generate(cfg)
     ids_d, x_d, w_d = to_dev(first["ids"]), to_dev(first["x"]), to_dev(first["w"])
     lay = ctx.new_layout()
