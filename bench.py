@@ -937,6 +937,8 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
                                          "combine": round(cb / us["combine"]["median_us"] / 1e3 / peak, 3),
                                          "dispatch_back_to_back": round(db / b2b["dispatch"] / 1e3 / peak, 3),
                                          "combine_back_to_back": round(cb / b2b["combine"] / 1e3 / peak, 3)},
+                    "min_p95": {k: [round(us[k]["min_us"], 2), round(us[k]["p95_us"], 2)]
+                                for k in ("layout", "dispatch", "combine", "step")},
                     "both_copies_at_measured_peak_us": round((db + cb) / peak / 1e3, 1),
                     "how": "median of 30 calls, each between two CUDA events; back_to_back: 30 calls between one "
                            "pair of events; step = layout + dispatch + combine",
