@@ -338,6 +338,20 @@ def per_call_us(case: DeviceCase, iters: int = 30, warmup: int = 3):
         ev[1].record()
         torch.cuda.synchronize()
         out[name]["back_to_back_us"] = ev[0].elapsed_time(ev[1]) * 1e3 / iters
+    # what the bracket itself costs: a one-element torch fill between two events, timed the same way
+    one = torch.zeros(1, device=case.dev)
+    for _ in range(warmup):
+        one.zero_()
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+    torch.cuda._sleep(10_000_000)
+    ev[0].record()
+    for i in range(iters):
+        one.zero_()
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    ts = sorted(ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(iters))
+    out["null_kernel"] = {"median_us": ts[len(ts) // 2], "min_us": ts[0], "p95_us": ts[int(0.95 * (len(ts) - 1))]}
     # the same three calls captured once in a CUDA graph and replayed (launch overhead paid once)
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
@@ -939,9 +953,11 @@ def run_gpu(args, rank: int, local_rank: int, world: int):
                                          "combine_back_to_back": round(cb / b2b["combine"] / 1e3 / peak, 3)},
                     "min_p95": {k: [round(us[k]["min_us"], 2), round(us[k]["p95_us"], 2)]
                                 for k in ("layout", "dispatch", "combine", "step")},
+                    "null_kernel_between_events": round(us["null_kernel"]["median_us"], 2),
                     "both_copies_at_measured_peak_us": round((db + cb) / peak / 1e3, 1),
-                    "how": "median of 30 calls, each between two CUDA events; back_to_back: 30 calls between one "
-                           "pair of events; step = layout + dispatch + combine",
+                    "how": "median of 30 calls, each between two CUDA events (null_kernel_between_events: a one-element "
+                           "fill timed the same way, i.e. what the bracket itself costs); back_to_back: 30 calls "
+                           "between one pair of events; step = layout + dispatch + combine",
                 }
             if name == "skew":
                 # load balance under Zipf routing: per-CTA finish-time spread, and the same shape with
